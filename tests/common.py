@@ -1,0 +1,50 @@
+"""Glue used by the tests: hands the same seeded bytes to the oracle and to the CUDA path."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import oracle
+from paper_2603_01399_b200 import synth
+
+
+def master_getter(shape, seed=0, device="cpu"):
+    """Returns get(kind, layer) -> bf16 torch tensor, regenerated on demand from its own sub-seed."""
+    def get(kind, layer=0):
+        if kind == "embed":
+            return synth.embedding(shape, seed, device)
+        if kind in ("attn_norm", "mlp_norm", "final_norm", "q_norm", "k_norm"):
+            return synth.gain(shape, kind, layer, seed, device)
+        return synth.matrix(shape, kind, layer, seed, device)
+    return get
+
+
+def oracle_model(shape, seed=0, int8=True, device="cpu"):
+    get = master_getter(shape, seed, device)
+    return oracle.build_model(shape, lambda kind, layer: synth.bf16_bits(get(kind, layer)), int8=int8)
+
+
+def oracle_greedy_continuation(model, kv, root_token, n):
+    """n greedy tokens after root_token by single-row verify calls on a scratch copy of the cache."""
+    import copy
+    kv2 = oracle.KVCache(kv.k_bits.copy(), kv.v_bits.copy(), kv.seq_len.copy())
+    out = []
+    tok = int(root_token)
+    for _ in range(n):
+        r = oracle.verify(model, kv2, np.array([[tok]], np.int32), None, np.array([1], np.int32))
+        oracle.kv_commit(kv2, r.accept_len, None)
+        tok = int(r.bonus[0])
+        out.append(tok)
+    return out
+
+
+def prefill_oracle(model, kv, tokens_1d, chunk):
+    """Push tokens through verify in chunks and commit all of them (chain blocks)."""
+    toks = list(int(t) for t in tokens_1d)
+    i = 0
+    while i < len(toks):
+        c = toks[i:i + chunk]
+        t = np.array([c], np.int32)
+        oracle.verify(model, kv, t, None, np.array([len(c)], np.int32), want_logits=False)
+        kv.seq_len[0] += len(c)
+        i += len(c)
