@@ -1,0 +1,361 @@
+#!/usr/bin/env python
+"""Benchmark of the quantised verification pass (Quasar, arXiv 2603.01399) on B200.
+
+One "step" = one whole verify pass (embedding -> 36 decoder layers with int8 weights -> LM head
+-> arg-max -> greedy acceptance) of the Qwen3-8B-shaped workload: batch 1, 1024 cached positions,
+chain draft of 5 (6 block rows).  Inputs are seeded and synthetic (random-init weights of that
+architecture, N(0,1) KV prefix, the bf16 model's greedy continuation corrupted with p = 0.3 as
+the draft); they stand in for the paper's Qwen3-8B runs on Spec-Bench style prompts.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints ONE JSON line.  `--impl reference` times the CPU oracle (the plain fp64 restatement the
+tests compare against) on the host cores, on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2603_01399_b200 import synth  # noqa: E402
+
+WORKLOAD = "qwen3-8b-shaped verify pass: B=1, prefix 1024, chain draft gamma=5 (6 block rows), int8 weights"
+PREFIX, GAMMA, BATCH = 1024, 5, 1
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            return json.load(f), "measured"
+    return {"hbm_gbs": FALLBACK_HBM_GBS}, "fallback"
+
+
+def algorithmic_bytes(shape, batch, t_rows, prefix_total, weight_bytes_per_elem):
+    """Bytes one verify pass has to move (Section 3.4's M * bytes / BW term plus the KV stream)."""
+    w = shape.weight_elems() * weight_bytes_per_elem
+    n_out = sum(n for _, n, _ in shape.linear_shapes()[:4]) * shape.n_layers + shape.vocab
+    scales = n_out * 4 if weight_bytes_per_elem == 1 else 0
+    m = batch * t_rows
+    kv_read = shape.n_layers * prefix_total * shape.n_kv_heads * shape.head_dim * 2 * 2
+    kv_write = shape.n_layers * m * shape.n_kv_heads * shape.head_dim * 2 * 2
+    embed = m * shape.hidden * 2
+    gains = (2 * shape.n_layers + 1) * shape.hidden * 2
+    return {"weights": w, "scales": scales, "kv_read": kv_read, "kv_write": kv_write, "embed": embed,
+            "gains": gains, "total": w + scales + kv_read + kv_write + embed + gains}
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm = [float(r[0]) for r in self.rows if len(r) >= 7 and r[0].replace(".", "").isdigit()]
+        mx = [float(r[1]) for r in self.rows if len(r) >= 7 and r[1].replace(".", "").isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(len(r) >= 7 and r[3 + i] == "Active" for r in self.rows)]
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": reasons, "samples": len(sm)}
+
+
+def master_getter(shape, seed, device):
+    cache = {}
+
+    def get(kind, layer=0):
+        if kind == "embed":
+            if "embed" not in cache:
+                cache["embed"] = synth.embedding(shape, seed, device)
+            return cache["embed"]
+        if kind in ("attn_norm", "mlp_norm", "final_norm", "q_norm", "k_norm"):
+            return synth.gain(shape, kind, layer, seed, device)
+        return synth.matrix(shape, kind, layer, seed, device)
+    return get
+
+
+def greedy_continuation(binding, model, kv, root, n):
+    """n greedy tokens of `model` after `root`, by plain decode steps on a scratch copy of the cache."""
+    scratch = binding.KVCache(model.shape, kv.batch, kv.s_max, k=kv.k.clone(), v=kv.v.clone(),
+                              seq_len=kv.seq_len.clone())
+    buf = binding.VerifyBuffers(model, kv.batch, 1, want_logits=False)
+    tok = root.clone()
+    out = []
+    for _ in range(n):
+        buf.tokens.copy_(tok.view(-1, 1))
+        binding.quasar_verify(model, scratch, buf)
+        binding.quasar_kv_commit(model, scratch, buf)
+        tok = buf.bonus.clone()
+        out.append(tok.clone())
+    torch.cuda.synchronize()
+    return torch.stack(out, dim=1)      # [B][n]
+
+
+# ------------------------------------------------------------------------------------------
+def run_ours(args):
+    from paper_2603_01399_b200 import binding, build
+    build.build()
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    shape = synth.SHAPES["qwen3_8b"]
+    t_rows = GAMMA + 1
+    s_max = PREFIX + 16
+    get = master_getter(shape, 0, "cuda")
+    m_int8 = binding.Model.from_master(shape, get, s_max, int8=True)
+    m_bf16 = binding.Model.from_master(shape, get, s_max, int8=False)
+    kk, vv = synth.kv_prefix(shape, BATCH, s_max, seed=1, device="cuda")
+    kv = binding.KVCache(shape, BATCH, s_max, k=kk, v=vv,
+                         seq_len=torch.full((BATCH,), PREFIX, dtype=torch.int32, device="cuda"))
+    root = synth.uniform_tokens((BATCH,), shape.vocab, synth.sub_seed(2, "tokens")).cuda()
+    greedy = greedy_continuation(binding, m_bf16, kv, root, GAMMA)
+    draft = synth.corrupt_draft(greedy, 0.3, shape.vocab, seed=2)
+    tokens_host = torch.cat([root.cpu().view(-1, 1), draft], dim=1).to(torch.int32).contiguous().pin_memory()
+
+    def timed_plan(model, steps, warmup, sample_clocks):
+        buf = binding.VerifyBuffers(model, BATCH, t_rows, want_logits=False)
+        buf.tokens.copy_(tokens_host)
+        plan = binding.Plan(model, kv, buf)
+        for _ in range(warmup):
+            plan.launch()
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        sampler = ClockSampler(local) if sample_clocks else None
+        if sampler:
+            sampler.start()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        l0 = binding.kernel_launches()
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(steps):
+            plan.launch()
+        e1.record()
+        torch.cuda.synchronize()
+        launches = binding.kernel_launches() - l0
+        clocks = sampler.stop() if sampler else None
+        if dist is not None:
+            dist.barrier()
+        ms = e0.elapsed_time(e1)
+        if dist is not None:
+            t = torch.tensor([ms], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t[0])
+        return ms / steps, buf, plan, launches, clocks
+
+    ms_step, buf, plan, launches, clocks = timed_plan(m_int8, args.steps, args.warmup, True)
+    accepted = int((buf.accept_len + 1).sum())            # accepted drafts + the bonus token, per pass
+    accepted_drafts = int(buf.accept_len.sum())
+    status = int(buf.status[0])
+
+    # end to end: host tokens in, host decision out, every step
+    al = torch.zeros(BATCH, dtype=torch.int32).pin_memory()
+    bo = torch.zeros(BATCH, dtype=torch.int32).pin_memory()
+    for _ in range(3):
+        plan.run_host(tokens_host, al, bo)
+    if dist is not None:
+        dist.barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        plan.run_host(tokens_host, al, bo)
+    e2e_ms = (time.perf_counter() - t0) * 1e3 / args.steps
+    if dist is not None:
+        t = torch.tensor([e2e_ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t[0])
+
+    # the dominant kernel alone: the skinny GEMM over the model's 145 weight matrices in pass order
+    gemm = time_gemm_sweep(binding, m_int8, shape, BATCH * t_rows, max(3, args.steps // 4))
+
+    # bf16-weight sibling pass (the "BF16 verifier" of Section 3.4, same kernels)
+    bf16_ms, bbuf, bplan, _, _ = timed_plan(m_bf16, max(3, args.steps // 4), 3, False)
+
+    peaks, peak_kind = measured_peaks()
+    hbm_peak = float(peaks["hbm_gbs"])
+    ab = algorithmic_bytes(shape, BATCH, t_rows, PREFIX * BATCH, 1)
+    ab16 = algorithmic_bytes(shape, BATCH, t_rows, PREFIX * BATCH, 2)
+    pass_gbs = ab["total"] / (ms_step * 1e-3) / 1e9
+    out = {
+        "metric": "accepted tokens/s of the verify pass (Qwen3-8B shape)", "value": world * accepted / (ms_step * 1e-3),
+        "unit": "tok/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8 weights x bf16, f32 accumulate",
+        "data": "synthetic",
+        "config": {"workload": WORKLOAD, "replicas": world, "batch": BATCH, "prefix": PREFIX, "gamma": GAMMA,
+                   "l2": "inputs (7.7 GB of weights + KV per pass) exceed the 126 MB L2; no flush needed",
+                   "launch": "one CUDA-graph replay per step"},
+        "verify_latency_ms": ms_step, "accepted_per_pass": accepted, "accepted_drafts_per_pass": accepted_drafts,
+        "accepted_drafts_tok_s": world * accepted_drafts / (ms_step * 1e-3), "device_status": status,
+        "pass_bytes": ab, "pass_hbm_gbs": pass_gbs, "pass_hbm_frac_of_measured_copy": pass_gbs / hbm_peak,
+        "pass_hbm_frac_of_nominal_8TBs": pass_gbs / NOMINAL_HBM_GBS,
+        "bf16_sibling": {"verify_latency_ms": bf16_ms, "ratio_vs_int8": bf16_ms / ms_step,
+                         "pass_hbm_gbs": ab16["total"] / (bf16_ms * 1e-3) / 1e9},
+        "clocks": clocks,
+        "e2e": {"value": world * accepted / (e2e_ms * 1e-3), "unit": "tok/s", "ms_per_step": e2e_ms,
+                "h2d_bytes_per_step": tokens_host.numel() * 4, "d2h_bytes_per_step": 2 * BATCH * 4},
+        "gpu_launches": int(launches),
+        "roofline": {"bound": "hbm", "kernel": "skinny_gemm_kernel (145 launches per pass, timed alone over the model's weights)",
+                     "achieved": gemm["gbs"], "peak": hbm_peak, "unit": "GB/s", "frac": gemm["gbs"] / hbm_peak,
+                     "peak_kind": f"{peak_kind} copy bandwidth", "traffic": None,
+                     "avg_launch_us": gemm["avg_us"], "bytes_per_launch": gemm["bytes_per_launch"]},
+    }
+    if rank == 0:
+        out["cpu_baseline"] = cpu_baseline(shape, accepted)
+        print(json.dumps(out))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def time_gemm_sweep(binding, model, shape, m_rows, reps):
+    """All GEMM launches of one pass, back to back, between two events on the launching stream."""
+    t = model.tensors
+    x_h = synth.normal_bf16((m_rows, shape.hidden), 1.0, 5, "cuda")
+    x_q = synth.normal_bf16((m_rows, shape.q_dim), 1.0, 6, "cuda")
+    x_f = synth.normal_bf16((m_rows, shape.ffn), 1.0, 7, "cuda")
+    outs = {n: torch.empty((m_rows, n), dtype=torch.bfloat16, device="cuda")
+            for n in (shape.qkv_dim, shape.hidden, 2 * shape.ffn)}
+    logits = torch.empty((m_rows, shape.vocab), dtype=torch.float32, device="cuda")
+    ws = torch.zeros(model.workspace_bytes(BATCH, m_rows // BATCH), dtype=torch.uint8, device="cuda")
+    jobs = []
+    for l in range(shape.n_layers):
+        jobs += [(x_h, t[f"l{l}.qkv_w"], t[f"l{l}.qkv_delta"], outs[shape.qkv_dim], False),
+                 (x_q, t[f"l{l}.o_w"], t[f"l{l}.o_delta"], outs[shape.hidden], False),
+                 (x_h, t[f"l{l}.gateup_w"], t[f"l{l}.gateup_delta"], outs[2 * shape.ffn], False),
+                 (x_f, t[f"l{l}.down_w"], t[f"l{l}.down_delta"], outs[shape.hidden], False)]
+    jobs.append((x_h, t["lm_w"], t["lm_delta"], logits, True))
+    nbytes = sum(j[1].numel() + j[2].numel() * 4 for j in jobs)
+
+    def sweep():
+        for x, w, d, y, f32 in jobs:
+            binding.quasar_linear(x, w, d, out_f32=f32, workspace=ws, out=y)
+    sweep()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        sweep()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / reps
+    return {"gbs": nbytes / (ms * 1e-3) / 1e9, "avg_us": ms * 1e3 / len(jobs), "bytes_per_launch": nbytes / len(jobs),
+            "launches": len(jobs)}
+
+
+# ------------------------------------------------------------------------------------------
+def oracle_sample(shape, n_layers_sample=1):
+    """Times the CPU oracle on a bounded sample of the workload: `n_layers_sample` decoder layers
+    (with the 1024-position KV prefix) and the LM head, at the full Qwen3-8B widths.  Returns
+    (seconds per layer, seconds for embedding + final norm + LM head + acceptance, threads)."""
+    import oracle
+    small = synth.ModelShape("sample", n_layers_sample, shape.hidden, shape.n_q_heads, shape.n_kv_heads,
+                             shape.head_dim, shape.ffn, shape.vocab, shape.qk_norm, shape.rope_theta, shape.rms_eps)
+    get = master_getter(small, 0, "cpu")
+    om = oracle.build_model(small, lambda kind, layer: synth.bf16_bits(get(kind, layer)), int8=True)
+    kk, vv = synth.kv_prefix(small, BATCH, PREFIX + 16, seed=1)
+    okv = oracle.KVCache(synth.bf16_bits(kk), synth.bf16_bits(vv), np.full(BATCH, PREFIX, np.int32))
+    toks = synth.uniform_tokens((BATCH, GAMMA + 1), shape.vocab, synth.sub_seed(2, "tokens")).numpy()
+    bl = np.full(BATCH, GAMMA + 1, np.int32)
+    t0 = time.perf_counter()
+    oracle.verify(om, okv, toks, None, bl, n_layers_run=0)
+    t_head = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    oracle.verify(om, okv, toks, None, bl, want_logits=False)
+    t_layers = time.perf_counter() - t0
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+    except Exception:
+        threads = os.cpu_count() or 1
+    return t_layers / n_layers_sample, t_head, threads
+
+
+def cpu_baseline(shape, accepted):
+    per_layer, head, threads = oracle_sample(shape)
+    full = per_layer * shape.n_layers + head
+    return {"value": accepted / full, "unit": "tok/s", "cores": threads, "kind": "oracle",
+            "sample": f"1 of {shape.n_layers} decoder layers ({per_layer:.2f} s) + LM head and acceptance ({head:.2f} s) "
+                      f"at full Qwen3-8B widths, B=1, prefix 1024, 6 block rows; scaled to {shape.n_layers} layers "
+                      f"= {full:.1f} s per pass",
+            "seconds_per_pass_extrapolated": full, "host_cpus": os.cpu_count()}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    shape = synth.SHAPES["qwen3_8b"]
+    times = []
+    threads = 1
+    for i in range(args.warmup + args.steps):
+        per_layer, head, threads = oracle_sample(shape)
+        if i >= args.warmup:
+            times.append(per_layer * shape.n_layers + head)
+    full = sum(times) / len(times)
+    accepted = 1.0   # the oracle's pass emits at least the bonus token; drafts are not generated on this arm
+    val = accepted / full
+    print(json.dumps({
+        "impl": "reference", "metric": "accepted tokens/s of the verify pass (Qwen3-8B shape)", "value": val,
+        "unit": "tok/s", "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": full * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": {"workload": WORKLOAD},
+        "cpu_baseline": {"value": val, "unit": "tok/s", "kind": "oracle", "cores": threads,
+                         "sample": "each step: 1 of 36 decoder layers + LM head at full widths, scaled to 36 layers; "
+                                   "counts the bonus token only (1 token per pass)"},
+        "e2e": {"value": val, "unit": "tok/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,237 @@
+/*
+ * quasar.h — C ABI of the B200 (sm_100a) quantised verification pass.
+ *
+ * The library implements the verification half of one speculative-decoding
+ * iteration (Quasar, arXiv 2603.01399, Section 3.1 "Verification" and
+ * Section 3.3): the target decoder, holding low-bit weights, scores a block of
+ * drafted tokens against its KV cache in ONE parallel forward pass, then the
+ * longest draft prefix that agrees with the verifier's own top-1 choices is
+ * accepted and one more token (the verifier's) is emitted.
+ *
+ * Weights are int8, symmetric, one fp32 step size per output channel
+ * (Section 3.2, Eq. 6-8: W_int8 = Q(W, delta_w), Y ~= delta_w * (W_int8 X));
+ * activations stay bf16 and accumulation is fp32.  A bf16-weight pass built
+ * from the same kernels (the "BF16 verifier" the paper compares with,
+ * Section 3.4 Eq. 11) is selected with weight_dtype = QUASAR_W_BF16.
+ *
+ * Conventions
+ *  - C linkage; every function returns QUASAR_OK (0) or a negative error code
+ *    and never throws or aborts.  quasar_last_error() gives a thread-local
+ *    message for the last failing call of the calling thread.
+ *  - Unless a parameter says "host", every pointer is DEVICE memory owned by
+ *    the caller, 16-byte aligned, valid until the work queued by the call has
+ *    finished.  The library allocates no device memory per call; scratch comes
+ *    from a caller-provided workspace (quasar_workspace_bytes).
+ *  - `stream` is a cudaStream_t passed as void*.  Calls only enqueue work
+ *    (no synchronisation, no allocation), so they may be stream-captured;
+ *    results are valid once the stream has been synchronised.
+ *  - Argument errors that the host can see are reported before anything is
+ *    launched.  Errors only the device can see (a token id out of range, a
+ *    malformed parent array, a sequence that would overflow its cache) set the
+ *    caller's `status` word to a negative code; the offending sequence is
+ *    skipped, nothing is written out of bounds and nothing traps.
+ *  - Matrices are row-major with the contraction index contiguous:
+ *    W is [N][K] = [d_out][d_in] (the paper's W in R^{d_out x d_in}, Section 3.2).
+ */
+#ifndef QUASAR_H_
+#define QUASAR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define QUASAR_OK 0
+#define QUASAR_ERR_INVALID_ARG (-1) /* null pointer, negative size, bad enum     */
+#define QUASAR_ERR_SHAPE (-2)       /* size not supported (see each call)        */
+#define QUASAR_ERR_CAPACITY (-3)    /* workspace / cache / batch limit exceeded  */
+#define QUASAR_ERR_ALIGN (-4)       /* pointer not 16-byte aligned               */
+#define QUASAR_ERR_CUDA (-5)        /* a CUDA runtime call failed                */
+#define QUASAR_ERR_TIMEOUT (-6)     /* a bounded device-side wait ran out        */
+#define QUASAR_ERR_TOKEN (-7)       /* device: token id outside [0, vocab)       */
+#define QUASAR_ERR_TREE (-8)        /* device: parents[] is not a rooted forest order */
+
+#define QUASAR_W_INT8 0
+#define QUASAR_W_BF16 1
+
+#define QUASAR_MAX_BLOCK 64 /* rows of one sequence's draft block (root + drafts / tree nodes) */
+
+const char* quasar_last_error(void);
+
+/* ------------------------------------------------------------------------
+ * Offline weight preparation (Section 3.3 "Offline Weight Preparation";
+ * Q(., delta) of Section 3.2 Eq. 6).  Per output channel n:
+ *   delta[n] = max_k |W[n][k]| / 127   (fp32 IEEE division; 1.0f for an all-zero row)
+ *   q[n][k]  = clamp(round_half_even(W[n][k] / delta[n]), -127, 127)   (fp32 division)
+ * w_bf16: [N][K] bf16.  q_out: [N][K] int8.  delta_out: [N] fp32.  K % 8 == 0.
+ * Bit-exact with the definition above; no fast-math anywhere on this path.
+ * ---------------------------------------------------------------------- */
+int quasar_quantize(const void* w_bf16, int64_t N, int64_t K, int8_t* q_out, float* delta_out, void* stream);
+
+/* ------------------------------------------------------------------------
+ * One quantised linear layer (Section 3.2 Eq. 8 / Section 3.3 Eq. 10, weight-only):
+ *   Y[m][n] = delta[n] * sum_k X[m][k] * (float)W[n][k]   (+ R[m][n] if residual != NULL)
+ * x: [M][K] bf16.  w: [N][K] int8 (weight_dtype = QUASAR_W_INT8) or bf16
+ * (QUASAR_W_BF16, delta ignored and may be NULL).  y: [M][N], bf16 or fp32
+ * (y_is_f32).  residual: [M][N] bf16 or NULL; with a residual the product is
+ * first rounded to bf16, then added, then rounded again (the order the decoder
+ * layer uses).  y may alias residual.  M >= 1 (rows are processed in groups of
+ * at most 72), K % 16 == 0, N >= 1.
+ * workspace: at least quasar_linear_workspace_bytes(M, N, K) bytes; its first
+ * use must find it zero-filled and every call leaves it reusable by the next.
+ * ---------------------------------------------------------------------- */
+int quasar_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, size_t* bytes_out /* host */);
+int quasar_linear(const void* x, const void* w, const float* delta, int32_t weight_dtype, int64_t M, int64_t N,
+                  int64_t K, void* y, int32_t y_is_f32, const void* residual, void* workspace,
+                  size_t workspace_bytes, void* stream);
+
+/* ------------------------------------------------------------------------
+ * Model description.  The paper fixes only the linear layers; the rest of the
+ * decoder layer (Section 3.3: "non-linear layers" stay in high precision) is a
+ * pre-norm decoder: RMSNorm (y = x * rsqrt(mean(x^2) + eps) * g), optional
+ * per-head RMSNorm of q and k over head_dim before RoPE, rotate-half RoPE
+ * (pairs (i, i + head_dim/2), inv_freq_i = theta^(-2i/head_dim)), grouped-query
+ * attention, SwiGLU  down(silu(gate) * up), no biases, untied LM head.
+ * ---------------------------------------------------------------------- */
+typedef struct quasar_config {
+  int32_t n_layers;
+  int32_t hidden;       /* H, multiple of 16                                  */
+  int32_t n_q_heads;    /* Hq, multiple of n_kv_heads, Hq / Hkv <= 8          */
+  int32_t n_kv_heads;   /* Hkv                                                */
+  int32_t head_dim;     /* D: 64 or 128                                       */
+  int32_t ffn;          /* F, multiple of 16                                  */
+  int32_t vocab;        /* V                                                  */
+  int32_t qk_norm;      /* 1: per-head RMSNorm of q and k before RoPE         */
+  float rope_theta;
+  float rms_eps;
+  int32_t weight_dtype; /* QUASAR_W_INT8 or QUASAR_W_BF16                     */
+  int32_t max_seq;      /* cache capacity S_max (positions) the RoPE table covers */
+} quasar_config;
+
+typedef struct quasar_layer_weights {
+  const void* attn_norm;  /* bf16 [H]                                             */
+  const void* qkv_w;      /* [(Hq + 2 Hkv) D][H]: q heads, then k heads, then v   */
+  const float* qkv_delta; /* fp32 [(Hq + 2 Hkv) D]   (NULL for bf16 weights)      */
+  const void* q_norm;     /* bf16 [D] or NULL when qk_norm == 0                   */
+  const void* k_norm;     /* bf16 [D] or NULL                                     */
+  const void* o_w;        /* [H][Hq D]                                            */
+  const float* o_delta;
+  const void* mlp_norm;   /* bf16 [H]                                             */
+  const void* gateup_w;   /* [2F][H]: rows [0,F) gate, rows [F,2F) up             */
+  const float* gateup_delta;
+  const void* down_w;     /* [H][F]                                               */
+  const float* down_delta;
+} quasar_layer_weights;
+
+typedef struct quasar_weights {
+  const void* embed;                  /* bf16 [V][H]                               */
+  const quasar_layer_weights* layers; /* HOST array of n_layers entries (device pointers inside) */
+  const void* final_norm;             /* bf16 [H]                                  */
+  const void* lm_w;                   /* [V][H]                                    */
+  const float* lm_delta;              /* fp32 [V]                                  */
+} quasar_weights;
+
+/* KV cache of the context x_<t (Section 3.1): bf16, [L][B][Hkv][S_max][D], K
+ * already rotated.  seq_len[b] = positions of sequence b that are committed. */
+typedef struct quasar_kv {
+  void* k;
+  void* v;
+  int32_t* seq_len; /* device int32 [batch]                                       */
+  int32_t batch;    /* B the cache was laid out for                               */
+  int32_t s_max;    /* <= config.max_seq                                          */
+} quasar_kv;
+
+typedef struct quasar_model quasar_model;
+
+/* The model borrows every weight pointer (they must outlive it) and owns a
+ * RoPE cos/sin table built in fp64 on the device.  Allocates; not capturable. */
+int quasar_model_create(const quasar_config* cfg /* host */, const quasar_weights* w /* host */, quasar_model** out);
+int quasar_model_destroy(quasar_model* m);
+
+/* Bytes of scratch quasar_verify needs for batch B and T_max block rows. */
+int quasar_workspace_bytes(const quasar_model* m, int32_t B, int32_t T_max, size_t* bytes_out /* host */);
+
+/* ------------------------------------------------------------------------
+ * The verification pass (Section 3.1 "Verification", Section 3.3) with greedy
+ * acceptance (Eq. 2 at temperature 0: a draft token is kept while it equals the
+ * verifier's top-1 prediction).
+ *
+ * tokens     int32 [B][T_max]; row 0 of a sequence is its last emitted token
+ *            (not yet in the cache), rows 1.. are the drafted tokens (chain) or
+ *            tree nodes.
+ * parents    NULL for chains (row i follows row i-1); else int32 [B][T_max] with
+ *            parents[b][0] = -1 and 0 <= parents[b][i] < i.  Row i sits at
+ *            position seq_len[b] + depth(i) and attends to the whole cached
+ *            prefix, its ancestors and itself.
+ * block_len  int32 [B], 1 <= block_len[b] <= T_max <= QUASAR_MAX_BLOCK; rows
+ *            beyond it are ignored (1 = one plain decode step).
+ * logits_out fp32 [B][T_max][V] or NULL.  Row i predicts the token after row i.
+ * accept_len int32 [B]: number of accepted DRAFT tokens, in [0, block_len-1].
+ * bonus      int32 [B]: the verifier's token after the last accepted row.
+ * accept_path int32 [B][T_max] or NULL: accept_path[b][d] = block row accepted at
+ *            depth d (entry 0 is the root, entries past accept_len are -1).
+ * status     int32 [1]: left untouched on success, else a negative code.
+ *
+ * K and V of every block row are written to cache slot seq_len[b] + row; seq_len
+ * is not changed, so the call is idempotent until quasar_kv_commit.  Ties in the
+ * argmax go to the lowest token id; equal sibling tokens to the lowest row.
+ * ---------------------------------------------------------------------- */
+int quasar_verify(quasar_model* m, const quasar_kv* kv /* host struct */, const int32_t* tokens,
+                  const int32_t* parents, const int32_t* block_len, int32_t B, int32_t T_max, float* logits_out,
+                  int32_t* accept_len, int32_t* bonus, int32_t* accept_path, void* workspace,
+                  size_t workspace_bytes, int32_t* status, void* stream);
+
+/* ------------------------------------------------------------------------
+ * Commit the accepted tokens (the cache reuse Section 3.1 implies between
+ * iterations).  Chain (accept_path NULL): seq_len[b] += 1 + accept_len[b].
+ * Tree: K,V of the accepted row at depth d move to slot seq_len[b] + d for
+ * d = 1..accept_len[b], then the same bump.  The only call that changes seq_len.
+ * ---------------------------------------------------------------------- */
+int quasar_kv_commit(quasar_model* m, const quasar_kv* kv /* host struct */, const int32_t* accept_len,
+                     const int32_t* accept_path, int32_t B, int32_t T_max, void* stream);
+
+/* ------------------------------------------------------------------------
+ * A verify pass frozen into a CUDA graph: same arguments as quasar_verify,
+ * captured once, replayed with one launch.  Every pointer is baked in; their
+ * CONTENTS may change between launches.  quasar_plan_create captures on an
+ * internal stream and synchronises it (not capturable itself).
+ * ---------------------------------------------------------------------- */
+typedef struct quasar_plan quasar_plan;
+int quasar_plan_create(quasar_model* m, const quasar_kv* kv, const int32_t* tokens, const int32_t* parents,
+                       const int32_t* block_len, int32_t B, int32_t T_max, float* logits_out, int32_t* accept_len,
+                       int32_t* bonus, int32_t* accept_path, void* workspace, size_t workspace_bytes,
+                       int32_t* status, quasar_plan** out);
+int quasar_plan_launch(quasar_plan* p, void* stream);
+int quasar_plan_destroy(quasar_plan* p);
+
+/* The call a serving loop makes with HOST buffers: copies tokens (and parents,
+ * block_len when given) from host memory into the plan's device buffers,
+ * replays the plan, copies accept_len, bonus (and accept_path, status) back and
+ * synchronises the stream.  Host buffers should be pinned for the copies to be
+ * asynchronous.  Any host pointer except tokens_host may be NULL (that
+ * transfer is skipped). */
+int quasar_plan_run_host(quasar_plan* p, const int32_t* tokens_host, const int32_t* parents_host,
+                         const int32_t* block_len_host, int32_t* accept_len_host, int32_t* bonus_host,
+                         int32_t* accept_path_host, int32_t* status_host, void* stream);
+
+/* ------------------------------------------------------------------------
+ * Debug tap: when a trace buffer is set, quasar_verify copies every
+ * intermediate tensor into it in a fixed order (see quasar_trace_bytes) so each
+ * step of the pass can be compared on its own.  Pass NULL to switch it off.
+ * Per call: embed [M][H]; per layer: h1 [M][H], qkv [M][(Hq+2Hkv)D] (before
+ * RoPE), q [M][(Hq+2Hkv)D] (the same buffer after QK-norm + RoPE of its q part),
+ * attn [M][Hq D], x_attn [M][H], act [M][F], x_mlp [M][H]; then hf [M][H].
+ * All bf16, M = B * T_max rows.
+ * ---------------------------------------------------------------------- */
+int quasar_trace_bytes(const quasar_model* m, int32_t B, int32_t T_max, size_t* bytes_out /* host */);
+int quasar_set_trace(quasar_model* m, void* trace_buf, size_t bytes);
+
+/* Count of kernels the library has launched in this process (all calls). */
+int64_t quasar_kernel_launches(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QUASAR_H_ */

@@ -1,0 +1,333 @@
+"""ctypes binding of libquasar.so: same names as the C ABI, argument marshalling only.
+
+PyTorch is used for device memory and the current CUDA stream; every step of the
+verification pass runs inside the library's kernels.  There is no CPU fallback: if
+the library has not been built, `lib()` raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, List, Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libquasar.so")
+
+QUASAR_W_INT8 = 0
+QUASAR_W_BF16 = 1
+QUASAR_MAX_BLOCK = 64
+
+ERROR_NAMES = {0: "OK", -1: "INVALID_ARG", -2: "SHAPE", -3: "CAPACITY", -4: "ALIGN", -5: "CUDA", -6: "TIMEOUT",
+               -7: "TOKEN", -8: "TREE"}
+
+
+class QuasarError(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__(f"quasar error {code} ({ERROR_NAMES.get(code, '?')}): {msg}")
+        self.code = code
+
+
+class Config(C.Structure):
+    _fields_ = [("n_layers", C.c_int32), ("hidden", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
+                ("head_dim", C.c_int32), ("ffn", C.c_int32), ("vocab", C.c_int32), ("qk_norm", C.c_int32),
+                ("rope_theta", C.c_float), ("rms_eps", C.c_float), ("weight_dtype", C.c_int32),
+                ("max_seq", C.c_int32)]
+
+
+class LayerWeights(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in
+                ("attn_norm", "qkv_w", "qkv_delta", "q_norm", "k_norm", "o_w", "o_delta", "mlp_norm", "gateup_w",
+                 "gateup_delta", "down_w", "down_delta")]
+
+
+class Weights(C.Structure):
+    _fields_ = [("embed", C.c_void_p), ("layers", C.POINTER(LayerWeights)), ("final_norm", C.c_void_p),
+                ("lm_w", C.c_void_p), ("lm_delta", C.c_void_p)]
+
+
+class KV(C.Structure):
+    _fields_ = [("k", C.c_void_p), ("v", C.c_void_p), ("seq_len", C.c_void_p), ("batch", C.c_int32),
+                ("s_max", C.c_int32)]
+
+
+_lib = None
+
+_vp, _i32, _i64, _sz = C.c_void_p, C.c_int32, C.c_int64, C.c_size_t
+_verify_args = [_vp, C.POINTER(KV), _vp, _vp, _vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
+SIGNATURES = {
+    "quasar_last_error": (C.c_char_p, []),
+    "quasar_kernel_launches": (_i64, []),
+    "quasar_quantize": (C.c_int, [_vp, _i64, _i64, _vp, _vp, _vp]),
+    "quasar_linear_workspace_bytes": (C.c_int, [_i64, _i64, _i64, C.POINTER(_sz)]),
+    "quasar_linear": (C.c_int, [_vp, _vp, _vp, _i32, _i64, _i64, _i64, _vp, _i32, _vp, _vp, _sz, _vp]),
+    "quasar_model_create": (C.c_int, [C.POINTER(Config), C.POINTER(Weights), C.POINTER(_vp)]),
+    "quasar_model_destroy": (C.c_int, [_vp]),
+    "quasar_workspace_bytes": (C.c_int, [_vp, _i32, _i32, C.POINTER(_sz)]),
+    "quasar_verify": (C.c_int, _verify_args + [_vp]),
+    "quasar_kv_commit": (C.c_int, [_vp, C.POINTER(KV), _vp, _vp, _i32, _i32, _vp]),
+    "quasar_plan_create": (C.c_int, _verify_args + [C.POINTER(_vp)]),
+    "quasar_plan_launch": (C.c_int, [_vp, _vp]),
+    "quasar_plan_destroy": (C.c_int, [_vp]),
+    "quasar_plan_run_host": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "quasar_trace_bytes": (C.c_int, [_vp, _i32, _i32, C.POINTER(_sz)]),
+    "quasar_set_trace": (C.c_int, [_vp, _vp, _sz]),
+}
+
+
+def lib() -> C.CDLL:
+    """Loads the CUDA library; raises if it has not been built (there is no fallback)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2603_01399_b200.build`")
+        l = C.CDLL(LIB_PATH)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(l, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib = l
+    return _lib
+
+
+def _check(rc: int) -> None:
+    if rc != 0:
+        raise QuasarError(rc, lib().quasar_last_error().decode())
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else t.data_ptr()
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def kernel_launches() -> int:
+    return int(lib().quasar_kernel_launches())
+
+
+# ------------------------------------------------------------------------------------------
+def quasar_quantize(w_bf16: torch.Tensor):
+    """bf16 [N][K] on the device -> (int8 [N][K], fp32 [N])."""
+    assert w_bf16.is_cuda and w_bf16.dtype == torch.bfloat16 and w_bf16.is_contiguous() and w_bf16.dim() == 2
+    n, k = w_bf16.shape
+    q = torch.empty((n, k), dtype=torch.int8, device=w_bf16.device)
+    d = torch.empty((n,), dtype=torch.float32, device=w_bf16.device)
+    _check(lib().quasar_quantize(_ptr(w_bf16), n, k, _ptr(q), _ptr(d), _stream()))
+    return q, d
+
+
+def quasar_linear_workspace_bytes(m: int, n: int, k: int) -> int:
+    out = _sz(0)
+    _check(lib().quasar_linear_workspace_bytes(m, n, k, C.byref(out)))
+    return int(out.value)
+
+
+def quasar_linear(x: torch.Tensor, w: torch.Tensor, delta: Optional[torch.Tensor], residual=None, out_f32=False,
+                  workspace: Optional[torch.Tensor] = None, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """x bf16 [M][K]; w int8 or bf16 [N][K]; delta fp32 [N] (int8 weights)."""
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.is_contiguous() and w.is_contiguous()
+    m, k = x.shape
+    n = w.shape[0]
+    wd = QUASAR_W_INT8 if w.dtype == torch.int8 else QUASAR_W_BF16
+    if out is None:
+        out = torch.empty((m, n), dtype=torch.float32 if out_f32 else torch.bfloat16, device=x.device)
+    if workspace is None:
+        workspace = torch.zeros(max(quasar_linear_workspace_bytes(m, n, k), 16), dtype=torch.uint8, device=x.device)
+    _check(lib().quasar_linear(_ptr(x), _ptr(w), _ptr(delta), wd, m, n, k, _ptr(out), 1 if out_f32 else 0,
+                               _ptr(residual), _ptr(workspace), workspace.numel(), _stream()))
+    return out
+
+
+# ------------------------------------------------------------------------------------------
+class Model:
+    """Owns the device weight tensors (keeps them alive) and the library's model handle.
+
+    `tensors` maps names to device tensors: embed, final_norm, lm_w, lm_delta and per layer l
+    `l{l}.attn_norm`, `.qkv_w`, `.qkv_delta`, `.q_norm`, `.k_norm`, `.o_w`, `.o_delta`, `.mlp_norm`,
+    `.gateup_w`, `.gateup_delta`, `.down_w`, `.down_delta` (deltas absent for bf16 weights)."""
+
+    def __init__(self, shape, tensors: Dict[str, torch.Tensor], max_seq: int, weight_dtype: int = QUASAR_W_INT8):
+        self.shape = shape
+        self.tensors = tensors
+        self.weight_dtype = weight_dtype
+        self.max_seq = max_seq
+        self.cfg = Config(shape.n_layers, shape.hidden, shape.n_q_heads, shape.n_kv_heads, shape.head_dim, shape.ffn,
+                          shape.vocab, 1 if shape.qk_norm else 0, shape.rope_theta, shape.rms_eps, weight_dtype,
+                          max_seq)
+        layers = (LayerWeights * max(shape.n_layers, 1))()
+        for l in range(shape.n_layers):
+            for name, _ in LayerWeights._fields_:
+                setattr(layers[l], name, _ptr(tensors.get(f"l{l}.{name}")))
+        self._layers = layers
+        w = Weights(_ptr(tensors["embed"]), layers, _ptr(tensors["final_norm"]), _ptr(tensors["lm_w"]),
+                    _ptr(tensors.get("lm_delta")))
+        handle = _vp()
+        _check(lib().quasar_model_create(C.byref(self.cfg), C.byref(w), C.byref(handle)))
+        self.handle = handle
+        self._trace = None
+
+    @classmethod
+    def from_master(cls, shape, get_master, max_seq: int, int8: bool = True, device="cuda"):
+        """get_master(kind, layer) -> bf16 master tensor (any device).  int8=True quantises every
+        matrix on the GPU with quasar_quantize (the offline weight preparation)."""
+        t: Dict[str, torch.Tensor] = {}
+
+        def put_linear(prefix, kind, layer):
+            w = get_master(kind, layer).to(device)
+            if int8:
+                q, d = quasar_quantize(w)
+                t[prefix + "_w"], t[prefix + "_delta"] = q, d
+            else:
+                t[prefix + "_w"] = w
+
+        t["embed"] = get_master("embed", 0).to(device)
+        t["final_norm"] = get_master("final_norm", 0).to(device)
+        put_linear("lm", "lm_head", 0)
+        for l in range(shape.n_layers):
+            t[f"l{l}.attn_norm"] = get_master("attn_norm", l).to(device)
+            t[f"l{l}.mlp_norm"] = get_master("mlp_norm", l).to(device)
+            if shape.qk_norm:
+                t[f"l{l}.q_norm"] = get_master("q_norm", l).to(device)
+                t[f"l{l}.k_norm"] = get_master("k_norm", l).to(device)
+            put_linear(f"l{l}.qkv", "qkv", l)
+            put_linear(f"l{l}.o", "o", l)
+            put_linear(f"l{l}.gateup", "gateup", l)
+            put_linear(f"l{l}.down", "down", l)
+        torch.cuda.synchronize()
+        return cls(shape, t, max_seq, QUASAR_W_INT8 if int8 else QUASAR_W_BF16)
+
+    def workspace_bytes(self, batch: int, t_max: int) -> int:
+        out = _sz(0)
+        _check(lib().quasar_workspace_bytes(self.handle, batch, t_max, C.byref(out)))
+        return int(out.value)
+
+    def trace_bytes(self, batch: int, t_max: int) -> int:
+        out = _sz(0)
+        _check(lib().quasar_trace_bytes(self.handle, batch, t_max, C.byref(out)))
+        return int(out.value)
+
+    def set_trace(self, buf: Optional[torch.Tensor]) -> None:
+        self._trace = buf
+        _check(lib().quasar_set_trace(self.handle, _ptr(buf), 0 if buf is None else buf.numel() * buf.element_size()))
+
+    def weight_bytes(self) -> int:
+        return sum(v.numel() * v.element_size() for k, v in self.tensors.items()
+                   if k.endswith("_w") or k.endswith("_delta"))
+
+    def close(self) -> None:
+        if self.handle is not None:
+            lib().quasar_model_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+class KVCache:
+    """bf16 K and V [L][B][Hkv][S_max][D] and int32 seq_len [B] on the device."""
+
+    def __init__(self, shape, batch: int, s_max: int, device="cuda", k=None, v=None, seq_len=None):
+        dims = (shape.n_layers, batch, shape.n_kv_heads, s_max, shape.head_dim)
+        self.k = torch.zeros(dims, dtype=torch.bfloat16, device=device) if k is None else k
+        self.v = torch.zeros(dims, dtype=torch.bfloat16, device=device) if v is None else v
+        assert tuple(self.k.shape) == dims and tuple(self.v.shape) == dims
+        self.seq_len = torch.zeros(batch, dtype=torch.int32, device=device) if seq_len is None else seq_len
+        self.batch, self.s_max = batch, s_max
+        self.c = KV(_ptr(self.k), _ptr(self.v), _ptr(self.seq_len), batch, s_max)
+
+
+class VerifyBuffers:
+    """Device buffers of one verify call (inputs, outputs, workspace)."""
+
+    def __init__(self, model: Model, batch: int, t_max: int, want_logits: bool = True, tree: bool = False,
+                 device="cuda"):
+        self.batch, self.t_max = batch, t_max
+        self.tokens = torch.zeros((batch, t_max), dtype=torch.int32, device=device)
+        self.parents = torch.zeros((batch, t_max), dtype=torch.int32, device=device) if tree else None
+        self.block_len = torch.full((batch,), t_max, dtype=torch.int32, device=device)
+        self.logits = torch.zeros((batch, t_max, model.shape.vocab), dtype=torch.float32, device=device) \
+            if want_logits else None
+        self.accept_len = torch.zeros(batch, dtype=torch.int32, device=device)
+        self.bonus = torch.zeros(batch, dtype=torch.int32, device=device)
+        self.accept_path = torch.zeros((batch, t_max), dtype=torch.int32, device=device)
+        self.status = torch.zeros(4, dtype=torch.int32, device=device)
+        self.workspace = torch.zeros(model.workspace_bytes(batch, t_max), dtype=torch.uint8, device=device)
+
+    def args(self, model: Model, kv: KVCache):
+        return (model.handle, C.byref(kv.c), _ptr(self.tokens), _ptr(self.parents), _ptr(self.block_len), self.batch,
+                self.t_max, _ptr(self.logits), _ptr(self.accept_len), _ptr(self.bonus), _ptr(self.accept_path),
+                _ptr(self.workspace), self.workspace.numel(), _ptr(self.status))
+
+
+def quasar_verify(model: Model, kv: KVCache, buf: VerifyBuffers) -> None:
+    """Enqueues one verification pass on the current stream; results land in `buf`."""
+    _check(lib().quasar_verify(*buf.args(model, kv), _stream()))
+
+
+def quasar_kv_commit(model: Model, kv: KVCache, buf: VerifyBuffers, tree: bool = False) -> None:
+    _check(lib().quasar_kv_commit(model.handle, C.byref(kv.c), _ptr(buf.accept_len),
+                                  _ptr(buf.accept_path) if tree else None, buf.batch, buf.t_max, _stream()))
+
+
+class Plan:
+    """A verify pass captured into a CUDA graph by the library."""
+
+    def __init__(self, model: Model, kv: KVCache, buf: VerifyBuffers):
+        self.model, self.kv, self.buf = model, kv, buf
+        h = _vp()
+        _check(lib().quasar_plan_create(*buf.args(model, kv), C.byref(h)))
+        self.handle = h
+
+    def launch(self) -> None:
+        _check(lib().quasar_plan_launch(self.handle, _stream()))
+
+    def run_host(self, tokens_host: torch.Tensor, accept_len_host: torch.Tensor, bonus_host: torch.Tensor,
+                 block_len_host=None, parents_host=None, accept_path_host=None, status_host=None) -> None:
+        """Host (pinned) buffers in, host buffers out; returns after the stream has drained."""
+        _check(lib().quasar_plan_run_host(self.handle, _ptr(tokens_host), _ptr(parents_host), _ptr(block_len_host),
+                                          _ptr(accept_len_host), _ptr(bonus_host), _ptr(accept_path_host),
+                                          _ptr(status_host), _stream()))
+
+    def close(self) -> None:
+        if self.handle is not None:
+            lib().quasar_plan_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def split_trace(model: Model, buf_bytes: torch.Tensor, batch: int, t_max: int) -> Dict[str, torch.Tensor]:
+    """Cuts a trace buffer into named bf16 tensors [B][T_max][width] in the order the library writes them."""
+    s = model.shape
+    m = batch * t_max
+    qkv_w = s.qkv_dim
+    flat = buf_bytes.view(torch.bfloat16)
+    out: Dict[str, torch.Tensor] = {}
+    off = 0
+
+    def take(name, width):
+        nonlocal off
+        out[name] = flat[off: off + m * width].view(batch, t_max, width)
+        off += m * width
+
+    take("embed", s.hidden)
+    for l in range(s.n_layers):
+        take(f"l{l}.h1", s.hidden)
+        take(f"l{l}.qkv", qkv_w)
+        take(f"l{l}.qkv_rope", qkv_w)
+        take(f"l{l}.attn", s.q_dim)
+        take(f"l{l}.x_attn", s.hidden)
+        take(f"l{l}.act", s.ffn)
+        take(f"l{l}.x_mlp", s.hidden)
+    take("hf", s.hidden)
+    return out

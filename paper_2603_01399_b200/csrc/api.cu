@@ -1,0 +1,470 @@
+// C ABI of the library: argument checks, the model object, and the sequence of launches
+// that makes up one verification pass (Section 3.1 "Verification", Section 3.3).
+#include <stdarg.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <atomic>
+#include <new>
+#include <vector>
+
+#include "common.cuh"
+
+namespace quasar {
+
+static thread_local char g_err[512] = "";
+static std::atomic<long long> g_launches{0};
+
+void set_error(const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(g_err, sizeof(g_err), fmt, ap);
+  va_end(ap);
+}
+
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+}  // namespace quasar
+
+using namespace quasar;
+
+struct quasar_model {
+  quasar_config cfg;
+  std::vector<quasar_layer_weights> layers;
+  quasar_weights w;
+  float2* rope_table = nullptr;
+  void* trace_buf = nullptr;
+  size_t trace_bytes = 0;
+};
+
+struct quasar_plan {
+  cudaGraph_t graph = nullptr;
+  cudaGraphExec_t exec = nullptr;
+  const int32_t *tokens, *parents, *block_len;
+  int32_t *accept_len, *bonus, *accept_path, *status;
+  int B, T_max;
+  int kernels = 0;  // kernel nodes one replay runs
+};
+
+namespace {
+
+size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
+
+// Layout of the verify workspace; every offset is a multiple of 256 bytes.
+struct Workspace {
+  size_t x, h, qkv, attn, gu, act, logits, top1, anc, depth, valid, lin, att, total;
+  size_t lin_bytes, att_bytes;
+};
+
+Workspace layout(const quasar_config& c, int B, int T_max, int s_max) {
+  Workspace w;
+  const size_t M = (size_t)B * T_max;
+  const size_t qkv_w = (size_t)(c.n_q_heads + 2 * c.n_kv_heads) * c.head_dim;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes); return o; };
+  w.x = take(M * c.hidden * 2);
+  w.h = take(M * c.hidden * 2);
+  w.qkv = take(M * qkv_w * 2);
+  w.attn = take(M * (size_t)c.n_q_heads * c.head_dim * 2);
+  w.gu = take(M * 2 * (size_t)c.ffn * 2);
+  w.act = take(M * (size_t)c.ffn * 2);
+  w.logits = take(M * (size_t)c.vocab * 4);
+  w.top1 = take(M * 4);
+  w.anc = take(M * 8);
+  w.depth = take(M * 4);
+  w.valid = take((size_t)B * 4);
+  size_t lin = 0;
+  const int64_t shapes[5][2] = {{(int64_t)qkv_w, c.hidden},
+                                {c.hidden, (int64_t)c.n_q_heads * c.head_dim},
+                                {2 * (int64_t)c.ffn, c.hidden},
+                                {c.hidden, c.ffn},
+                                {c.vocab, c.hidden}};
+  for (auto& s : shapes) {
+    const size_t b = linear_workspace_bytes((int64_t)M, s[0], s[1]);
+    lin = b > lin ? b : lin;
+  }
+  w.lin_bytes = lin;
+  w.lin = take(lin);
+  w.att_bytes = attention_workspace_bytes(B, T_max, c.n_q_heads, c.n_kv_heads, c.head_dim, s_max);
+  w.att = take(w.att_bytes);
+  w.total = off;
+  return w;
+}
+
+int check_cfg(const quasar_config& c) {
+  if (c.n_layers < 0 || c.hidden <= 0 || c.n_q_heads <= 0 || c.n_kv_heads <= 0 || c.ffn <= 0 || c.vocab <= 0 ||
+      c.max_seq <= 0) {
+    set_error("config: non-positive size");
+    return QUASAR_ERR_INVALID_ARG;
+  }
+  if (c.weight_dtype != QUASAR_W_INT8 && c.weight_dtype != QUASAR_W_BF16) {
+    set_error("config: weight_dtype %d", c.weight_dtype);
+    return QUASAR_ERR_INVALID_ARG;
+  }
+  if ((c.head_dim != 64 && c.head_dim != 128) || c.hidden % 16 || c.ffn % 16 || c.n_q_heads % c.n_kv_heads ||
+      c.n_q_heads / c.n_kv_heads > 8 || ((int64_t)c.n_q_heads * c.head_dim) % 16) {
+    set_error("config: unsupported shape (head_dim 64/128, hidden and ffn multiples of 16, group size <= 8)");
+    return QUASAR_ERR_SHAPE;
+  }
+  return QUASAR_OK;
+}
+
+#define REQUIRE_PTR(p, name)                                  \
+  do {                                                        \
+    if ((p) == nullptr) {                                     \
+      set_error("%s is NULL", name);                          \
+      return QUASAR_ERR_INVALID_ARG;                          \
+    }                                                         \
+    if (!aligned16(p)) {                                      \
+      set_error("%s is not 16-byte aligned", name);           \
+      return QUASAR_ERR_ALIGN;                                \
+    }                                                         \
+  } while (0)
+
+struct TraceCursor {
+  unsigned char* base;
+  size_t off, cap;
+  cudaStream_t stream;
+  int put(const void* src, size_t bytes) {
+    if (base == nullptr) return QUASAR_OK;
+    if (off + bytes > cap) {
+      set_error("trace buffer too small");
+      return QUASAR_ERR_CAPACITY;
+    }
+    QUASAR_CUDA_CHECK(cudaMemcpyAsync(base + off, src, bytes, cudaMemcpyDeviceToDevice, stream));
+    off += bytes;
+    return QUASAR_OK;
+  }
+};
+
+#define TRY(expr)                       \
+  do {                                  \
+    int rc__ = (expr);                  \
+    if (rc__ != QUASAR_OK) return rc__; \
+  } while (0)
+
+int verify_impl(quasar_model* m, const quasar_kv* kv, const int32_t* tokens, const int32_t* parents,
+                const int32_t* block_len, int32_t B, int32_t T_max, float* logits_out, int32_t* accept_len,
+                int32_t* bonus, int32_t* accept_path, void* workspace, size_t workspace_bytes, int32_t* status,
+                cudaStream_t stream) {
+  if (m == nullptr || kv == nullptr) {
+    set_error("model or kv is NULL");
+    return QUASAR_ERR_INVALID_ARG;
+  }
+  const quasar_config& c = m->cfg;
+  if (B < 1 || T_max < 1 || T_max > QUASAR_MAX_BLOCK) {
+    set_error("verify: B=%d T_max=%d (T_max must be 1..%d)", B, T_max, QUASAR_MAX_BLOCK);
+    return QUASAR_ERR_SHAPE;
+  }
+  if (B > kv->batch || kv->s_max > c.max_seq || kv->s_max < 1) {
+    set_error("verify: batch %d exceeds cache batch %d, or s_max %d outside 1..max_seq %d", B, kv->batch, kv->s_max,
+              c.max_seq);
+    return QUASAR_ERR_CAPACITY;
+  }
+  REQUIRE_PTR(kv->k, "kv.k");
+  REQUIRE_PTR(kv->v, "kv.v");
+  REQUIRE_PTR(kv->seq_len, "kv.seq_len");
+  REQUIRE_PTR(tokens, "tokens");
+  REQUIRE_PTR(block_len, "block_len");
+  REQUIRE_PTR(accept_len, "accept_len");
+  REQUIRE_PTR(bonus, "bonus");
+  REQUIRE_PTR(workspace, "workspace");
+  REQUIRE_PTR(status, "status");
+  if (parents && !aligned16(parents)) { set_error("parents is not 16-byte aligned"); return QUASAR_ERR_ALIGN; }
+  if (logits_out && !aligned16(logits_out)) { set_error("logits_out is not 16-byte aligned"); return QUASAR_ERR_ALIGN; }
+  if (accept_path && !aligned16(accept_path)) { set_error("accept_path is not 16-byte aligned"); return QUASAR_ERR_ALIGN; }
+  const Workspace ws = layout(c, B, T_max, kv->s_max);
+  if (workspace_bytes < ws.total) {
+    set_error("verify: workspace of %zu bytes, need %zu", workspace_bytes, ws.total);
+    return QUASAR_ERR_CAPACITY;
+  }
+
+  unsigned char* wsp = reinterpret_cast<unsigned char*>(workspace);
+  __nv_bfloat16* x = reinterpret_cast<__nv_bfloat16*>(wsp + ws.x);
+  __nv_bfloat16* h = reinterpret_cast<__nv_bfloat16*>(wsp + ws.h);
+  __nv_bfloat16* qkv = reinterpret_cast<__nv_bfloat16*>(wsp + ws.qkv);
+  __nv_bfloat16* attn = reinterpret_cast<__nv_bfloat16*>(wsp + ws.attn);
+  __nv_bfloat16* gu = reinterpret_cast<__nv_bfloat16*>(wsp + ws.gu);
+  __nv_bfloat16* act = reinterpret_cast<__nv_bfloat16*>(wsp + ws.act);
+  float* logits = logits_out ? logits_out : reinterpret_cast<float*>(wsp + ws.logits);
+  int32_t* top1 = reinterpret_cast<int32_t*>(wsp + ws.top1);
+  BlockInfo bi;
+  bi.anc = reinterpret_cast<uint64_t*>(wsp + ws.anc);
+  bi.depth = reinterpret_cast<int32_t*>(wsp + ws.depth);
+  bi.valid = reinterpret_cast<int32_t*>(wsp + ws.valid);
+  void* lin = wsp + ws.lin;
+  void* att = wsp + ws.att;
+
+  const int M = B * T_max;
+  const int H = c.hidden, D = c.head_dim, Hq = c.n_q_heads, Hkv = c.n_kv_heads, F = c.ffn;
+  const int qkv_w = (Hq + 2 * Hkv) * D;
+  const int wd = c.weight_dtype;
+  const size_t layer_stride = (size_t)kv->batch * Hkv * (size_t)kv->s_max * D;
+  TraceCursor tr{reinterpret_cast<unsigned char*>(m->trace_buf), 0, m->trace_bytes, stream};
+
+  // arrival counters of the split-K reduction start at zero and reset themselves
+  QUASAR_CUDA_CHECK(cudaMemsetAsync(lin, 0, ws.lin_bytes < 65536 ? ws.lin_bytes : 65536, stream));
+  TRY(launch_block_prep(tokens, parents, block_len, kv->seq_len, B, T_max, kv->s_max, c.vocab, bi, status, stream));
+  TRY(launch_embed(tokens, reinterpret_cast<const __nv_bfloat16*>(m->w.embed), M, H, c.vocab, x, stream));
+  TRY(tr.put(x, (size_t)M * H * 2));
+
+  for (int l = 0; l < c.n_layers; ++l) {
+    const quasar_layer_weights& L = m->layers[l];
+    __nv_bfloat16* kc = reinterpret_cast<__nv_bfloat16*>(kv->k) + (size_t)l * layer_stride;
+    __nv_bfloat16* vc = reinterpret_cast<__nv_bfloat16*>(kv->v) + (size_t)l * layer_stride;
+    TRY(launch_rmsnorm(x, reinterpret_cast<const __nv_bfloat16*>(L.attn_norm), M, H, c.rms_eps, h, stream));
+    TRY(tr.put(h, (size_t)M * H * 2));
+    TRY(launch_linear(h, L.qkv_w, L.qkv_delta, wd, M, qkv_w, H, qkv, false, nullptr, lin, ws.lin_bytes, stream));
+    TRY(tr.put(qkv, (size_t)M * qkv_w * 2));
+    TRY(launch_rope_append(qkv, reinterpret_cast<const __nv_bfloat16*>(c.qk_norm ? L.q_norm : nullptr),
+                           reinterpret_cast<const __nv_bfloat16*>(c.qk_norm ? L.k_norm : nullptr), m->rope_table,
+                           kv->seq_len, block_len, bi, B, T_max, Hq, Hkv, D, c.rms_eps, kc, vc, kv->s_max, stream));
+    TRY(tr.put(qkv, (size_t)M * qkv_w * 2));
+    TRY(launch_attention(qkv, kc, vc, kv->seq_len, block_len, bi, B, T_max, Hq, Hkv, D, kv->s_max, attn, att,
+                         ws.att_bytes, stream));
+    TRY(tr.put(attn, (size_t)M * Hq * D * 2));
+    TRY(launch_linear(attn, L.o_w, L.o_delta, wd, M, H, Hq * D, x, false, x, lin, ws.lin_bytes, stream));
+    TRY(tr.put(x, (size_t)M * H * 2));
+    TRY(launch_rmsnorm(x, reinterpret_cast<const __nv_bfloat16*>(L.mlp_norm), M, H, c.rms_eps, h, stream));
+    TRY(launch_linear(h, L.gateup_w, L.gateup_delta, wd, M, 2 * F, H, gu, false, nullptr, lin, ws.lin_bytes, stream));
+    TRY(launch_swiglu(gu, M, F, act, stream));
+    TRY(tr.put(act, (size_t)M * F * 2));
+    TRY(launch_linear(act, L.down_w, L.down_delta, wd, M, H, F, x, false, x, lin, ws.lin_bytes, stream));
+    TRY(tr.put(x, (size_t)M * H * 2));
+  }
+  TRY(launch_rmsnorm(x, reinterpret_cast<const __nv_bfloat16*>(m->w.final_norm), M, H, c.rms_eps, h, stream));
+  TRY(tr.put(h, (size_t)M * H * 2));
+  TRY(launch_linear(h, m->w.lm_w, m->w.lm_delta, wd, M, c.vocab, H, logits, true, nullptr, lin, ws.lin_bytes, stream));
+  TRY(launch_argmax(logits, M, c.vocab, top1, stream));
+  TRY(launch_accept(tokens, parents, block_len, top1, bi, B, T_max, accept_len, bonus, accept_path, stream));
+  return QUASAR_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* quasar_last_error(void) { return g_err; }
+
+int64_t quasar_kernel_launches(void) { return (int64_t)g_launches.load(); }
+
+int quasar_quantize(const void* w_bf16, int64_t N, int64_t K, int8_t* q_out, float* delta_out, void* stream) {
+  if (N < 0 || K < 0) { set_error("quantize: negative size"); return QUASAR_ERR_INVALID_ARG; }
+  if (N == 0 || K == 0) return QUASAR_OK;
+  if (K % 8 != 0 || N > 0x7fffffffLL) { set_error("quantize: K=%lld must be a multiple of 8", (long long)K); return QUASAR_ERR_SHAPE; }
+  REQUIRE_PTR(w_bf16, "w_bf16");
+  REQUIRE_PTR(q_out, "q_out");
+  REQUIRE_PTR(delta_out, "delta_out");
+  return launch_quantize(reinterpret_cast<const __nv_bfloat16*>(w_bf16), N, K, q_out, delta_out, (cudaStream_t)stream);
+}
+
+int quasar_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, size_t* bytes_out) {
+  if (bytes_out == nullptr || M <= 0 || N <= 0 || K <= 0) { set_error("linear_workspace_bytes: bad argument"); return QUASAR_ERR_INVALID_ARG; }
+  *bytes_out = linear_workspace_bytes(M, N, K);
+  return QUASAR_OK;
+}
+
+int quasar_linear(const void* x, const void* w, const float* delta, int32_t weight_dtype, int64_t M, int64_t N,
+                  int64_t K, void* y, int32_t y_is_f32, const void* residual, void* workspace, size_t workspace_bytes,
+                  void* stream) {
+  if (weight_dtype != QUASAR_W_INT8 && weight_dtype != QUASAR_W_BF16) { set_error("linear: weight_dtype %d", weight_dtype); return QUASAR_ERR_INVALID_ARG; }
+  REQUIRE_PTR(x, "x");
+  REQUIRE_PTR(w, "w");
+  REQUIRE_PTR(y, "y");
+  REQUIRE_PTR(workspace, "workspace");
+  if (weight_dtype == QUASAR_W_INT8) REQUIRE_PTR(delta, "delta");
+  if (residual && !aligned16(residual)) { set_error("residual is not 16-byte aligned"); return QUASAR_ERR_ALIGN; }
+  return launch_linear(reinterpret_cast<const __nv_bfloat16*>(x), w, delta, weight_dtype, M, N, K, y, y_is_f32 != 0,
+                       reinterpret_cast<const __nv_bfloat16*>(residual), workspace, workspace_bytes,
+                       (cudaStream_t)stream);
+}
+
+int quasar_model_create(const quasar_config* cfg, const quasar_weights* w, quasar_model** out) {
+  if (cfg == nullptr || w == nullptr || out == nullptr) { set_error("model_create: NULL argument"); return QUASAR_ERR_INVALID_ARG; }
+  *out = nullptr;
+  TRY(check_cfg(*cfg));
+  if (cfg->n_layers > 0 && w->layers == nullptr) { set_error("model_create: layers is NULL"); return QUASAR_ERR_INVALID_ARG; }
+  const bool q = cfg->weight_dtype == QUASAR_W_INT8;
+  REQUIRE_PTR(w->embed, "embed");
+  REQUIRE_PTR(w->final_norm, "final_norm");
+  REQUIRE_PTR(w->lm_w, "lm_w");
+  if (q) REQUIRE_PTR(w->lm_delta, "lm_delta");
+  for (int l = 0; l < cfg->n_layers; ++l) {
+    const quasar_layer_weights& L = w->layers[l];
+    REQUIRE_PTR(L.attn_norm, "attn_norm");
+    REQUIRE_PTR(L.qkv_w, "qkv_w");
+    REQUIRE_PTR(L.o_w, "o_w");
+    REQUIRE_PTR(L.mlp_norm, "mlp_norm");
+    REQUIRE_PTR(L.gateup_w, "gateup_w");
+    REQUIRE_PTR(L.down_w, "down_w");
+    if (q) {
+      REQUIRE_PTR(L.qkv_delta, "qkv_delta");
+      REQUIRE_PTR(L.o_delta, "o_delta");
+      REQUIRE_PTR(L.gateup_delta, "gateup_delta");
+      REQUIRE_PTR(L.down_delta, "down_delta");
+    }
+    if (cfg->qk_norm) {
+      REQUIRE_PTR(L.q_norm, "q_norm");
+      REQUIRE_PTR(L.k_norm, "k_norm");
+    }
+  }
+  quasar_model* m = new (std::nothrow) quasar_model();
+  if (m == nullptr) { set_error("model_create: out of host memory"); return QUASAR_ERR_INVALID_ARG; }
+  m->cfg = *cfg;
+  m->w = *w;
+  m->layers.assign(w->layers, w->layers + cfg->n_layers);
+  m->w.layers = m->layers.data();
+  const size_t tbytes = (size_t)cfg->max_seq * (cfg->head_dim / 2) * sizeof(float2);
+  cudaError_t e = cudaMalloc(&m->rope_table, tbytes);
+  if (e != cudaSuccess) {
+    set_error("model_create: cudaMalloc(%zu) failed: %s", tbytes, cudaGetErrorString(e));
+    delete m;
+    return QUASAR_ERR_CUDA;
+  }
+  int rc = launch_rope_table(m->rope_table, cfg->max_seq, cfg->head_dim, cfg->rope_theta, 0);
+  if (rc == QUASAR_OK && cudaStreamSynchronize(0) != cudaSuccess) { set_error("model_create: rope table kernel failed"); rc = QUASAR_ERR_CUDA; }
+  if (rc != QUASAR_OK) {
+    cudaFree(m->rope_table);
+    delete m;
+    return rc;
+  }
+  *out = m;
+  return QUASAR_OK;
+}
+
+int quasar_model_destroy(quasar_model* m) {
+  if (m == nullptr) return QUASAR_OK;
+  if (m->rope_table) cudaFree(m->rope_table);
+  delete m;
+  return QUASAR_OK;
+}
+
+int quasar_workspace_bytes(const quasar_model* m, int32_t B, int32_t T_max, size_t* bytes_out) {
+  if (m == nullptr || bytes_out == nullptr || B < 1 || T_max < 1 || T_max > QUASAR_MAX_BLOCK) { set_error("workspace_bytes: bad argument"); return QUASAR_ERR_INVALID_ARG; }
+  *bytes_out = layout(m->cfg, B, T_max, m->cfg.max_seq).total;
+  return QUASAR_OK;
+}
+
+int quasar_trace_bytes(const quasar_model* m, int32_t B, int32_t T_max, size_t* bytes_out) {
+  if (m == nullptr || bytes_out == nullptr || B < 1 || T_max < 1) { set_error("trace_bytes: bad argument"); return QUASAR_ERR_INVALID_ARG; }
+  const quasar_config& c = m->cfg;
+  const size_t M = (size_t)B * T_max;
+  const size_t qkv_w = (size_t)(c.n_q_heads + 2 * c.n_kv_heads) * c.head_dim;
+  const size_t per_layer = M * 2 * ((size_t)c.hidden * 3 + qkv_w * 2 + (size_t)c.n_q_heads * c.head_dim + c.ffn);
+  *bytes_out = M * c.hidden * 2 * 2 + per_layer * c.n_layers;
+  return QUASAR_OK;
+}
+
+int quasar_set_trace(quasar_model* m, void* trace_buf, size_t bytes) {
+  if (m == nullptr) { set_error("set_trace: model is NULL"); return QUASAR_ERR_INVALID_ARG; }
+  m->trace_buf = trace_buf;
+  m->trace_bytes = trace_buf ? bytes : 0;
+  return QUASAR_OK;
+}
+
+int quasar_verify(quasar_model* m, const quasar_kv* kv, const int32_t* tokens, const int32_t* parents,
+                  const int32_t* block_len, int32_t B, int32_t T_max, float* logits_out, int32_t* accept_len,
+                  int32_t* bonus, int32_t* accept_path, void* workspace, size_t workspace_bytes, int32_t* status,
+                  void* stream) {
+  return verify_impl(m, kv, tokens, parents, block_len, B, T_max, logits_out, accept_len, bonus, accept_path, workspace,
+                     workspace_bytes, status, (cudaStream_t)stream);
+}
+
+int quasar_kv_commit(quasar_model* m, const quasar_kv* kv, const int32_t* accept_len, const int32_t* accept_path,
+                     int32_t B, int32_t T_max, void* stream) {
+  if (m == nullptr || kv == nullptr) { set_error("kv_commit: NULL argument"); return QUASAR_ERR_INVALID_ARG; }
+  if (B < 1 || B > kv->batch || T_max < 1 || T_max > QUASAR_MAX_BLOCK) { set_error("kv_commit: B=%d T_max=%d", B, T_max); return QUASAR_ERR_SHAPE; }
+  REQUIRE_PTR(kv->k, "kv.k");
+  REQUIRE_PTR(kv->v, "kv.v");
+  REQUIRE_PTR(kv->seq_len, "kv.seq_len");
+  REQUIRE_PTR(accept_len, "accept_len");
+  const quasar_config& c = m->cfg;
+  return launch_kv_commit(reinterpret_cast<__nv_bfloat16*>(kv->k), reinterpret_cast<__nv_bfloat16*>(kv->v), kv->seq_len,
+                          accept_len, accept_path, c.n_layers, kv->batch, B, T_max, c.n_kv_heads, c.head_dim, kv->s_max,
+                          (cudaStream_t)stream);
+}
+
+int quasar_plan_create(quasar_model* m, const quasar_kv* kv, const int32_t* tokens, const int32_t* parents,
+                       const int32_t* block_len, int32_t B, int32_t T_max, float* logits_out, int32_t* accept_len,
+                       int32_t* bonus, int32_t* accept_path, void* workspace, size_t workspace_bytes, int32_t* status,
+                       quasar_plan** out) {
+  if (out == nullptr) { set_error("plan_create: out is NULL"); return QUASAR_ERR_INVALID_ARG; }
+  *out = nullptr;
+  if (m != nullptr && m->trace_buf != nullptr) { set_error("plan_create: switch the trace off first"); return QUASAR_ERR_INVALID_ARG; }
+  cudaStream_t s;
+  QUASAR_CUDA_CHECK(cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking));
+  quasar_plan* p = new (std::nothrow) quasar_plan();
+  if (p == nullptr) { cudaStreamDestroy(s); set_error("plan_create: out of host memory"); return QUASAR_ERR_INVALID_ARG; }
+  // one eager pass first: it configures kernel attributes (not allowed while capturing) and validates arguments
+  int rc = verify_impl(m, kv, tokens, parents, block_len, B, T_max, logits_out, accept_len, bonus, accept_path,
+                       workspace, workspace_bytes, status, s);
+  if (rc == QUASAR_OK && cudaStreamSynchronize(s) != cudaSuccess) { set_error("plan_create: eager pass failed: %s", cudaGetErrorString(cudaGetLastError())); rc = QUASAR_ERR_CUDA; }
+  if (rc == QUASAR_OK) {
+    const long long before = quasar_kernel_launches();
+    cudaError_t e = cudaStreamBeginCapture(s, cudaStreamCaptureModeThreadLocal);
+    if (e != cudaSuccess) { set_error("plan_create: begin capture: %s", cudaGetErrorString(e)); rc = QUASAR_ERR_CUDA; }
+    if (rc == QUASAR_OK) {
+      rc = verify_impl(m, kv, tokens, parents, block_len, B, T_max, logits_out, accept_len, bonus, accept_path,
+                       workspace, workspace_bytes, status, s);
+      e = cudaStreamEndCapture(s, &p->graph);
+      if (rc == QUASAR_OK && e != cudaSuccess) { set_error("plan_create: end capture: %s", cudaGetErrorString(e)); rc = QUASAR_ERR_CUDA; }
+    }
+    p->kernels = (int)(quasar_kernel_launches() - before);
+    count_launch(-p->kernels);  // captured launches did not run
+    if (rc == QUASAR_OK) {
+      e = cudaGraphInstantiate(&p->exec, p->graph, 0);
+      if (e != cudaSuccess) { set_error("plan_create: instantiate: %s", cudaGetErrorString(e)); rc = QUASAR_ERR_CUDA; }
+    }
+  }
+  cudaStreamDestroy(s);
+  if (rc != QUASAR_OK) {
+    if (p->exec) cudaGraphExecDestroy(p->exec);
+    if (p->graph) cudaGraphDestroy(p->graph);
+    delete p;
+    return rc;
+  }
+  p->tokens = tokens; p->parents = parents; p->block_len = block_len;
+  p->accept_len = accept_len; p->bonus = bonus; p->accept_path = accept_path; p->status = status;
+  p->B = B; p->T_max = T_max;
+  *out = p;
+  return QUASAR_OK;
+}
+
+int quasar_plan_launch(quasar_plan* p, void* stream) {
+  if (p == nullptr) { set_error("plan_launch: plan is NULL"); return QUASAR_ERR_INVALID_ARG; }
+  QUASAR_CUDA_CHECK(cudaGraphLaunch(p->exec, (cudaStream_t)stream));
+  count_launch(p->kernels);
+  return QUASAR_OK;
+}
+
+int quasar_plan_destroy(quasar_plan* p) {
+  if (p == nullptr) return QUASAR_OK;
+  if (p->exec) cudaGraphExecDestroy(p->exec);
+  if (p->graph) cudaGraphDestroy(p->graph);
+  delete p;
+  return QUASAR_OK;
+}
+
+int quasar_plan_run_host(quasar_plan* p, const int32_t* tokens_host, const int32_t* parents_host,
+                         const int32_t* block_len_host, int32_t* accept_len_host, int32_t* bonus_host,
+                         int32_t* accept_path_host, int32_t* status_host, void* stream) {
+  if (p == nullptr || tokens_host == nullptr) { set_error("plan_run_host: NULL argument"); return QUASAR_ERR_INVALID_ARG; }
+  cudaStream_t s = (cudaStream_t)stream;
+  const size_t bt = (size_t)p->B * p->T_max * sizeof(int32_t), bb = (size_t)p->B * sizeof(int32_t);
+  QUASAR_CUDA_CHECK(cudaMemcpyAsync(const_cast<int32_t*>(p->tokens), tokens_host, bt, cudaMemcpyHostToDevice, s));
+  if (parents_host && p->parents)
+    QUASAR_CUDA_CHECK(cudaMemcpyAsync(const_cast<int32_t*>(p->parents), parents_host, bt, cudaMemcpyHostToDevice, s));
+  if (block_len_host)
+    QUASAR_CUDA_CHECK(cudaMemcpyAsync(const_cast<int32_t*>(p->block_len), block_len_host, bb, cudaMemcpyHostToDevice, s));
+  QUASAR_CUDA_CHECK(cudaGraphLaunch(p->exec, s));
+  count_launch(p->kernels);
+  if (accept_len_host) QUASAR_CUDA_CHECK(cudaMemcpyAsync(accept_len_host, p->accept_len, bb, cudaMemcpyDeviceToHost, s));
+  if (bonus_host) QUASAR_CUDA_CHECK(cudaMemcpyAsync(bonus_host, p->bonus, bb, cudaMemcpyDeviceToHost, s));
+  if (accept_path_host && p->accept_path)
+    QUASAR_CUDA_CHECK(cudaMemcpyAsync(accept_path_host, p->accept_path, bt, cudaMemcpyDeviceToHost, s));
+  if (status_host) QUASAR_CUDA_CHECK(cudaMemcpyAsync(status_host, p->status, sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+  QUASAR_CUDA_CHECK(cudaStreamSynchronize(s));
+  return QUASAR_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,352 @@
+// Grouped-query verify-attention (the attention of the verification pass, Section 3.1:
+// every block row attends to the cached context x_<t plus the block rows its mask allows —
+// earlier rows for a chain, ancestors for a tree).
+//
+// The second HBM stream of the pass: K and V of the prefix are read once per layer
+// (2 * 2 B * D per cached position per kv head).  One kv head serves R = G * T query rows
+// (G = Hq / Hkv query heads x T block rows; 24..85 here), i.e. 2R flop per K/V byte, which
+// is far above what FMA pipes sustain at HBM speed, so QK^T and PV run on the tensor
+// cores (mma.m16n8k16, bf16 in, fp32 accumulate) with the softmax in registers and
+// warp-shuffle row reductions.
+//
+// Parallelism: the key range of a sequence is cut into chunks of `chunk` positions; a CTA
+// handles one (sequence, kv head, chunk) with one warp per 16 query rows, all warps
+// sharing the K/V tiles staged in shared memory.  Each CTA leaves an un-normalised partial
+// (row max, row sum, O) and a second kernel merges the partials of a row in chunk order.
+// P is fed to the PV product as a bf16 high part plus a bf16 low part (two MMAs), which
+// keeps ~16 bits of the probabilities.
+#include <math.h>
+
+#include "common.cuh"
+
+namespace quasar {
+
+namespace {
+
+constexpr int kKeyTile = 64;   // keys staged in shared memory at a time
+constexpr int kMaxWarps = 8;
+constexpr float kLog2e = 1.4426950408889634f;
+
+struct AttnArgs {
+  const __nv_bfloat16* qkv;  // [B*T_max][(Hq+2Hkv)*D], q part already normalised + rotated
+  const __nv_bfloat16* kc;   // [B][Hkv][s_max][D]
+  const __nv_bfloat16* vc;
+  const int32_t* seq_len;
+  const int32_t* block_len;
+  BlockInfo bi;
+  float* o_part;             // [B][Hkv][nchunk][Rpad][D]
+  float* ml_part;            // [B][Hkv][nchunk][Rpad][2]
+  __nv_bfloat16* out;        // [B*T_max][Hq*D]
+  int B, T_max, Hq, Hkv, s_max, chunk, nchunk, Rpad, ngroups;
+};
+
+__device__ __forceinline__ void mma16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                         uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3,
+                                                  const void* smem_ptr) {
+  const uint32_t addr = (uint32_t)__cvta_generic_to_shared(smem_ptr);
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"(addr));
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 p = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&p);
+}
+
+// high and low bf16 parts of a pair of probabilities
+__device__ __forceinline__ void split_bf16(float a, float b, uint32_t& hi, uint32_t& lo) {
+  const __nv_bfloat16 ah = __float2bfloat16_rn(a), bh = __float2bfloat16_rn(b);
+  const float ar = a - __bfloat162float(ah), br = b - __bfloat162float(bh);
+  __nv_bfloat162 h;
+  h.x = ah;
+  h.y = bh;
+  hi = *reinterpret_cast<uint32_t*>(&h);
+  lo = pack_bf16(ar, br);
+}
+
+template <int D>
+__global__ void __launch_bounds__(kMaxWarps * 32) verify_attention_kernel(AttnArgs a) {
+  constexpr int kStride = D + 8;  // padded row of the staged K / V tiles (bf16 elements)
+  constexpr int kDSteps = D / 16;
+  __shared__ __align__(16) __nv_bfloat16 k_s[kKeyTile * kStride];
+  __shared__ __align__(16) __nv_bfloat16 v_s[kKeyTile * kStride];
+
+  const int c = blockIdx.x / a.ngroups, group = blockIdx.x % a.ngroups;
+  const int hk = blockIdx.y, b = blockIdx.z;
+  if (!a.bi.valid[b]) return;
+  const int T = a.block_len[b];
+  const int P = a.seq_len[b];
+  const int Lk = P + T;
+  const int key_begin = c * a.chunk;
+  const int key_end = min(Lk, key_begin + a.chunk);
+  if (key_begin >= key_end) return;
+
+  const int G = a.Hq / a.Hkv;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int nwarps = blockDim.x >> 5;
+  const int g = lane >> 2, t = lane & 3;
+  const int row_tile = group * nwarps + warp;
+  const int qkv_w = (a.Hq + 2 * a.Hkv) * D;
+
+  // the two query rows of this thread: r = node * G + head-in-group
+  int node[2];
+  uint64_t anc[2];
+  uint32_t qf[kDSteps][4];
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    const int r = row_tile * 16 + g + 8 * h;
+    node[h] = r / G;
+    const bool ok = node[h] < T;
+    anc[h] = ok ? a.bi.anc[b * a.T_max + node[h]] : 0ull;
+    const __nv_bfloat16* qrow =
+        a.qkv + (size_t)(b * a.T_max + (ok ? node[h] : 0)) * qkv_w + (size_t)(hk * G + (r % G)) * D;
+#pragma unroll
+    for (int kd = 0; kd < kDSteps; ++kd) {
+      qf[kd][h] = ok ? *reinterpret_cast<const uint32_t*>(qrow + kd * 16 + 2 * t) : 0u;
+      qf[kd][h + 2] = ok ? *reinterpret_cast<const uint32_t*>(qrow + kd * 16 + 8 + 2 * t) : 0u;
+    }
+  }
+
+  float o[D / 8][4];
+#pragma unroll
+  for (int i = 0; i < D / 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+  float row_max[2] = {-INFINITY, -INFINITY};
+  float row_sum[2] = {0.f, 0.f};
+  const float scale_log2 = kLog2e / sqrtf((float)D);
+
+  const __nv_bfloat16* kbase = a.kc + ((size_t)b * a.Hkv + hk) * (size_t)a.s_max * D;
+  const __nv_bfloat16* vbase = a.vc + ((size_t)b * a.Hkv + hk) * (size_t)a.s_max * D;
+
+  for (int k0 = key_begin; k0 < key_end; k0 += kKeyTile) {
+    __syncthreads();
+    for (int i = threadIdx.x; i < kKeyTile * (D / 8); i += blockDim.x) {
+      const int key = i / (D / 8), ch = i % (D / 8);
+      uint4 kv4 = make_uint4(0, 0, 0, 0), vv4 = make_uint4(0, 0, 0, 0);
+      if (k0 + key < key_end) {
+        kv4 = __ldg(reinterpret_cast<const uint4*>(kbase + (size_t)(k0 + key) * D) + ch);
+        vv4 = __ldg(reinterpret_cast<const uint4*>(vbase + (size_t)(k0 + key) * D) + ch);
+      }
+      *reinterpret_cast<uint4*>(k_s + key * kStride + ch * 8) = kv4;
+      *reinterpret_cast<uint4*>(v_s + key * kStride + ch * 8) = vv4;
+    }
+    __syncthreads();
+
+    // S = Q K^T for 16 rows x 64 keys
+    float s[kKeyTile / 8][4];
+#pragma unroll
+    for (int j = 0; j < kKeyTile / 8; ++j) {
+      s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f;
+#pragma unroll
+      for (int kd = 0; kd < kDSteps; ++kd) {
+        const __nv_bfloat16* kr = k_s + (8 * j + g) * kStride + kd * 16 + 2 * t;
+        const uint32_t b0 = *reinterpret_cast<const uint32_t*>(kr);
+        const uint32_t b1 = *reinterpret_cast<const uint32_t*>(kr + 8);
+        mma16816(s[j], qf[kd][0], qf[kd][1], qf[kd][2], qf[kd][3], b0, b1);
+      }
+    }
+
+    // mask, running max
+    float tile_max[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+    for (int j = 0; j < kKeyTile / 8; ++j) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int h = e >> 1;
+        const int key = k0 + 8 * j + 2 * t + (e & 1);
+        bool ok = key < key_end;
+        if (ok && key >= P) ok = (anc[h] >> (key - P)) & 1ull;
+        const float v = ok ? s[j][e] * scale_log2 : -INFINITY;
+        s[j][e] = v;
+        tile_max[h] = fmaxf(tile_max[h], v);
+      }
+    }
+    float alpha[2], m_use[2];
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      tile_max[h] = fmaxf(tile_max[h], __shfl_xor_sync(0xffffffffu, tile_max[h], 1));
+      tile_max[h] = fmaxf(tile_max[h], __shfl_xor_sync(0xffffffffu, tile_max[h], 2));
+      const float m_new = fmaxf(row_max[h], tile_max[h]);
+      m_use[h] = (m_new == -INFINITY) ? 0.f : m_new;
+      alpha[h] = exp2f(row_max[h] - m_use[h]);  // 0 when nothing has been seen yet
+      row_max[h] = m_new;
+      row_sum[h] *= alpha[h];
+    }
+#pragma unroll
+    for (int i = 0; i < D / 8; ++i) {
+      o[i][0] *= alpha[0];
+      o[i][1] *= alpha[0];
+      o[i][2] *= alpha[1];
+      o[i][3] *= alpha[1];
+    }
+#pragma unroll
+    for (int j = 0; j < kKeyTile / 8; ++j) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float p = exp2f(s[j][e] - m_use[e >> 1]);
+        s[j][e] = p;
+        row_sum[e >> 1] += p;
+      }
+    }
+
+    // O += P V, 16 keys per step
+#pragma unroll
+    for (int kk = 0; kk < kKeyTile / 16; ++kk) {
+      uint32_t ah[4], al[4];
+      split_bf16(s[2 * kk][0], s[2 * kk][1], ah[0], al[0]);
+      split_bf16(s[2 * kk][2], s[2 * kk][3], ah[1], al[1]);
+      split_bf16(s[2 * kk + 1][0], s[2 * kk + 1][1], ah[2], al[2]);
+      split_bf16(s[2 * kk + 1][2], s[2 * kk + 1][3], ah[3], al[3]);
+#pragma unroll
+      for (int dt = 0; dt < D / 16; ++dt) {
+        uint32_t b0, b1, b2, b3;
+        const int mat = lane >> 3, r = lane & 7;
+        ldmatrix_x4_trans(b0, b1, b2, b3, v_s + (kk * 16 + (mat & 1) * 8 + r) * kStride + dt * 16 + (mat >> 1) * 8);
+        mma16816(o[2 * dt], ah[0], ah[1], ah[2], ah[3], b0, b1);
+        mma16816(o[2 * dt], al[0], al[1], al[2], al[3], b0, b1);
+        mma16816(o[2 * dt + 1], ah[0], ah[1], ah[2], ah[3], b2, b3);
+        mma16816(o[2 * dt + 1], al[0], al[1], al[2], al[3], b2, b3);
+      }
+    }
+  }
+
+  // ---- partial results ----------------------------------------------------------------------
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    row_sum[h] += __shfl_xor_sync(0xffffffffu, row_sum[h], 1);
+    row_sum[h] += __shfl_xor_sync(0xffffffffu, row_sum[h], 2);
+  }
+  const size_t slot = (((size_t)b * a.Hkv + hk) * a.nchunk + c) * a.Rpad;
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    const int r = row_tile * 16 + g + 8 * h;
+    if (r >= a.Rpad) continue;
+    float* op = a.o_part + (slot + r) * D;
+#pragma unroll
+    for (int i = 0; i < D / 8; ++i) {
+      *reinterpret_cast<float2*>(op + 8 * i + 2 * t) = make_float2(o[i][2 * h], o[i][2 * h + 1]);
+    }
+    if (t == 0) {
+      a.ml_part[(slot + r) * 2] = row_max[h];
+      a.ml_part[(slot + r) * 2 + 1] = row_sum[h];
+    }
+  }
+}
+
+// One warp per (sequence, block row, query head): merge the chunk partials in chunk order.
+template <int D>
+__global__ void __launch_bounds__(128) attention_merge_kernel(AttnArgs a) {
+  const int item = blockIdx.x * 4 + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (item >= a.B * a.T_max * a.Hq) return;
+  const int hq = item % a.Hq;
+  const int m = item / a.Hq;
+  const int b = m / a.T_max, i = m % a.T_max;
+  __nv_bfloat16* dst = a.out + (size_t)m * a.Hq * D + (size_t)hq * D;
+  constexpr int kPer = D / 32;
+  if (!a.bi.valid[b] || i >= a.block_len[b]) {
+#pragma unroll
+    for (int e = 0; e < kPer; ++e) dst[lane * kPer + e] = __float2bfloat16_rn(0.f);
+    return;
+  }
+  const int G = a.Hq / a.Hkv;
+  const int hk = hq / G;
+  const int r = i * G + (hq % G);
+  const int Lk = a.seq_len[b] + a.block_len[b];
+  const int nch = (Lk + a.chunk - 1) / a.chunk;
+  const size_t slot0 = ((size_t)b * a.Hkv + hk) * a.nchunk * a.Rpad;
+  float mx = -INFINITY;
+  for (int c = 0; c < nch; ++c) mx = fmaxf(mx, a.ml_part[(slot0 + (size_t)c * a.Rpad + r) * 2]);
+  float acc[kPer];
+#pragma unroll
+  for (int e = 0; e < kPer; ++e) acc[e] = 0.f;
+  float den = 0.f;
+  for (int c = 0; c < nch; ++c) {
+    const size_t s = slot0 + (size_t)c * a.Rpad + r;
+    const float mc = a.ml_part[s * 2];
+    if (mc == -INFINITY) continue;
+    const float w = exp2f(mc - mx);
+    den += w * a.ml_part[s * 2 + 1];
+#pragma unroll
+    for (int e = 0; e < kPer; ++e) acc[e] += w * a.o_part[s * D + lane * kPer + e];
+  }
+  const float inv = 1.0f / den;
+#pragma unroll
+  for (int e = 0; e < kPer; ++e) dst[lane * kPer + e] = __float2bfloat16_rn(acc[e] * inv);
+}
+
+struct AttnPlan {
+  int chunk, nchunk, Rpad, ngroups, warps;
+};
+
+AttnPlan plan_attention(int B, int T_max, int Hq, int Hkv, int s_max) {
+  AttnPlan p;
+  const int units = B * Hkv;
+  int per_unit = (2 * 148 + units - 1) / units;
+  if (per_unit < 1) per_unit = 1;
+  int chunk = (s_max + per_unit - 1) / per_unit;
+  chunk = (chunk + kKeyTile - 1) / kKeyTile * kKeyTile;
+  if (chunk < kKeyTile) chunk = kKeyTile;
+  if (chunk > 256) chunk = 256;
+  p.chunk = chunk;
+  p.nchunk = (s_max + chunk - 1) / chunk;
+  const int R = (Hq / Hkv) * T_max;
+  const int tiles = (R + 15) / 16;
+  p.warps = tiles < kMaxWarps ? tiles : kMaxWarps;
+  p.ngroups = (tiles + p.warps - 1) / p.warps;
+  p.Rpad = p.ngroups * p.warps * 16;
+  return p;
+}
+
+}  // namespace
+
+size_t attention_workspace_bytes(int B, int T_max, int Hq, int Hkv, int D, int s_max) {
+  const AttnPlan p = plan_attention(B, T_max, Hq, Hkv, s_max);
+  const size_t rows = (size_t)B * Hkv * p.nchunk * p.Rpad;
+  return rows * D * sizeof(float) + rows * 2 * sizeof(float);
+}
+
+int launch_attention(const __nv_bfloat16* qkv, const __nv_bfloat16* k_cache_layer, const __nv_bfloat16* v_cache_layer,
+                     const int32_t* seq_len, const int32_t* block_len, BlockInfo bi, int B, int T_max, int Hq, int Hkv,
+                     int D, int s_max, __nv_bfloat16* out, void* workspace, size_t workspace_bytes,
+                     cudaStream_t stream) {
+  const AttnPlan p = plan_attention(B, T_max, Hq, Hkv, s_max);
+  if (workspace_bytes < attention_workspace_bytes(B, T_max, Hq, Hkv, D, s_max)) {
+    set_error("attention: workspace too small");
+    return QUASAR_ERR_CAPACITY;
+  }
+  AttnArgs a;
+  a.qkv = qkv; a.kc = k_cache_layer; a.vc = v_cache_layer; a.seq_len = seq_len; a.block_len = block_len; a.bi = bi;
+  const size_t rows = (size_t)B * Hkv * p.nchunk * p.Rpad;
+  a.o_part = reinterpret_cast<float*>(workspace);
+  a.ml_part = a.o_part + rows * D;
+  a.out = out;
+  a.B = B; a.T_max = T_max; a.Hq = Hq; a.Hkv = Hkv; a.s_max = s_max;
+  a.chunk = p.chunk; a.nchunk = p.nchunk; a.Rpad = p.Rpad; a.ngroups = p.ngroups;
+  dim3 grid(p.nchunk * p.ngroups, Hkv, B);
+  const int items = B * T_max * Hq;
+  if (D == 128) {
+    verify_attention_kernel<128><<<grid, p.warps * 32, 0, stream>>>(a);
+    QUASAR_LAUNCH_CHECK();
+    attention_merge_kernel<128><<<(items + 3) / 4, 128, 0, stream>>>(a);
+    QUASAR_LAUNCH_CHECK();
+  } else if (D == 64) {
+    verify_attention_kernel<64><<<grid, p.warps * 32, 0, stream>>>(a);
+    QUASAR_LAUNCH_CHECK();
+    attention_merge_kernel<64><<<(items + 3) / 4, 128, 0, stream>>>(a);
+    QUASAR_LAUNCH_CHECK();
+  } else {
+    set_error("head_dim %d not supported (64 or 128)", D);
+    return QUASAR_ERR_SHAPE;
+  }
+  return QUASAR_OK;
+}
+
+}  // namespace quasar

@@ -1,0 +1,89 @@
+// Shared declarations of the CUDA path (never included by the CPU oracle).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/quasar.h"
+
+namespace quasar {
+
+void set_error(const char* fmt, ...);
+void count_launch(int n = 1);
+
+#define QUASAR_CUDA_CHECK(expr)                                                        \
+  do {                                                                                 \
+    cudaError_t e__ = (expr);                                                          \
+    if (e__ != cudaSuccess) {                                                          \
+      quasar::set_error("%s failed: %s (%s:%d)", #expr, cudaGetErrorString(e__), __FILE__, __LINE__); \
+      return QUASAR_ERR_CUDA;                                                          \
+    }                                                                                  \
+  } while (0)
+
+#define QUASAR_LAUNCH_CHECK()                                                          \
+  do {                                                                                 \
+    quasar::count_launch();                                                            \
+    cudaError_t e__ = cudaGetLastError();                                              \
+    if (e__ != cudaSuccess) {                                                          \
+      quasar::set_error("kernel launch failed: %s (%s:%d)", cudaGetErrorString(e__), __FILE__, __LINE__); \
+      return QUASAR_ERR_CUDA;                                                          \
+    }                                                                                  \
+  } while (0)
+
+static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+constexpr int kMaxRowsPerGemm = 72;  // rows one skinny-GEMM launch handles (9 MMA column tiles)
+
+// ---- launchers (each only enqueues work on `stream`) -------------------------------------------
+
+int launch_quantize(const __nv_bfloat16* w, int64_t N, int64_t K, int8_t* q, float* delta, cudaStream_t stream);
+
+size_t linear_workspace_bytes(int64_t M, int64_t N, int64_t K);
+int launch_linear(const __nv_bfloat16* x, const void* w, const float* delta, int weight_dtype, int64_t M, int64_t N,
+                  int64_t K, void* y, bool y_is_f32, const __nv_bfloat16* residual, void* workspace,
+                  size_t workspace_bytes, cudaStream_t stream);
+
+// Per-call description of the draft blocks, derived on the device from tokens / parents / block_len.
+struct BlockInfo {
+  uint64_t* anc;    // [B*T_max] bit j set: block row j is row i itself or an ancestor of it
+  int32_t* depth;   // [B*T_max]
+  int32_t* valid;   // [B] 1 if the sequence is processed (block fits, parents well formed)
+};
+
+int launch_block_prep(const int32_t* tokens, const int32_t* parents, const int32_t* block_len, const int32_t* seq_len,
+                      int B, int T_max, int s_max, int vocab, BlockInfo bi, int32_t* status, cudaStream_t stream);
+
+int launch_embed(const int32_t* tokens, const __nv_bfloat16* embed, int M, int H, int vocab, __nv_bfloat16* x,
+                 cudaStream_t stream);
+
+int launch_rmsnorm(const __nv_bfloat16* x, const __nv_bfloat16* g, int M, int H, float eps, __nv_bfloat16* y,
+                   cudaStream_t stream);
+
+// QK-RMSNorm + RoPE on the q and k heads of qkv (in place) and K/V append at slot seq_len[b] + row.
+int launch_rope_append(__nv_bfloat16* qkv, const __nv_bfloat16* q_norm, const __nv_bfloat16* k_norm,
+                       const float2* rope_table, const int32_t* seq_len, const int32_t* block_len, BlockInfo bi, int B,
+                       int T_max, int Hq, int Hkv, int D, float eps, __nv_bfloat16* k_cache_layer,
+                       __nv_bfloat16* v_cache_layer, int s_max, cudaStream_t stream);
+
+size_t attention_workspace_bytes(int B, int T_max, int Hq, int Hkv, int D, int s_max);
+int launch_attention(const __nv_bfloat16* qkv, const __nv_bfloat16* k_cache_layer, const __nv_bfloat16* v_cache_layer,
+                     const int32_t* seq_len, const int32_t* block_len, BlockInfo bi, int B, int T_max, int Hq, int Hkv,
+                     int D, int s_max, __nv_bfloat16* out, void* workspace, size_t workspace_bytes,
+                     cudaStream_t stream);
+
+int launch_swiglu(const __nv_bfloat16* gu, int M, int F, __nv_bfloat16* act, cudaStream_t stream);
+
+int launch_argmax(const float* logits, int M, int V, int32_t* top1, cudaStream_t stream);
+
+int launch_accept(const int32_t* tokens, const int32_t* parents, const int32_t* block_len, const int32_t* top1,
+                  BlockInfo bi, int B, int T_max, int32_t* accept_len, int32_t* bonus, int32_t* accept_path,
+                  cudaStream_t stream);
+
+int launch_kv_commit(__nv_bfloat16* k_cache, __nv_bfloat16* v_cache, int32_t* seq_len, const int32_t* accept_len,
+                     const int32_t* accept_path, int L, int B_cache, int B, int T_max, int Hkv, int D, int s_max,
+                     cudaStream_t stream);
+
+int launch_rope_table(float2* table, int max_pos, int D, float theta, cudaStream_t stream);
+
+}  // namespace quasar

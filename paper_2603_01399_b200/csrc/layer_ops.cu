@@ -1,0 +1,372 @@
+// The small steps around the GEMMs of the verification pass (Section 3.3: the "non-linear
+// layers" that stay in high precision): block bookkeeping, embedding gather, RMSNorm,
+// QK-RMSNorm + RoPE + KV append, SwiGLU, arg-max, greedy acceptance (Section 3.1 Eq. 2 at
+// temperature 0) and the cache commit.  All are HBM/L2-bound on a few KB..MB; fp32 math,
+// bf16 storage.
+#include <math.h>
+
+#include "common.cuh"
+
+namespace quasar {
+
+namespace {
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// ---- block bookkeeping -------------------------------------------------------------------
+// One thread per sequence: checks tokens / parents / capacity, derives ancestor bit masks and depths.
+__global__ void block_prep_kernel(const int32_t* __restrict__ tokens, const int32_t* __restrict__ parents,
+                                  const int32_t* __restrict__ block_len, const int32_t* __restrict__ seq_len, int B,
+                                  int T_max, int s_max, int vocab, BlockInfo bi, int32_t* status) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= B) return;
+  const int T = block_len[b];
+  const int P = seq_len[b];
+  int err = 0;
+  if (T < 1 || T > T_max || P < 0) err = QUASAR_ERR_INVALID_ARG;
+  else if (P + T > s_max) err = QUASAR_ERR_CAPACITY;
+  if (!err) {
+    for (int i = 0; i < T; ++i) {
+      const int tok = tokens[b * T_max + i];
+      if (tok < 0 || tok >= vocab) err = QUASAR_ERR_TOKEN;
+      int p = (parents == nullptr) ? i - 1 : parents[b * T_max + i];
+      if ((i == 0 && p != -1) || (i > 0 && (p < 0 || p >= i))) err = QUASAR_ERR_TREE;
+      if (err) break;
+      uint64_t m = 1ull << i;
+      int d = 0;
+      if (i > 0) {
+        m |= bi.anc[b * T_max + p];
+        d = bi.depth[b * T_max + p] + 1;
+      }
+      bi.anc[b * T_max + i] = m;
+      bi.depth[b * T_max + i] = d;
+    }
+  }
+  for (int i = (err ? 0 : T); i < T_max; ++i) {
+    bi.anc[b * T_max + i] = 0;
+    bi.depth[b * T_max + i] = 0;
+  }
+  bi.valid[b] = err ? 0 : 1;
+  if (err && status) atomicMin(status, err);
+}
+
+// ---- embedding gather ----------------------------------------------------------------------
+__global__ void embed_kernel(const int32_t* __restrict__ tokens, const __nv_bfloat16* __restrict__ embed, int H,
+                             int vocab, __nv_bfloat16* __restrict__ x) {
+  const int m = blockIdx.x;
+  int tok = tokens[m];
+  const bool ok = tok >= 0 && tok < vocab;
+  const uint4* src = reinterpret_cast<const uint4*>(embed + (size_t)(ok ? tok : 0) * H);
+  uint4* dst = reinterpret_cast<uint4*>(x + (size_t)m * H);
+  for (int i = threadIdx.x; i < H / 8; i += blockDim.x) dst[i] = ok ? __ldg(src + i) : make_uint4(0, 0, 0, 0);
+}
+
+// ---- RMSNorm: y = x * rsqrt(mean(x^2) + eps) * g ------------------------------------------
+__global__ void __launch_bounds__(256)
+rmsnorm_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ g, int H, float eps,
+               __nv_bfloat16* __restrict__ y) {
+  const int m = blockIdx.x;
+  const __nv_bfloat162* xr = reinterpret_cast<const __nv_bfloat162*>(x + (size_t)m * H);
+  const __nv_bfloat162* gr = reinterpret_cast<const __nv_bfloat162*>(g);
+  __nv_bfloat162* yr = reinterpret_cast<__nv_bfloat162*>(y + (size_t)m * H);
+  float ss = 0.f;
+  for (int i = threadIdx.x; i < H / 2; i += blockDim.x) {
+    const float2 f = __bfloat1622float2(xr[i]);
+    ss += f.x * f.x + f.y * f.y;
+  }
+  ss = warp_sum(ss);
+  __shared__ float s_part[8];
+  if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = ss;
+  __syncthreads();
+  float tot = 0.f;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) tot += s_part[i];
+  const float r = 1.0f / sqrtf(tot / (float)H + eps);
+  for (int i = threadIdx.x; i < H / 2; i += blockDim.x) {
+    const float2 f = __bfloat1622float2(xr[i]);
+    const float2 gg = __bfloat1622float2(gr[i]);
+    yr[i] = __floats2bfloat162_rn(f.x * r * gg.x, f.y * r * gg.y);
+  }
+}
+
+// ---- RoPE table: cos/sin(pos * theta^(-2i/D)) evaluated in fp64, stored as fp32 -------------
+__global__ void rope_table_kernel(float2* table, int max_pos, int D, double theta) {
+  const int half = D / 2;
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= max_pos * half) return;
+  const int pos = idx / half, i = idx % half;
+  const double inv_freq = pow(theta, -2.0 * (double)i / (double)D);
+  double s, c;
+  sincos((double)pos * inv_freq, &s, &c);
+  table[idx] = make_float2((float)c, (float)s);
+}
+
+// ---- QK-RMSNorm + RoPE + KV append: one warp per (row, head) --------------------------------
+template <int D>
+__global__ void __launch_bounds__(128)
+rope_append_kernel(__nv_bfloat16* __restrict__ qkv, const __nv_bfloat16* __restrict__ q_norm,
+                   const __nv_bfloat16* __restrict__ k_norm, const float2* __restrict__ rope_table,
+                   const int32_t* __restrict__ seq_len, const int32_t* __restrict__ block_len, BlockInfo bi, int T_max,
+                   int Hq, int Hkv, float eps, __nv_bfloat16* __restrict__ k_cache, __nv_bfloat16* __restrict__ v_cache,
+                   int s_max, int n_items) {
+  constexpr int kPairs = D / 64;  // rotation pairs (i, i + D/2) per lane
+  const int item = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (item >= n_items) return;
+  const int lane = threadIdx.x & 31;
+  const int heads = Hq + 2 * Hkv;
+  const int m = item / heads, head = item % heads;
+  const int b = m / T_max, i = m % T_max;
+  if (!bi.valid[b] || i >= block_len[b]) return;
+  const int P = seq_len[b];
+  __nv_bfloat16* src = qkv + (size_t)m * heads * D + (size_t)head * D;
+
+  if (head >= Hq + Hkv) {  // v head: copy into the cache
+    const int hk = head - Hq - Hkv;
+    __nv_bfloat16* dst = v_cache + (((size_t)b * Hkv + hk) * s_max + (P + i)) * D;
+    if (lane < D / 8) reinterpret_cast<uint4*>(dst)[lane] = reinterpret_cast<const uint4*>(src)[lane];
+    return;
+  }
+  const bool is_q = head < Hq;
+  const __nv_bfloat16* gain = is_q ? q_norm : k_norm;
+  float lo[kPairs], hi[kPairs];
+  float ss = 0.f;
+#pragma unroll
+  for (int p = 0; p < kPairs; ++p) {
+    const int d = lane + 32 * p;
+    lo[p] = __bfloat162float(src[d]);
+    hi[p] = __bfloat162float(src[d + D / 2]);
+    ss += lo[p] * lo[p] + hi[p] * hi[p];
+  }
+  if (gain != nullptr) {
+    ss = warp_sum(ss);
+    const float r = 1.0f / sqrtf(ss / (float)D + eps);
+#pragma unroll
+    for (int p = 0; p < kPairs; ++p) {
+      const int d = lane + 32 * p;
+      lo[p] = lo[p] * r * __bfloat162float(gain[d]);
+      hi[p] = hi[p] * r * __bfloat162float(gain[d + D / 2]);
+    }
+  }
+  const int pos = P + bi.depth[m];
+  __nv_bfloat16* dst = is_q ? src : k_cache + (((size_t)b * Hkv + (head - Hq)) * s_max + (P + i)) * D;
+#pragma unroll
+  for (int p = 0; p < kPairs; ++p) {
+    const int d = lane + 32 * p;
+    const float2 cs = rope_table[(size_t)pos * (D / 2) + d];
+    dst[d] = __float2bfloat16_rn(lo[p] * cs.x - hi[p] * cs.y);
+    dst[d + D / 2] = __float2bfloat16_rn(hi[p] * cs.x + lo[p] * cs.y);
+  }
+}
+
+// ---- SwiGLU: act = silu(gate) * up -----------------------------------------------------------
+__global__ void swiglu_kernel(const __nv_bfloat16* __restrict__ gu, int F, __nv_bfloat16* __restrict__ act) {
+  const int m = blockIdx.y;
+  const int f2 = blockIdx.x * blockDim.x + threadIdx.x;  // pair index
+  if (f2 >= F / 2) return;
+  const float2 gt = __bfloat1622float2(reinterpret_cast<const __nv_bfloat162*>(gu + (size_t)m * 2 * F)[f2]);
+  const float2 up = __bfloat1622float2(reinterpret_cast<const __nv_bfloat162*>(gu + (size_t)m * 2 * F + F)[f2]);
+  const float a0 = gt.x / (1.0f + expf(-gt.x)) * up.x;
+  const float a1 = gt.y / (1.0f + expf(-gt.y)) * up.y;
+  reinterpret_cast<__nv_bfloat162*>(act + (size_t)m * F)[f2] = __floats2bfloat162_rn(a0, a1);
+}
+
+// ---- arg-max over the vocabulary, lowest index on ties ---------------------------------------
+__global__ void __launch_bounds__(1024) argmax_kernel(const float* __restrict__ logits, int V, int32_t* top1) {
+  const int m = blockIdx.x;
+  const float* row = logits + (size_t)m * V;
+  float best = -INFINITY;
+  int bi = 0x7fffffff;
+  for (int v = threadIdx.x; v < V; v += blockDim.x) {
+    const float x = row[v];
+    if (x > best || (x == best && v < bi)) { best = x; bi = v; }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float ob = __shfl_xor_sync(0xffffffffu, best, o);
+    const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+    if (ob > best || (ob == best && oi < bi)) { best = ob; bi = oi; }
+  }
+  __shared__ float s_b[32];
+  __shared__ int s_i[32];
+  if ((threadIdx.x & 31) == 0) { s_b[threadIdx.x >> 5] = best; s_i[threadIdx.x >> 5] = bi; }
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    const int nw = blockDim.x >> 5;
+    best = threadIdx.x < nw ? s_b[threadIdx.x] : -INFINITY;
+    bi = threadIdx.x < nw ? s_i[threadIdx.x] : 0x7fffffff;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float ob = __shfl_xor_sync(0xffffffffu, best, o);
+      const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+      if (ob > best || (ob == best && oi < bi)) { best = ob; bi = oi; }
+    }
+    if (threadIdx.x == 0) top1[m] = bi == 0x7fffffff ? 0 : bi;
+  }
+}
+
+// ---- greedy acceptance: one thread per sequence ----------------------------------------------
+__global__ void accept_kernel(const int32_t* __restrict__ tokens, const int32_t* __restrict__ parents,
+                              const int32_t* __restrict__ block_len, const int32_t* __restrict__ top1, BlockInfo bi,
+                              int B, int T_max, int32_t* accept_len, int32_t* bonus, int32_t* accept_path) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= B) return;
+  const int base = b * T_max;
+  if (!bi.valid[b]) {
+    accept_len[b] = 0;
+    bonus[b] = -1;
+    if (accept_path) for (int d = 0; d < T_max; ++d) accept_path[base + d] = -1;
+    return;
+  }
+  const int T = block_len[b];
+  int cur = 0, n = 0;
+  if (accept_path) accept_path[base] = 0;
+  while (true) {
+    int nxt = -1;
+    const int want = top1[base + cur];
+    for (int c = cur + 1; c < T; ++c) {
+      const int p = parents ? parents[base + c] : c - 1;
+      if (p == cur && tokens[base + c] == want) { nxt = c; break; }
+    }
+    if (nxt < 0) break;
+    cur = nxt;
+    ++n;
+    if (accept_path) accept_path[base + n] = cur;
+  }
+  accept_len[b] = n;
+  bonus[b] = top1[base + cur];
+  if (accept_path) for (int d = n + 1; d < T_max; ++d) accept_path[base + d] = -1;
+}
+
+// ---- commit: (tree) move accepted rows into place, then bump seq_len --------------------------
+// One thread per 16-byte piece of a (layer, sequence, kv head) row; depths are walked in
+// increasing order inside the thread, which keeps every source slot intact until it is read
+// (the accepted row at depth d has block index >= d).
+__global__ void kv_gather_kernel(__nv_bfloat16* __restrict__ k_cache, __nv_bfloat16* __restrict__ v_cache,
+                                 const int32_t* __restrict__ seq_len, const int32_t* __restrict__ accept_len,
+                                 const int32_t* __restrict__ accept_path, int L, int B_cache, int B, int T_max,
+                                 int Hkv, int D, int s_max) {
+  const int chunks = D / 8;
+  const size_t total = (size_t)L * B * Hkv * chunks;
+  const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= total) return;
+  const int c = (int)(idx % chunks);
+  size_t r = idx / chunks;
+  const int hk = (int)(r % Hkv); r /= Hkv;
+  const int b = (int)(r % B);
+  const int l = (int)(r / B);
+  const int n = accept_len[b];
+  const int P = seq_len[b];
+  if (n < 0 || n >= T_max || P < 0) return;
+  const size_t base = (((size_t)l * B_cache + b) * Hkv + hk) * (size_t)s_max;
+  for (int d = 1; d <= n; ++d) {
+    const int j = accept_path[b * T_max + d];
+    if (j == d || j < d || j >= T_max || P + j >= s_max) continue;
+    uint4* kd = reinterpret_cast<uint4*>(k_cache + (base + P + d) * D) + c;
+    uint4* vd = reinterpret_cast<uint4*>(v_cache + (base + P + d) * D) + c;
+    *kd = *(reinterpret_cast<const uint4*>(k_cache + (base + P + j) * D) + c);
+    *vd = *(reinterpret_cast<const uint4*>(v_cache + (base + P + j) * D) + c);
+  }
+}
+
+__global__ void seq_bump_kernel(int32_t* seq_len, const int32_t* __restrict__ accept_len, int B, int T_max, int s_max) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= B) return;
+  const int n = accept_len[b];
+  if (n < 0 || n >= T_max) return;
+  const int v = seq_len[b] + 1 + n;
+  if (v <= s_max) seq_len[b] = v;
+}
+
+}  // namespace
+
+int launch_block_prep(const int32_t* tokens, const int32_t* parents, const int32_t* block_len, const int32_t* seq_len,
+                      int B, int T_max, int s_max, int vocab, BlockInfo bi, int32_t* status, cudaStream_t stream) {
+  block_prep_kernel<<<(B + 63) / 64, 64, 0, stream>>>(tokens, parents, block_len, seq_len, B, T_max, s_max, vocab, bi,
+                                                     status);
+  QUASAR_LAUNCH_CHECK();
+  return QUASAR_OK;
+}
+
+int launch_embed(const int32_t* tokens, const __nv_bfloat16* embed, int M, int H, int vocab, __nv_bfloat16* x,
+                 cudaStream_t stream) {
+  embed_kernel<<<M, 128, 0, stream>>>(tokens, embed, H, vocab, x);
+  QUASAR_LAUNCH_CHECK();
+  return QUASAR_OK;
+}
+
+int launch_rmsnorm(const __nv_bfloat16* x, const __nv_bfloat16* g, int M, int H, float eps, __nv_bfloat16* y,
+                   cudaStream_t stream) {
+  rmsnorm_kernel<<<M, 256, 0, stream>>>(x, g, H, eps, y);
+  QUASAR_LAUNCH_CHECK();
+  return QUASAR_OK;
+}
+
+int launch_rope_table(float2* table, int max_pos, int D, float theta, cudaStream_t stream) {
+  const int total = max_pos * (D / 2);
+  rope_table_kernel<<<(total + 255) / 256, 256, 0, stream>>>(table, max_pos, D, (double)theta);
+  QUASAR_LAUNCH_CHECK();
+  return QUASAR_OK;
+}
+
+int launch_rope_append(__nv_bfloat16* qkv, const __nv_bfloat16* q_norm, const __nv_bfloat16* k_norm,
+                       const float2* rope_table, const int32_t* seq_len, const int32_t* block_len, BlockInfo bi, int B,
+                       int T_max, int Hq, int Hkv, int D, float eps, __nv_bfloat16* k_cache_layer,
+                       __nv_bfloat16* v_cache_layer, int s_max, cudaStream_t stream) {
+  const int n_items = B * T_max * (Hq + 2 * Hkv);
+  const int grid = (n_items + 3) / 4;
+  if (D == 128) {
+    rope_append_kernel<128><<<grid, 128, 0, stream>>>(qkv, q_norm, k_norm, rope_table, seq_len, block_len, bi, T_max,
+                                                       Hq, Hkv, eps, k_cache_layer, v_cache_layer, s_max, n_items);
+  } else if (D == 64) {
+    rope_append_kernel<64><<<grid, 128, 0, stream>>>(qkv, q_norm, k_norm, rope_table, seq_len, block_len, bi, T_max,
+                                                      Hq, Hkv, eps, k_cache_layer, v_cache_layer, s_max, n_items);
+  } else {
+    set_error("head_dim %d not supported (64 or 128)", D);
+    return QUASAR_ERR_SHAPE;
+  }
+  QUASAR_LAUNCH_CHECK();
+  return QUASAR_OK;
+}
+
+int launch_swiglu(const __nv_bfloat16* gu, int M, int F, __nv_bfloat16* act, cudaStream_t stream) {
+  dim3 grid((F / 2 + 255) / 256, M);
+  swiglu_kernel<<<grid, 256, 0, stream>>>(gu, F, act);
+  QUASAR_LAUNCH_CHECK();
+  return QUASAR_OK;
+}
+
+int launch_argmax(const float* logits, int M, int V, int32_t* top1, cudaStream_t stream) {
+  argmax_kernel<<<M, 1024, 0, stream>>>(logits, V, top1);
+  QUASAR_LAUNCH_CHECK();
+  return QUASAR_OK;
+}
+
+int launch_accept(const int32_t* tokens, const int32_t* parents, const int32_t* block_len, const int32_t* top1,
+                  BlockInfo bi, int B, int T_max, int32_t* accept_len, int32_t* bonus, int32_t* accept_path,
+                  cudaStream_t stream) {
+  accept_kernel<<<(B + 63) / 64, 64, 0, stream>>>(tokens, parents, block_len, top1, bi, B, T_max, accept_len, bonus,
+                                                 accept_path);
+  QUASAR_LAUNCH_CHECK();
+  return QUASAR_OK;
+}
+
+int launch_kv_commit(__nv_bfloat16* k_cache, __nv_bfloat16* v_cache, int32_t* seq_len, const int32_t* accept_len,
+                     const int32_t* accept_path, int L, int B_cache, int B, int T_max, int Hkv, int D, int s_max,
+                     cudaStream_t stream) {
+  if (accept_path != nullptr) {
+    const size_t total = (size_t)L * B * Hkv * (D / 8);
+    kv_gather_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(k_cache, v_cache, seq_len, accept_len,
+                                                                          accept_path, L, B_cache, B, T_max, Hkv, D,
+                                                                          s_max);
+    QUASAR_LAUNCH_CHECK();
+  }
+  seq_bump_kernel<<<(B + 63) / 64, 64, 0, stream>>>(seq_len, accept_len, B, T_max, s_max);
+  QUASAR_LAUNCH_CHECK();
+  return QUASAR_OK;
+}
+
+}  // namespace quasar

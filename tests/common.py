@@ -48,3 +48,24 @@ def prefill_oracle(model, kv, tokens_1d, chunk):
         oracle.verify(model, kv, t, None, np.array([len(c)], np.int32), want_logits=False)
         kv.seq_len[0] += len(c)
         i += len(c)
+
+
+# ---- CUDA-path side (imports nothing from oracle) ------------------------------------------
+def gpu_model(shape, seed=0, int8=True, max_seq=128, gen_device="cpu"):
+    from paper_2603_01399_b200 import binding
+    return binding.Model.from_master(shape, master_getter(shape, seed, gen_device), max_seq, int8=int8)
+
+
+def logits_close(gpu, ref, abs_tol=2e-2, rel_tol=1e-2):
+    """Element passes if |g - o| <= max(abs_tol, rel_tol * |o|).  Returns (ok, max_abs, max_rel)."""
+    gpu = np.asarray(gpu, np.float64)
+    ref = np.asarray(ref, np.float64)
+    diff = np.abs(gpu - ref)
+    ok = bool(np.all(diff <= np.maximum(abs_tol, rel_tol * np.abs(ref))))
+    return ok, float(diff.max()), float((diff / np.maximum(np.abs(ref), 1e-30)).max())
+
+
+def margins(logits):
+    """top1 - top2 per row of fp32 logits [..., V]."""
+    part = np.partition(logits, -2, axis=-1)
+    return part[..., -1] - part[..., -2]
