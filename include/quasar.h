@@ -193,8 +193,9 @@ int quasar_kv_commit(quasar_model* m, const quasar_kv* kv /* host struct */, con
                      const int32_t* accept_path, int32_t B, int32_t T_max, void* stream);
 
 /* ------------------------------------------------------------------------
- * A verify pass frozen into a CUDA graph: same arguments as quasar_verify,
- * captured once, replayed with one launch.  Every pointer is baked in; their
+ * A verify pass frozen for replay: same arguments as quasar_verify, captured
+ * once into a CUDA graph (or, when the pass is a single persistent kernel, kept
+ * as that one launch), replayed with one call.  Every pointer is baked in; their
  * CONTENTS may change between launches.  quasar_plan_create captures on an
  * internal stream and synchronises it (not capturable itself).
  * ---------------------------------------------------------------------- */
@@ -227,6 +228,12 @@ int quasar_plan_run_host(quasar_plan* p, const int32_t* tokens_host, const int32
  * ---------------------------------------------------------------------- */
 int quasar_trace_bytes(const quasar_model* m, int32_t B, int32_t T_max, size_t* bytes_out /* host */);
 int quasar_set_trace(quasar_model* m, void* trace_buf, size_t bytes);
+
+/* Which implementation quasar_verify uses: 0 = automatic (the persistent single-kernel pass
+ * when the block has at most 8 rows in total, else one kernel per step), 1 = always one kernel
+ * per step, 2 = require the persistent kernel (QUASAR_ERR_SHAPE if the call does not fit it).
+ * Both compute the same pass (Section 3.1, 3.3); they differ in summation order only. */
+int quasar_set_path(quasar_model* m, int32_t path);
 
 /* Count of kernels the library has launched in this process (all calls). */
 int64_t quasar_kernel_launches(void);

@@ -73,6 +73,7 @@ SIGNATURES = {
     "quasar_plan_run_host": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "quasar_trace_bytes": (C.c_int, [_vp, _i32, _i32, C.POINTER(_sz)]),
     "quasar_set_trace": (C.c_int, [_vp, _vp, _sz]),
+    "quasar_set_path": (C.c_int, [_vp, _i32]),
 }
 
 
@@ -212,6 +213,10 @@ class Model:
     def set_trace(self, buf: Optional[torch.Tensor]) -> None:
         self._trace = buf
         _check(lib().quasar_set_trace(self.handle, _ptr(buf), 0 if buf is None else buf.numel() * buf.element_size()))
+
+    def set_path(self, path: int) -> None:
+        """0 automatic, 1 one kernel per step, 2 persistent single-kernel pass."""
+        _check(lib().quasar_set_path(self.handle, path))
 
     def weight_bytes(self) -> int:
         return sum(v.numel() * v.element_size() for k, v in self.tensors.items()

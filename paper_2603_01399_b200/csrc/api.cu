@@ -9,6 +9,7 @@
 #include <vector>
 
 #include "common.cuh"
+#include "megakernel.cuh"
 
 namespace quasar {
 
@@ -35,11 +36,21 @@ struct quasar_model {
   float2* rope_table = nullptr;
   void* trace_buf = nullptr;
   size_t trace_bytes = 0;
+  // persistent single-kernel path
+  MegaJob* mega_jobs = nullptr;     // device
+  MegaLayer* mega_layers = nullptr; // device
+  int mega_ncta = 0;                // 0: not available on this device
+  int path = 0;                     // 0 auto, 1 one kernel per step, 2 persistent kernel
 };
 
 struct quasar_plan {
   cudaGraph_t graph = nullptr;
-  cudaGraphExec_t exec = nullptr;
+  cudaGraphExec_t exec = nullptr;   // null: the pass is a single persistent kernel, launched directly
+  quasar_model* model = nullptr;
+  quasar_kv kv;
+  float* logits_out = nullptr;
+  void* workspace = nullptr;
+  size_t workspace_bytes = 0;
   const int32_t *tokens, *parents, *block_len;
   int32_t *accept_len, *bonus, *accept_path, *status;
   int B, T_max;
@@ -52,9 +63,11 @@ size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
 
 // Layout of the verify workspace; every offset is a multiple of 256 bytes.
 struct Workspace {
-  size_t x, h, qkv, attn, gu, act, logits, top1, anc, depth, valid, lin, att, total;
+  size_t x, h, qkv, attn, gu, act, logits, top1, anc, depth, valid, lin, att, cand, barrier, total;
   size_t lin_bytes, att_bytes;
 };
+
+constexpr int kMaxGrid = 1024;  // upper bound on CTAs of the persistent kernel (SM count)
 
 Workspace layout(const quasar_config& c, int B, int T_max, int s_max) {
   Workspace w;
@@ -86,7 +99,14 @@ Workspace layout(const quasar_config& c, int B, int T_max, int s_max) {
   w.lin_bytes = lin;
   w.lin = take(lin);
   w.att_bytes = attention_workspace_bytes(B, T_max, c.n_q_heads, c.n_kv_heads, c.head_dim, s_max);
+  {
+    const size_t rows = (size_t)B * c.n_kv_heads * mega_attn_nchunk(s_max) * mega_attn_rpad(T_max, c.n_q_heads, c.n_kv_heads);
+    const size_t mega = rows * c.head_dim * sizeof(float) + rows * 2 * sizeof(float);
+    if (mega > w.att_bytes) w.att_bytes = mega;
+  }
   w.att = take(w.att_bytes);
+  w.cand = take((size_t)kMaxGrid * 8 * 2 * sizeof(float));
+  w.barrier = take(256);
   w.total = off;
   return w;
 }
@@ -142,6 +162,12 @@ struct TraceCursor {
     int rc__ = (expr);                  \
     if (rc__ != QUASAR_OK) return rc__; \
   } while (0)
+
+bool uses_persistent_kernel(const quasar_model* m, int B, int T_max) {
+  const quasar_config& c = m->cfg;
+  return m->path != 1 && m->mega_ncta > 0 && m->mega_ncta <= kMaxGrid && m->trace_buf == nullptr &&
+         mega_supported(B * T_max, T_max, c.n_q_heads, c.n_kv_heads, c.head_dim);
+}
 
 int verify_impl(quasar_model* m, const quasar_kv* kv, const int32_t* tokens, const int32_t* parents,
                 const int32_t* block_len, int32_t B, int32_t T_max, float* logits_out, int32_t* accept_len,
@@ -202,6 +228,35 @@ int verify_impl(quasar_model* m, const quasar_kv* kv, const int32_t* tokens, con
   const size_t layer_stride = (size_t)kv->batch * Hkv * (size_t)kv->s_max * D;
   TraceCursor tr{reinterpret_cast<unsigned char*>(m->trace_buf), 0, m->trace_bytes, stream};
 
+  const bool can_mega = m->mega_ncta > 0 && m->mega_ncta <= kMaxGrid && m->trace_buf == nullptr &&
+                        mega_supported(M, T_max, Hq, Hkv, D);
+  if (m->path == 2 && !can_mega) {
+    set_error("verify: the persistent kernel handles at most 8 block rows in total and no trace");
+    return QUASAR_ERR_SHAPE;
+  }
+  if (can_mega && m->path != 1) {
+    MegaParams p;
+    p.jobs = m->mega_jobs; p.layers = m->mega_layers; p.n_jobs = 4 * c.n_layers + 1; p.L = c.n_layers;
+    p.B = B; p.T_max = T_max; p.M = M; p.H = H; p.Hq = Hq; p.Hkv = Hkv; p.vocab = c.vocab; p.s_max = kv->s_max;
+    p.kv_batch = kv->batch; p.rms_eps = c.rms_eps;
+    p.embed = reinterpret_cast<const __nv_bfloat16*>(m->w.embed);
+    p.rope_table = m->rope_table;
+    p.tokens = tokens; p.parents = parents; p.block_len = block_len; p.seq_len = kv->seq_len;
+    p.k_cache = reinterpret_cast<__nv_bfloat16*>(kv->k); p.v_cache = reinterpret_cast<__nv_bfloat16*>(kv->v);
+    p.x = x; p.qkv = qkv; p.attn = attn; p.act = act; p.logits = logits_out; p.top1 = top1; p.bi = bi;
+    p.attn_nchunk = mega_attn_nchunk(kv->s_max);
+    p.attn_rpad = mega_attn_rpad(T_max, Hq, Hkv);
+    const size_t rows = (size_t)B * Hkv * p.attn_nchunk * p.attn_rpad;
+    p.o_part = reinterpret_cast<float*>(att);
+    p.ml_part = p.o_part + rows * D;
+    p.cand_val = reinterpret_cast<float*>(wsp + ws.cand);
+    p.cand_idx = reinterpret_cast<int*>(wsp + ws.cand + (size_t)kMaxGrid * 8 * sizeof(float));
+    p.barrier = reinterpret_cast<unsigned*>(wsp + ws.barrier);
+    p.accept_len = accept_len; p.bonus = bonus; p.accept_path = accept_path; p.status = status;
+    QUASAR_CUDA_CHECK(cudaMemsetAsync(p.barrier, 0, 256, stream));
+    return launch_verify_mega(p, wd, D, m->mega_ncta, stream);
+  }
+
   // arrival counters of the split-K reduction start at zero and reset themselves
   QUASAR_CUDA_CHECK(cudaMemsetAsync(lin, 0, ws.lin_bytes < 65536 ? ws.lin_bytes : 65536, stream));
   TRY(launch_block_prep(tokens, parents, block_len, kv->seq_len, B, T_max, kv->s_max, c.vocab, bi, status, stream));
@@ -237,6 +292,16 @@ int verify_impl(quasar_model* m, const quasar_kv* kv, const int32_t* tokens, con
   TRY(launch_linear(h, m->w.lm_w, m->w.lm_delta, wd, M, c.vocab, H, logits, true, nullptr, lin, ws.lin_bytes, stream));
   TRY(launch_argmax(logits, M, c.vocab, top1, stream));
   TRY(launch_accept(tokens, parents, block_len, top1, bi, B, T_max, accept_len, bonus, accept_path, stream));
+  return QUASAR_OK;
+}
+
+int plan_replay(quasar_plan* p, cudaStream_t stream) {
+  if (p->exec == nullptr) {  // the pass is one persistent kernel: nothing to replay, launch it
+    return verify_impl(p->model, &p->kv, p->tokens, p->parents, p->block_len, p->B, p->T_max, p->logits_out,
+                       p->accept_len, p->bonus, p->accept_path, p->workspace, p->workspace_bytes, p->status, stream);
+  }
+  QUASAR_CUDA_CHECK(cudaGraphLaunch(p->exec, stream));
+  count_launch(p->kernels);
   return QUASAR_OK;
 }
 
@@ -328,12 +393,51 @@ int quasar_model_create(const quasar_config* cfg, const quasar_weights* w, quasa
     delete m;
     return rc;
   }
+  // tables of the persistent kernel: the GEMMs of the pass in execution order
+  {
+    std::vector<MegaJob> jobs;
+    std::vector<MegaLayer> mls;
+    const int qkv_w = (cfg->n_q_heads + 2 * cfg->n_kv_heads) * cfg->head_dim;
+    for (int l = 0; l < cfg->n_layers; ++l) {
+      const quasar_layer_weights& L = m->layers[l];
+      jobs.push_back({L.qkv_w, q ? L.qkv_delta : nullptr, reinterpret_cast<const __nv_bfloat16*>(L.attn_norm), qkv_w,
+                      cfg->hidden, kJobQkv, 0});
+      jobs.push_back({L.o_w, q ? L.o_delta : nullptr, nullptr, cfg->hidden, cfg->n_q_heads * cfg->head_dim, kJobO, 0});
+      jobs.push_back({L.gateup_w, q ? L.gateup_delta : nullptr, reinterpret_cast<const __nv_bfloat16*>(L.mlp_norm),
+                      2 * cfg->ffn, cfg->hidden, kJobGateUp, 0});
+      jobs.push_back({L.down_w, q ? L.down_delta : nullptr, nullptr, cfg->hidden, cfg->ffn, kJobDown, 0});
+      mls.push_back({reinterpret_cast<const __nv_bfloat16*>(cfg->qk_norm ? L.q_norm : nullptr),
+                     reinterpret_cast<const __nv_bfloat16*>(cfg->qk_norm ? L.k_norm : nullptr)});
+    }
+    jobs.push_back({w->lm_w, q ? w->lm_delta : nullptr, reinterpret_cast<const __nv_bfloat16*>(w->final_norm),
+                    cfg->vocab, cfg->hidden, kJobLm, 0});
+    if (mls.empty()) mls.push_back({nullptr, nullptr});
+    cudaError_t e2 = cudaMalloc(&m->mega_jobs, jobs.size() * sizeof(MegaJob));
+    if (e2 == cudaSuccess) e2 = cudaMalloc(&m->mega_layers, mls.size() * sizeof(MegaLayer));
+    if (e2 == cudaSuccess) e2 = cudaMemcpy(m->mega_jobs, jobs.data(), jobs.size() * sizeof(MegaJob), cudaMemcpyHostToDevice);
+    if (e2 == cudaSuccess) e2 = cudaMemcpy(m->mega_layers, mls.data(), mls.size() * sizeof(MegaLayer), cudaMemcpyHostToDevice);
+    if (e2 != cudaSuccess) {
+      set_error("model_create: job tables: %s", cudaGetErrorString(e2));
+      quasar_model_destroy(m);
+      return QUASAR_ERR_CUDA;
+    }
+    int ncta = 0;
+    if (mega_grid_size(cfg->weight_dtype, cfg->head_dim, &ncta) == QUASAR_OK) m->mega_ncta = ncta;
+  }
   *out = m;
+  return QUASAR_OK;
+}
+
+int quasar_set_path(quasar_model* m, int32_t path) {
+  if (m == nullptr || path < 0 || path > 2) { set_error("set_path: bad argument"); return QUASAR_ERR_INVALID_ARG; }
+  m->path = path;
   return QUASAR_OK;
 }
 
 int quasar_model_destroy(quasar_model* m) {
   if (m == nullptr) return QUASAR_OK;
+  if (m->mega_jobs) cudaFree(m->mega_jobs);
+  if (m->mega_layers) cudaFree(m->mega_layers);
   if (m->rope_table) cudaFree(m->rope_table);
   delete m;
   return QUASAR_OK;
@@ -399,7 +503,7 @@ int quasar_plan_create(quasar_model* m, const quasar_kv* kv, const int32_t* toke
   int rc = verify_impl(m, kv, tokens, parents, block_len, B, T_max, logits_out, accept_len, bonus, accept_path,
                        workspace, workspace_bytes, status, s);
   if (rc == QUASAR_OK && cudaStreamSynchronize(s) != cudaSuccess) { set_error("plan_create: eager pass failed: %s", cudaGetErrorString(cudaGetLastError())); rc = QUASAR_ERR_CUDA; }
-  if (rc == QUASAR_OK) {
+  if (rc == QUASAR_OK && !uses_persistent_kernel(m, B, T_max)) {
     const long long before = quasar_kernel_launches();
     cudaError_t e = cudaStreamBeginCapture(s, cudaStreamCaptureModeThreadLocal);
     if (e != cudaSuccess) { set_error("plan_create: begin capture: %s", cudaGetErrorString(e)); rc = QUASAR_ERR_CUDA; }
@@ -426,15 +530,14 @@ int quasar_plan_create(quasar_model* m, const quasar_kv* kv, const int32_t* toke
   p->tokens = tokens; p->parents = parents; p->block_len = block_len;
   p->accept_len = accept_len; p->bonus = bonus; p->accept_path = accept_path; p->status = status;
   p->B = B; p->T_max = T_max;
+  p->model = m; p->kv = *kv; p->logits_out = logits_out; p->workspace = workspace; p->workspace_bytes = workspace_bytes;
   *out = p;
   return QUASAR_OK;
 }
 
 int quasar_plan_launch(quasar_plan* p, void* stream) {
   if (p == nullptr) { set_error("plan_launch: plan is NULL"); return QUASAR_ERR_INVALID_ARG; }
-  QUASAR_CUDA_CHECK(cudaGraphLaunch(p->exec, (cudaStream_t)stream));
-  count_launch(p->kernels);
-  return QUASAR_OK;
+  return plan_replay(p, (cudaStream_t)stream);
 }
 
 int quasar_plan_destroy(quasar_plan* p) {
@@ -456,8 +559,7 @@ int quasar_plan_run_host(quasar_plan* p, const int32_t* tokens_host, const int32
     QUASAR_CUDA_CHECK(cudaMemcpyAsync(const_cast<int32_t*>(p->parents), parents_host, bt, cudaMemcpyHostToDevice, s));
   if (block_len_host)
     QUASAR_CUDA_CHECK(cudaMemcpyAsync(const_cast<int32_t*>(p->block_len), block_len_host, bb, cudaMemcpyHostToDevice, s));
-  QUASAR_CUDA_CHECK(cudaGraphLaunch(p->exec, s));
-  count_launch(p->kernels);
+  TRY(plan_replay(p, s));
   if (accept_len_host) QUASAR_CUDA_CHECK(cudaMemcpyAsync(accept_len_host, p->accept_len, bb, cudaMemcpyDeviceToHost, s));
   if (bonus_host) QUASAR_CUDA_CHECK(cudaMemcpyAsync(bonus_host, p->bonus, bb, cudaMemcpyDeviceToHost, s));
   if (accept_path_host && p->accept_path)

@@ -1,0 +1,54 @@
+// Parameters of the persistent single-kernel verification pass.
+#pragma once
+
+#include "common.cuh"
+
+namespace quasar {
+
+constexpr int kMegaWarps = 16;
+
+enum MegaJobKind { kJobQkv = 0, kJobO = 1, kJobGateUp = 2, kJobDown = 3, kJobLm = 4 };
+
+// One GEMM of the pass, in execution order: per layer qkv, o, gate+up, down; then the LM head.
+struct MegaJob {
+  const void* w;               // [N][K] int8 or bf16
+  const float* delta;          // [N] or nullptr
+  const __nv_bfloat16* gain;   // RMSNorm gain fused into the operand load, or nullptr
+  int N, K, kind, pad;
+};
+
+struct MegaLayer {
+  const __nv_bfloat16* q_norm;  // [D] or nullptr
+  const __nv_bfloat16* k_norm;
+};
+
+struct MegaParams {
+  const MegaJob* jobs;      // device array, 4 L + 1 entries
+  const MegaLayer* layers;  // device array, L entries
+  int n_jobs, L;
+  int B, T_max, M, H, Hq, Hkv, vocab, s_max, kv_batch;
+  float rms_eps;
+  const __nv_bfloat16* embed;
+  const float2* rope_table;
+  const int32_t *tokens, *parents, *block_len, *seq_len;
+  __nv_bfloat16 *k_cache, *v_cache;
+  // workspace
+  __nv_bfloat16 *x, *qkv, *attn, *act;
+  float* logits;            // [M][V] or nullptr
+  int32_t* top1;
+  BlockInfo bi;
+  float *o_part, *ml_part;  // attention partials
+  int attn_nchunk, attn_rpad;
+  float* cand_val;          // [grid][8] per-CTA arg-max candidates
+  int* cand_idx;
+  unsigned* barrier;        // zeroed before every launch
+  int32_t *accept_len, *bonus, *accept_path, *status;
+};
+
+bool mega_supported(int M, int T_max, int Hq, int Hkv, int D);
+int mega_attn_nchunk(int s_max);
+int mega_attn_rpad(int T_max, int Hq, int Hkv);
+int mega_grid_size(int weight_dtype, int D, int* ncta_out);
+int launch_verify_mega(const MegaParams& p, int weight_dtype, int D, int ncta, cudaStream_t stream);
+
+}  // namespace quasar
