@@ -39,6 +39,7 @@ struct quasar_model {
   // persistent single-kernel path
   MegaJob* mega_jobs = nullptr;     // device
   MegaLayer* mega_layers = nullptr; // device
+  unsigned char* mega_weights = nullptr;  // device: every matrix again, permuted for the persistent kernel
   int mega_ncta = 0;                // 0: not available on this device
   int path = 0;                     // 0 auto, 1 one kernel per step, 2 persistent kernel
 };
@@ -393,36 +394,59 @@ int quasar_model_create(const quasar_config* cfg, const quasar_weights* w, quasa
     delete m;
     return rc;
   }
-  // tables of the persistent kernel: the GEMMs of the pass in execution order
-  {
+  // The persistent kernel: its grid, a permuted copy of every matrix in the order each CTA streams it,
+  // and the table of the GEMMs of the pass in execution order.
+  int ncta = 0;
+  if (mega_grid_size(cfg->weight_dtype, cfg->head_dim, &ncta) == QUASAR_OK && ncta > 0 && ncta <= kMaxGrid) {
     std::vector<MegaJob> jobs;
     std::vector<MegaLayer> mls;
+    std::vector<const void*> src;
     const int qkv_w = (cfg->n_q_heads + 2 * cfg->n_kv_heads) * cfg->head_dim;
     for (int l = 0; l < cfg->n_layers; ++l) {
       const quasar_layer_weights& L = m->layers[l];
-      jobs.push_back({L.qkv_w, q ? L.qkv_delta : nullptr, reinterpret_cast<const __nv_bfloat16*>(L.attn_norm), qkv_w,
+      jobs.push_back({nullptr, q ? L.qkv_delta : nullptr, reinterpret_cast<const __nv_bfloat16*>(L.attn_norm), qkv_w,
                       cfg->hidden, kJobQkv, 0});
-      jobs.push_back({L.o_w, q ? L.o_delta : nullptr, nullptr, cfg->hidden, cfg->n_q_heads * cfg->head_dim, kJobO, 0});
-      jobs.push_back({L.gateup_w, q ? L.gateup_delta : nullptr, reinterpret_cast<const __nv_bfloat16*>(L.mlp_norm),
+      src.push_back(L.qkv_w);
+      jobs.push_back({nullptr, q ? L.o_delta : nullptr, nullptr, cfg->hidden, cfg->n_q_heads * cfg->head_dim, kJobO, 0});
+      src.push_back(L.o_w);
+      jobs.push_back({nullptr, q ? L.gateup_delta : nullptr, reinterpret_cast<const __nv_bfloat16*>(L.mlp_norm),
                       2 * cfg->ffn, cfg->hidden, kJobGateUp, 0});
-      jobs.push_back({L.down_w, q ? L.down_delta : nullptr, nullptr, cfg->hidden, cfg->ffn, kJobDown, 0});
+      src.push_back(L.gateup_w);
+      jobs.push_back({nullptr, q ? L.down_delta : nullptr, nullptr, cfg->hidden, cfg->ffn, kJobDown, 0});
+      src.push_back(L.down_w);
       mls.push_back({reinterpret_cast<const __nv_bfloat16*>(cfg->qk_norm ? L.q_norm : nullptr),
                      reinterpret_cast<const __nv_bfloat16*>(cfg->qk_norm ? L.k_norm : nullptr)});
     }
-    jobs.push_back({w->lm_w, q ? w->lm_delta : nullptr, reinterpret_cast<const __nv_bfloat16*>(w->final_norm),
+    jobs.push_back({nullptr, q ? w->lm_delta : nullptr, reinterpret_cast<const __nv_bfloat16*>(w->final_norm),
                     cfg->vocab, cfg->hidden, kJobLm, 0});
+    src.push_back(w->lm_w);
     if (mls.empty()) mls.push_back({nullptr, nullptr});
-    cudaError_t e2 = cudaMalloc(&m->mega_jobs, jobs.size() * sizeof(MegaJob));
-    if (e2 == cudaSuccess) e2 = cudaMalloc(&m->mega_layers, mls.size() * sizeof(MegaLayer));
-    if (e2 == cudaSuccess) e2 = cudaMemcpy(m->mega_jobs, jobs.data(), jobs.size() * sizeof(MegaJob), cudaMemcpyHostToDevice);
-    if (e2 == cudaSuccess) e2 = cudaMemcpy(m->mega_layers, mls.data(), mls.size() * sizeof(MegaLayer), cudaMemcpyHostToDevice);
-    if (e2 != cudaSuccess) {
-      set_error("model_create: job tables: %s", cudaGetErrorString(e2));
-      quasar_model_destroy(m);
-      return QUASAR_ERR_CUDA;
+    const size_t esz = q ? 1 : 2;
+    size_t total = 0;
+    std::vector<size_t> offs;
+    for (auto& j : jobs) {
+      offs.push_back(total);
+      total += align_up((size_t)j.N * j.K * esz);
     }
-    int ncta = 0;
-    if (mega_grid_size(cfg->weight_dtype, cfg->head_dim, &ncta) == QUASAR_OK) m->mega_ncta = ncta;
+    cudaError_t e2 = cudaMalloc(&m->mega_weights, total);
+    if (e2 == cudaSuccess) e2 = cudaMalloc(&m->mega_jobs, jobs.size() * sizeof(MegaJob));
+    if (e2 == cudaSuccess) e2 = cudaMalloc(&m->mega_layers, mls.size() * sizeof(MegaLayer));
+    int rc2 = QUASAR_OK;
+    if (e2 == cudaSuccess) {
+      for (size_t i = 0; i < jobs.size() && rc2 == QUASAR_OK; ++i) {
+        jobs[i].wp = m->mega_weights + offs[i];
+        rc2 = launch_repack(src[i], m->mega_weights + offs[i], jobs[i].N, jobs[i].K, jobs[i].kind, cfg->weight_dtype, ncta, 0);
+      }
+      if (rc2 == QUASAR_OK) e2 = cudaMemcpy(m->mega_jobs, jobs.data(), jobs.size() * sizeof(MegaJob), cudaMemcpyHostToDevice);
+      if (rc2 == QUASAR_OK && e2 == cudaSuccess) e2 = cudaMemcpy(m->mega_layers, mls.data(), mls.size() * sizeof(MegaLayer), cudaMemcpyHostToDevice);
+      if (rc2 == QUASAR_OK && e2 == cudaSuccess) e2 = cudaStreamSynchronize(0);
+    }
+    if (e2 != cudaSuccess || rc2 != QUASAR_OK) {
+      if (e2 != cudaSuccess) set_error("model_create: tables of the persistent kernel (%zu bytes): %s", total, cudaGetErrorString(e2));
+      quasar_model_destroy(m);
+      return e2 != cudaSuccess ? QUASAR_ERR_CUDA : rc2;
+    }
+    m->mega_ncta = ncta;
   }
   *out = m;
   return QUASAR_OK;
@@ -436,6 +460,7 @@ int quasar_set_path(quasar_model* m, int32_t path) {
 
 int quasar_model_destroy(quasar_model* m) {
   if (m == nullptr) return QUASAR_OK;
+  if (m->mega_weights) cudaFree(m->mega_weights);
   if (m->mega_jobs) cudaFree(m->mega_jobs);
   if (m->mega_layers) cudaFree(m->mega_layers);
   if (m->rope_table) cudaFree(m->rope_table);

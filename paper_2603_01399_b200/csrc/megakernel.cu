@@ -3,21 +3,35 @@
 // barrier.  Section 3.4 models the pass as  T ~= M * bytes / BW : the pass is one long read
 // of the weights, so the design goal is that this read never stops.
 //
-//  * Every warp owns a private ring of shared-memory stages that it fills with cp.async
-//    from a STATIC schedule covering all GEMMs of the pass.  The schedule does not depend on
-//    activations, so a warp keeps prefetching the next GEMM's weights while the CTA is in
-//    an epilogue, an attention phase or a grid barrier (160 KB in flight per SM).
 //  * Each weight matrix is cut into contiguous row ranges, one per CTA, balanced to a single
 //    row, so all SMs stream the same number of bytes and no cross-CTA reduction exists.
-//    Inside a CTA the 16 warps split the contraction index; their partial sums meet in
-//    shared memory in a fixed order (deterministic results).
-//  * int8 -> bf16 in registers, mma.m16n8k16 with the weights as the 16-row operand and the
-//    <= 8 activation rows as the 8-wide operand held in registers for a whole phase.
+//    Inside a CTA the 16 consumer warps split the contraction index; their partial sums meet
+//    in shared memory in a fixed order (deterministic results).
+//  * At model creation the bytes of every CTA's row range are permuted (same size, same
+//    place) into the order in which that CTA consumes them: blocks of <= 16 rows x 1024
+//    bytes, each block contiguous, 16-byte pieces XOR-swizzled for conflict-free 128-bit
+//    shared-memory reads, int8 sign bits pre-flipped.  A ring stage is then ONE bulk
+//    asynchronous copy (cp.async.bulk) of up to 16 KB from a pointer that only moves forward:
+//    measured on B200, 16 KB copies stream at 7.0 TB/s where 1 KB row pieces reach 2.9 TB/s
+//    (the copy engine's cost is per request).
+//  * A dedicated producer warp walks a STATIC schedule covering every GEMM of the pass and
+//    fills the ring (completion counted in bytes by an mbarrier per stage).  The schedule
+//    does not depend on activations, so the producer keeps prefetching the next GEMM's
+//    weights while the consumer warps are in an epilogue, an attention phase or a grid
+//    barrier (160 KB in flight per SM), and loading costs the consumers no instructions.
+//  * int8 -> fp16 in registers at one instruction per weight: the byte, stored with its sign
+//    bit flipped, becomes the low mantissa byte of the fp16 number 1024 + (w + 128), and one
+//    packed subtraction of 1152 leaves w exactly.  The activations are bf16 values converted
+//    to fp16 (exact; a per-row power-of-two pre-scale keeps any bf16 row inside the fp16
+//    range), so mma.m16n8k16 f16 x f16 -> f32 computes the same products the bf16 operands
+//    would.  The weights are the 16-row operand, the <= 8 activation rows the 8-wide operand
+//    held in registers for a whole phase.
 //  * RMSNorm is fused into the operand load of the following GEMM, SwiGLU / residual adds
 //    into the GEMM epilogues, QK-RMSNorm + RoPE + KV append into the attention phase.
 //
-// Every wait is bounded: a grid barrier that does not complete within its poll budget sets
-// QUASAR_ERR_TIMEOUT in the status word and the CTA leaves (after draining its copies).
+// Every wait is bounded: a grid barrier or an mbarrier that does not complete within its
+// time budget sets QUASAR_ERR_TIMEOUT in the status word and the CTA leaves (after its own
+// copies in flight have landed).
 #include <cooperative_groups.h>
 #include <math.h>
 
@@ -28,41 +42,49 @@ namespace quasar {
 
 namespace {
 
-constexpr int NW = kMegaWarps;          // warps per CTA
-constexpr int kThreads = NW * 32;
-constexpr int kStageBytes = 2048;       // 16 weight rows x 128 bytes
-constexpr int kChunk = 4096;            // contraction elements the CTA covers per chunk
-constexpr int kSlice = kChunk / NW;     // contraction elements one warp covers per chunk
-constexpr int kStages = 80 / NW;        // ring depth per warp (160 KB of stages per CTA)
-constexpr int kXr = kSlice / 32;        // 16-byte registers holding this thread's share of the operand slice
-constexpr int GT = 4;                   // 16-row tiles accumulated together before a reduction
+constexpr int NW = kMegaWarps;             // consumer warps per CTA
+constexpr int kCT = NW * 32;               // consumer threads
+constexpr int kThreads = kCT + 128;        // + the producer's warp group (one of its warps issues the copies)
+constexpr int kConsumerRegs = 112;         // registers per thread after the split (setmaxnreg): 16 consumer warps
+constexpr int kProducerRegs = 40;          // ... and the 4 warps of the producer's group
+constexpr int kRowBytes = 1024;            // bytes of one weight row per stage
+constexpr int kStageBytes = 16 * kRowBytes;  // 16 weight rows
+constexpr int kStages = 10;                // ring depth (160 KB of weights in flight per CTA)
+constexpr int kChunk = 4096;               // contraction elements whose activations a warp keeps in registers
+constexpr int kXr = 8;                     // 16-byte registers holding this thread's share of the operand chunk
+constexpr int GT = 4;                      // 16-row tiles accumulated together before a reduction
 constexpr int kKeyTile = 64;
-constexpr int kMaxRowsAttn = 64;        // query rows (heads-in-group x block rows) per kv head
+constexpr int kMaxRowsAttn = 64;           // query rows (heads-in-group x block rows) per kv head
 constexpr float kLog2e = 1.4426950408889634f;
-constexpr unsigned kBarrierPolls = 4u << 20;
+constexpr unsigned long long kWaitBudgetNs = 2000000000ull;  // every device-side wait gives up after 2 s
 
 // ---- shared memory map --------------------------------------------------------------------
-constexpr int kRingBytes = NW * kStages * kStageBytes;                   // 163840
+constexpr int kRingBytes = kStages * kStageBytes;                        // 163840
 constexpr int kRedBytes = NW * GT * 128 * 4;                             // 32768
 constexpr int kKvTileBytes = kKeyTile * (128 + 8) * 2;                   // 17408 (D = 128)
 constexpr int kUnionBytes = (2 * kKvTileBytes > kRedBytes) ? 2 * kKvTileBytes : kRedBytes;
 constexpr int kQTileBytes = kMaxRowsAttn * (128 + 8) * 2;                // 17408
 constexpr int kMiscBytes = 2048;
 constexpr int kSmemBytes = kRingBytes + kUnionBytes + kQTileBytes + kMiscBytes;
+static_assert(kSmemBytes <= 227 * 1024, "shared memory budget of one SM");
 
-__device__ __forceinline__ void cp_async16(void* smem, const void* gmem, bool valid) {
-  const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem);
-  const int n = valid ? 16 : 0;
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(d), "l"(gmem), "r"(n) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
+// misc region (floats): [0,128) per-warp row sums, [128,136) running arg-max values, [136,144) its
+// indices, [144,152) 1/scale of the operand rows, [200] abort flag, [256,512) candidates / per-warp
+// row maxima, byte 1536.. the mbarriers.
+constexpr int kMiscRowSum = 0, kMiscRunV = 128, kMiscRunI = 136, kMiscInvScale = 144, kMiscAbort = 200,
+              kMiscCand = 256, kMiscBarBytes = 1536;
 
-__device__ __forceinline__ void mma16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
-                                         uint32_t b0, uint32_t b1) {
+__device__ __forceinline__ void mma16816_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                              uint32_t b0, uint32_t b1) {
   asm volatile(
       "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void mma16816_f16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                             uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
@@ -75,17 +97,19 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t& r0, uint32_t& r1, ui
                : "r"(addr));
 }
 
-// Four signed bytes -> four bf16 (exact), see the skinny GEMM.
-__device__ __forceinline__ void s8x4_to_bf16x4(uint32_t w, uint32_t& lo, uint32_t& hi) {
-  const uint32_t u = w ^ 0x80808080u;
-  const float f0 = __uint_as_float(__byte_perm(u, 0x4B000000u, 0x7440)) - 8388736.f;
-  const float f1 = __uint_as_float(__byte_perm(u, 0x4B000000u, 0x7441)) - 8388736.f;
-  const float f2 = __uint_as_float(__byte_perm(u, 0x4B000000u, 0x7442)) - 8388736.f;
-  const float f3 = __uint_as_float(__byte_perm(u, 0x4B000000u, 0x7443)) - 8388736.f;
-  __nv_bfloat162 p0 = __floats2bfloat162_rn(f0, f1);
-  __nv_bfloat162 p1 = __floats2bfloat162_rn(f2, f3);
-  lo = *reinterpret_cast<uint32_t*>(&p0);
-  hi = *reinterpret_cast<uint32_t*>(&p1);
+// Four weight bytes -> four fp16 (exact).  The repacked bytes hold u = w + 128 in [1, 255]
+// (sign bit flipped); placed under the high byte 0x64, u reads 1024 + u as fp16 (the spacing of
+// fp16 in [1024, 2048) is 1), and subtracting 1152 leaves w.  lo = bytes 0,1; hi = bytes 2,3.
+constexpr float kWeightUnit = 1.f;
+constexpr float kWeightOffset = 0.f;
+__device__ __forceinline__ void u8x4_to_f16x4(uint32_t u, uint32_t& lo, uint32_t& hi) {
+  const uint32_t l = __byte_perm(u, 0x64646464u, 0x4140);
+  const uint32_t h = __byte_perm(u, 0x64646464u, 0x4342);
+  const __half2 bias = __halves2half2(__ushort_as_half(0x6480), __ushort_as_half(0x6480));
+  const __half2 lo2 = __hsub2(*reinterpret_cast<const __half2*>(&l), bias);
+  const __half2 hi2 = __hsub2(*reinterpret_cast<const __half2*>(&h), bias);
+  lo = *reinterpret_cast<const uint32_t*>(&lo2);
+  hi = *reinterpret_cast<const uint32_t*>(&hi2);
 }
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
@@ -107,153 +131,287 @@ __device__ __forceinline__ float warp_sum(float v) {
   return v;
 }
 
+// barrier among the consumer warps only (the producer warp never joins it)
+__device__ __forceinline__ void cbar() { asm volatile("bar.sync 1, %0;\n" ::"n"(kCT) : "memory"); }
+
+__device__ __forceinline__ unsigned long long now_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;\n" : "=l"(t));
+  return t;
+}
+
+#ifdef QUASAR_PHASE_TIMER
+// Diagnostic build only: thread 0 of every CTA stamps the SM clock at each phase boundary.
+constexpr int kMaxMarks = 640;
+__device__ long long g_phase_clk[160][kMaxMarks];
+__device__ int g_phase_n[160];
+__device__ long long g_gemm_clk[160][4];   // warp 0 of every CTA: cycles waiting for stages, in stats, in epilogues, in GEMM phases
+#define PHASE_MARK()                                                                         \
+  do {                                                                                       \
+    if (threadIdx.x == 0 && mark_n < kMaxMarks) g_phase_clk[blockIdx.x][mark_n++] = clock64(); \
+  } while (0)
+#ifdef QUASAR_GEMM_TIMER
+#define GEMM_CLK(i, expr)                                           \
+  do {                                                              \
+    const long long c0__ = clock64();                               \
+    expr;                                                           \
+    if (threadIdx.x == 0) g_gemm_clk[blockIdx.x][i] += clock64() - c0__; \
+  } while (0)
+#else
+#define GEMM_CLK(i, expr) do { expr; } while (0)
+#endif
+#else
+#define PHASE_MARK() do { } while (0)
+#define GEMM_CLK(i, expr) do { expr; } while (0)
+#endif
+
+// ---- mbarriers ----------------------------------------------------------------------------
+__device__ __forceinline__ void mbar_init(uint64_t* bar, int count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"((uint32_t)__cvta_generic_to_shared(bar)), "r"(count)
+               : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"((uint32_t)__cvta_generic_to_shared(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"((uint32_t)__cvta_generic_to_shared(bar)),
+               "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
+      : "=r"(ok)
+      : "r"((uint32_t)__cvta_generic_to_shared(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Waits for the phase of `bar` with the given parity.  Gives up when another thread of the CTA
+// has raised the abort flag or after kWaitBudgetNs (then raises the flag and the status itself).
+__device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
+  const unsigned long long t0 = now_ns();
+  unsigned it = 0;
+  while (true) {
+    if (mbar_try(bar, parity)) return true;
+    if ((++it & 63u) == 0) {
+      if (*abort_flag) return false;
+      if (now_ns() - t0 > kWaitBudgetNs) {
+        atomicMin(status, QUASAR_ERR_TIMEOUT);
+        *abort_flag = 1;
+        return false;
+      }
+    }
+  }
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
+  if (mbar_try(bar, parity)) return true;
+  return mbar_wait_slow(bar, parity, abort_flag, status);
+}
+
+// One block of weights (a multiple of 16 bytes, both addresses 16-byte aligned) from global to
+// shared memory; completion is counted in bytes on `bar`.  The weights are read once per pass, so
+// the copy asks L2 to evict them first.
+__device__ __forceinline__ void bulk_copy(void* smem_dst, const void* gmem_src, uint32_t bytes, uint64_t* bar,
+                                              uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;\n" ::"r"(
+          (uint32_t)__cvta_generic_to_shared(smem_dst)),
+      "l"(gmem_src), "r"(bytes), "r"((uint32_t)__cvta_generic_to_shared(bar)), "l"(policy)
+      : "memory");
+}
+
 // ---- the static weight schedule -----------------------------------------------------------
-// Position of one warp in the sequence of ring stages of the whole pass.  Order:
-// job -> tile group -> contraction chunk -> tile in group -> 128-byte piece of the warp's slice.
+// Order of the ring stages of the whole pass, identical for the producer, the consumers and
+// the repacked weight layout:  job -> tile group -> contraction chunk -> tile in group ->
+// 1024-byte piece of the chunk.  A stage holds one block: the rows of one tile (<= 16) x one
+// piece, rows at a pitch of the piece's bytes.
 struct JobView {
-  const unsigned char* w;
+  const unsigned char* wp;   // this CTA's repacked row range
   int K, units, u0, u1, rows_per_tile, tiles, ngroups, nchunks, kind, n_rows;
 };
 
-__device__ __forceinline__ JobView job_view(const MegaJob* jobs, int j, int cta, int ncta) {
-  JobView v;
-  const MegaJob jb = jobs[j];
-  v.w = reinterpret_cast<const unsigned char*>(jb.w);
-  v.K = jb.K;
-  v.kind = jb.kind;
-  v.n_rows = jb.N;
-  v.units = (jb.kind == kJobGateUp) ? jb.N / 2 : jb.N;
+__device__ __forceinline__ void job_split(int kind, int N, int K, int cta, int ncta, JobView& v) {
+  v.K = K;
+  v.kind = kind;
+  v.n_rows = N;
+  v.units = (kind == kJobGateUp) ? N / 2 : N;
   v.u0 = (int)(((long long)cta * v.units) / ncta);
   v.u1 = (int)(((long long)(cta + 1) * v.units) / ncta);
-  v.rows_per_tile = (jb.kind == kJobGateUp) ? 8 : 16;
+  v.rows_per_tile = (kind == kJobGateUp) ? 8 : 16;
   v.tiles = (v.u1 - v.u0 + v.rows_per_tile - 1) / v.rows_per_tile;
   v.ngroups = (v.tiles + GT - 1) / GT;
-  v.nchunks = (jb.K + kChunk - 1) / kChunk;
-  return v;
-}
-
-// global weight row behind ring row r (0..15) of tile `tile`, or -1 when the slot is padding
-__device__ __forceinline__ int ring_row_to_global(const JobView& v, int tile, int r) {
-  if (v.kind == kJobGateUp) {
-    const int p = v.u0 + tile * 8 + (r & 7);
-    if (p >= v.u1) return -1;
-    return (r < 8) ? p : v.units + p;
-  }
-  const int n = v.u0 + tile * 16 + r;
-  return n < v.u1 ? n : -1;
+  v.nchunks = (K + kChunk - 1) / kChunk;
 }
 
 template <bool W_INT8>
-struct Producer {
-  static constexpr int kStageElems = W_INT8 ? 128 : 64;
-  static constexpr int KB = kSlice / kStageElems;    // ring stages per (tile, chunk) per warp
-  const MegaJob* jobs;
-  int n_jobs, cta, ncta, warp, lane;
-  int job, tg, kc, tile, kb;
+__device__ __forceinline__ JobView job_view(const MegaJob* jobs, int j, int cta, int ncta) {
   JobView v;
-  bool done;
+  const MegaJob jb = jobs[j];
+  job_split(jb.kind, jb.N, jb.K, cta, ncta, v);
+  const size_t row_bytes = (size_t)jb.K * (W_INT8 ? 1 : 2);
+  v.wp = reinterpret_cast<const unsigned char*>(jb.wp) + (size_t)(jb.kind == kJobGateUp ? 2 * v.u0 : v.u0) * row_bytes;
+  return v;
+}
 
-  __device__ void init(const MegaJob* j, int nj, int c, int nc, int w, int l) {
-    jobs = j; n_jobs = nj; cta = c; ncta = nc; warp = w; lane = l;
-    job = -1; tg = kc = tile = kb = 0; done = false;
-    next_job();
+// units (output channels, or gate/up pairs) of tile `tile` of this CTA, and rows of its blocks
+__device__ __forceinline__ int tile_units(const JobView& v, int tile) {
+  return min(v.rows_per_tile, v.u1 - v.u0 - tile * v.rows_per_tile);
+}
+__device__ __forceinline__ int tile_rows(const JobView& v, int tile) {
+  const int u = tile_units(v, tile);
+  return v.kind == kJobGateUp ? 2 * u : u;
+}
+// global weight row stored in row `r` of the blocks of tile `tile` (r < tile_rows): a gate/up
+// tile keeps its gate rows first, then the matching up rows
+__device__ __forceinline__ int block_row_to_global(const JobView& v, int tile, int r) {
+  if (v.kind == kJobGateUp) {
+    const int u = tile_units(v, tile);
+    const int p = v.u0 + tile * 8 + (r < u ? r : r - u);
+    return r < u ? p : v.units + p;
   }
-  __device__ void next_job() {
-    while (true) {
-      ++job;
-      if (job >= n_jobs) { done = true; return; }
-      v = job_view(jobs, job, cta, ncta);
-      if (v.tiles > 0) break;
-    }
-    tg = kc = tile = kb = 0;
-  }
-  __device__ void advance() {
-    if (++kb < KB) return;
-    kb = 0;
-    const int gt = min(GT, v.tiles - tg * GT);
-    if (++tile < gt) return;
-    tile = 0;
-    if (++kc < v.nchunks) return;
-    kc = 0;
-    if (++tg < v.ngroups) return;
-    next_job();
-  }
-  // issue the copies of the current stage into `slot` and move on (always exactly one commit group)
-  __device__ void fetch(unsigned char* slot) {
-    if (!done) {
-      const int kbase = kc * kChunk + warp * kSlice + kb * kStageElems;
-      const int t_global = tg * GT + tile;
-      constexpr int kElemsPer16 = W_INT8 ? 16 : 8;
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const int q = lane + 32 * i;
-        const int r = q >> 3, c = q & 7;
-        const int n = ring_row_to_global(v, t_global, r);
-        const int k = kbase + c * kElemsPer16;
-        const bool ok = (n >= 0) && (k < v.K);
-        const unsigned char* src = v.w + ((size_t)(ok ? n : 0) * v.K + (ok ? k : 0)) * (W_INT8 ? 1 : 2);
-        cp_async16(slot + r * 128 + ((c * 16) ^ ((r & 1) << 6)), src, ok);
-      }
-      advance();
-    }
-    cp_async_commit();
-  }
+  return v.u0 + tile * 16 + r;
+}
+
+struct Pipe {
+  unsigned char* ring;
+  uint64_t* full;    // [kStages] producer -> consumers: the stage's bytes have landed
+  uint64_t* empty;   // [kStages] consumers -> producer: all 16 warps are done with the stage
+  volatile int* abort_flag;
+  int32_t* status;
 };
 
-// ---- bounded grid barrier -----------------------------------------------------------------
+template <bool W_INT8>
+__device__ void producer_loop(const MegaParams& p, const Pipe& pipe, int cta, int ncta) {
+  constexpr int kElemBytes = W_INT8 ? 1 : 2;
+  constexpr int kChunkBytes = kChunk * kElemBytes;
+  if ((threadIdx.x & 31) != 0) return;   // one thread issues every copy
+  uint64_t policy;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;\n" : "=l"(policy));
+  int slot = 0;
+  uint32_t phase = 0;
+  long long issued = 0;
+  bool ok = true;
+  for (int job = 0; job < p.n_jobs && ok; ++job) {
+    const JobView v = job_view<W_INT8>(p.jobs, job, cta, ncta);
+    const unsigned char* src = v.wp;
+    const int kbytes = v.K * kElemBytes;
+    for (int tg = 0; tg < v.ngroups && ok; ++tg) {
+      const int gt = min(GT, v.tiles - tg * GT);
+      for (int kc = 0; kc < v.nchunks && ok; ++kc) {
+        const int cb = min(kChunkBytes, kbytes - kc * kChunkBytes);
+        for (int tile = 0; tile < gt && ok; ++tile) {
+          const int rows = tile_rows(v, tg * GT + tile);
+          for (int b0 = 0; b0 < cb; b0 += kRowBytes) {
+            const uint32_t bytes = (uint32_t)(rows * min(kRowBytes, cb - b0));
+            if (!mbar_wait(pipe.empty + slot, phase ^ 1u, pipe.abort_flag, pipe.status)) { ok = false; break; }
+            mbar_arrive_expect_tx(pipe.full + slot, bytes);
+            bulk_copy(pipe.ring + slot * kStageBytes, src, bytes, pipe.full + slot, policy);
+            src += bytes;
+            ++issued;
+            if (++slot == kStages) { slot = 0; phase ^= 1u; }
+          }
+        }
+      }
+    }
+  }
+  // Nothing of ours may still be in flight when the CTA leaves: wait (bounded) for the stages
+  // armed last.  On the normal path the consumers have already waited for all of them.
+  const int back = issued < kStages ? (int)issued : kStages;
+  for (int i = 0; i < back; ++i) {
+    if (--slot < 0) { slot = kStages - 1; phase ^= 1u; }
+    const unsigned long long t0 = now_ns();
+    while (!mbar_try(pipe.full + slot, phase)) {
+      if (now_ns() - t0 > kWaitBudgetNs) { atomicMin(pipe.status, QUASAR_ERR_TIMEOUT); break; }
+    }
+  }
+}
+
+// ---- bounded grid barrier (consumer warps) ---------------------------------------------------
 struct GridSync {
   unsigned* counter;
   int32_t* status;
   unsigned ncta;
   unsigned epoch;
-  int* abort_flag;  // shared memory
+  volatile int* abort_flag;  // shared memory
   __device__ bool sync() {
-    __syncthreads();
+    cbar();
     if (threadIdx.x == 0) {
       ++epoch;
       __threadfence();
       atomicAdd(counter, 1u);
       const unsigned target = epoch * ncta;
+      const unsigned long long t0 = now_ns();
       unsigned polls = 0;
       while (true) {
         unsigned v;
         asm volatile("ld.acquire.gpu.global.u32 %0, [%1];\n" : "=r"(v) : "l"(counter) : "memory");
         if (v >= target) break;
-        if (++polls > kBarrierPolls) {
+        if ((++polls & 255u) == 0 && (*abort_flag || now_ns() - t0 > kWaitBudgetNs)) {
           atomicMin(status, QUASAR_ERR_TIMEOUT);
           *abort_flag = 1;
           break;
         }
-        __nanosleep(20);
       }
     } else {
       epoch++;
     }
-    __syncthreads();
+    cbar();
     return *abort_flag == 0;
   }
 };
 
-// ---- operand load: the <= 8 activation rows of this warp's contraction slice ------------------
-// xr[0..kXr): for int8 weights step s (64 elements) uses xr[2s], xr[2s+1] (16 bf16 of row g at
-// k = base + s*64 + t*16); for bf16 weights step s (32 elements) uses xr[s] (8 bf16 at base + s*32 + t*8).
+// ---- operand load: the <= 8 activation rows of this warp's share of a contraction chunk ----------
+// A stage holds a 1024-byte piece of every weight row of a tile; warp w reads bytes [64 w, 64 w + 64)
+// of the piece and lane (g, t) the 16 bytes at 16 t.  int8 weights: stage s of the chunk covers k = base + 1024 s + 64 w +
+// 16 t + (0..15), held in xr[2s], xr[2s+1] (fp16).  bf16 weights: k = base + 512 s + 32 w + 8 t + (0..7),
+// held in xr[s] (bf16).
+template <bool W_INT8>
+__device__ __forceinline__ int x_index(int i, int kbase, int warp, int t) {
+  return W_INT8 ? (kbase + (i >> 1) * 1024 + warp * 64 + t * 16 + (i & 1) * 8) : (kbase + i * 512 + warp * 32 + t * 8);
+}
+
 template <bool W_INT8>
 __device__ __forceinline__ void load_x_raw(uint4 (&xr)[kXr], const __nv_bfloat16* src, int ld, int M, int K, int kbase,
-                                           int g, int t) {
+                                           int warp, int g, int t) {
 #pragma unroll
   for (int i = 0; i < kXr; ++i) {
-    const int k = W_INT8 ? (kbase + (i >> 1) * 64 + t * 16 + (i & 1) * 8) : (kbase + i * 32 + t * 8);
+    const int k = x_index<W_INT8>(i, kbase, warp, t);
     xr[i] = make_uint4(0, 0, 0, 0);
     if (g < M && k < K) xr[i] = __ldcg(reinterpret_cast<const uint4*>(src + (size_t)g * ld + k));
   }
 }
 
+// per-row statistics of the raw operand: sum of squares and max |x * gain| (gain may be null)
 template <bool W_INT8>
-__device__ __forceinline__ void apply_norm(uint4 (&xr)[kXr], const __nv_bfloat16* gain, float r, int K, int kbase,
-                                           int t) {
+__device__ __forceinline__ void x_stats(const uint4 (&xr)[kXr], const __nv_bfloat16* gain, int K, int kbase, int warp,
+                                        int t, float& ss, float& amax) {
 #pragma unroll
   for (int i = 0; i < kXr; ++i) {
-    const int k = W_INT8 ? (kbase + (i >> 1) * 64 + t * 16 + (i & 1) * 8) : (kbase + i * 32 + t * 8);
+    const int k = x_index<W_INT8>(i, kbase, warp, t);
+    if (k < K) {
+      uint4 gv = make_uint4(0x3f803f80u, 0x3f803f80u, 0x3f803f80u, 0x3f803f80u);  // bf16 ones
+      if (gain != nullptr) gv = __ldg(reinterpret_cast<const uint4*>(gain + k));
+      const __nv_bfloat162* xp = reinterpret_cast<const __nv_bfloat162*>(&xr[i]);
+      const __nv_bfloat162* gp = reinterpret_cast<const __nv_bfloat162*>(&gv);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float2 xf = __bfloat1622float2(xp[e]);
+        const float2 gf = __bfloat1622float2(gp[e]);
+        ss += xf.x * xf.x + xf.y * xf.y;
+        amax = fmaxf(amax, fmaxf(fabsf(xf.x * gf.x), fabsf(xf.y * gf.y)));
+      }
+    }
+  }
+}
+
+// h = bf16(x * r * gain) in place (the RMSNorm output, rounded where the decoder layer rounds it)
+template <bool W_INT8>
+__device__ __forceinline__ void apply_norm(uint4 (&xr)[kXr], const __nv_bfloat16* gain, float r, int K, int kbase,
+                                           int warp, int t) {
+#pragma unroll
+  for (int i = 0; i < kXr; ++i) {
+    const int k = x_index<W_INT8>(i, kbase, warp, t);
     if (k < K) {
       const uint4 gv = __ldg(reinterpret_cast<const uint4*>(gain + k));
       const __nv_bfloat162* xp = reinterpret_cast<const __nv_bfloat162*>(&xr[i]);
@@ -270,92 +428,137 @@ __device__ __forceinline__ void apply_norm(uint4 (&xr)[kXr], const __nv_bfloat16
   }
 }
 
-__device__ __forceinline__ float sumsq(const uint4 (&xr)[kXr]) {
-  float s = 0.f;
+// bf16 -> fp16 in place after multiplying by the row's power-of-two scale (exact unless the
+// scaled value falls below the fp16 normal range).  Returns the sum of the fp16 values written
+// (the epilogue needs sum_k x_k to remove the weights' offset).
+__device__ __forceinline__ float to_f16(uint4 (&xr)[kXr], float scale) {
+  float sum = 0.f;
 #pragma unroll
   for (int i = 0; i < kXr; ++i) {
-    const __nv_bfloat162* xp = reinterpret_cast<const __nv_bfloat162*>(&xr[i]);
+    uint32_t* w = reinterpret_cast<uint32_t*>(&xr[i]);
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
-      const float2 f = __bfloat1622float2(xp[e]);
-      s += f.x * f.x + f.y * f.y;
+      const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w[e]));
+      const __half2 h = __floats2half2_rn(f.x * scale, f.y * scale);
+      const float2 b = __half22float2(h);
+      sum += b.x + b.y;
+      w[e] = *reinterpret_cast<const uint32_t*>(&h);
     }
   }
-  return s;
+  return sum;
 }
 
+// One stage = one block [rows][pb bytes].  MMA row g of the tile is block row ra, MMA row g + 8
+// block row rb; the 16-byte pieces of a row are XOR-swizzled by its parity when pb is a multiple
+// of 128 (off_a / off_b are this lane's byte offsets, computed once per tile and piece size).
+// The MMAs of a stage go to separate accumulators so that no MMA waits for the one before it.
 template <bool W_INT8>
-__device__ __forceinline__ void consume_stage(const unsigned char* stage, int kb, const uint4 (&xr)[kXr],
-                                              float (&acc)[4], int g, int t) {
-#pragma unroll
-  for (int s = 0; s < 2; ++s) {
-    const int off = (s * 64 + t * 16) ^ ((g & 1) << 6);
-    const uint4 wa = *reinterpret_cast<const uint4*>(stage + g * 128 + off);
-    const uint4 wb = *reinterpret_cast<const uint4*>(stage + (g + 8) * 128 + off);
-    const int step = kb * 2 + s;
-    if (W_INT8) {
-      const uint4 x0 = xr[2 * step], x1 = xr[2 * step + 1];
-      uint32_t a0, a1, a2, a3;
-      s8x4_to_bf16x4(wa.x, a0, a2); s8x4_to_bf16x4(wb.x, a1, a3);
-      mma16816(acc, a0, a1, a2, a3, x0.x, x0.y);
-      s8x4_to_bf16x4(wa.y, a0, a2); s8x4_to_bf16x4(wb.y, a1, a3);
-      mma16816(acc, a0, a1, a2, a3, x0.z, x0.w);
-      s8x4_to_bf16x4(wa.z, a0, a2); s8x4_to_bf16x4(wb.z, a1, a3);
-      mma16816(acc, a0, a1, a2, a3, x1.x, x1.y);
-      s8x4_to_bf16x4(wa.w, a0, a2); s8x4_to_bf16x4(wb.w, a1, a3);
-      mma16816(acc, a0, a1, a2, a3, x1.z, x1.w);
-    } else {
-      const uint4 x0 = xr[step];
-      mma16816(acc, wa.x, wb.x, wa.y, wb.y, x0.x, x0.y);
-      mma16816(acc, wa.z, wb.z, wa.w, wb.w, x0.z, x0.w);
-    }
+__device__ __forceinline__ void consume_stage(const unsigned char* stage, int s, int off_a, int off_b, bool lane_valid,
+                                              const uint4 (&xr)[kXr], float (&acc)[4][4]) {
+  uint4 wa = *reinterpret_cast<const uint4*>(stage + off_a);
+  uint4 wb = *reinterpret_cast<const uint4*>(stage + off_b);
+  if (W_INT8) {
+    // bytes no copy has written convert to finite numbers: they meet zero activations (k beyond K)
+    // or land in accumulator rows that are never stored (rows beyond the tile)
+    const uint4 x0 = xr[2 * s], x1 = xr[2 * s + 1];
+    uint32_t a0, a1, a2, a3;
+    u8x4_to_f16x4(wa.x, a0, a2); u8x4_to_f16x4(wb.x, a1, a3);
+    mma16816_f16(acc[0], a0, a1, a2, a3, x0.x, x0.y);
+    u8x4_to_f16x4(wa.y, a0, a2); u8x4_to_f16x4(wb.y, a1, a3);
+    mma16816_f16(acc[1], a0, a1, a2, a3, x0.z, x0.w);
+    u8x4_to_f16x4(wa.z, a0, a2); u8x4_to_f16x4(wb.z, a1, a3);
+    mma16816_f16(acc[2], a0, a1, a2, a3, x1.x, x1.y);
+    u8x4_to_f16x4(wa.w, a0, a2); u8x4_to_f16x4(wb.w, a1, a3);
+    mma16816_f16(acc[3], a0, a1, a2, a3, x1.z, x1.w);
+  } else {
+    if (!lane_valid) { wa = make_uint4(0, 0, 0, 0); wb = make_uint4(0, 0, 0, 0); }  // stale bytes may be NaN patterns
+    const uint4 x0 = xr[s];
+    mma16816_bf16(acc[0], wa.x, wb.x, wa.y, wb.y, x0.x, x0.y);
+    mma16816_bf16(acc[1], wa.z, wb.z, wa.w, wb.w, x0.z, x0.w);
   }
 }
 
-// ---- one GEMM phase -----------------------------------------------------------------------
+// byte offset, inside a block of pitch pb, of the 16 bytes lane (warp, t) reads from block row r
+__device__ __forceinline__ int block_offset(int r, int pb, int warp, int t) {
+  int chunk = warp * 4 + t;
+  if ((pb & 127) == 0) chunk ^= (r & 1) << 2;
+  return r * pb + chunk * 16;
+}
+
+// ---- one GEMM phase (consumer warps) -------------------------------------------------------------
 template <bool W_INT8>
 struct GemmPhase {
-  static constexpr int KB = Producer<W_INT8>::KB;
+  static constexpr int kElemBytes = W_INT8 ? 1 : 2;
+  static constexpr int kStageElems = kRowBytes / kElemBytes;
+  static constexpr int SPC = kChunk / kStageElems;   // stages per chunk: 4 (int8) or 8 (bf16)
 
-  __device__ __noinline__ static void run(const MegaParams& p, int job, Producer<W_INT8>& prod_io,
-                                          unsigned char* ring, unsigned& cstage_io, float* red, float* misc, int cta,
-                                          int ncta) {
-    Producer<W_INT8> prod = prod_io;  // registers while the phase runs
-    unsigned cstage = cstage_io;
+  __device__ __forceinline__ static bool run(const MegaParams& p, int job, const Pipe& pipe, int& slot_io,
+                                          uint32_t& phase_io, float* red, float* misc, int cta, int ncta) {
+    int slot = slot_io;
+    uint32_t phase = phase_io;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
-    const JobView v = job_view(p.jobs, job, cta, ncta);
+    const JobView v = job_view<W_INT8>(p.jobs, job, cta, ncta);
     const MegaJob jb = p.jobs[job];
     const int M = p.M;
     const bool normed = jb.gain != nullptr;
     const __nv_bfloat16* xsrc = jb.kind == kJobO ? p.attn : (jb.kind == kJobDown ? p.act : p.x);
     const int ld = jb.K;
 
-    // RMSNorm factor of every row (the operand of a normed GEMM is h = x * r * gain)
-    float rnorm = 1.f;
+    // Row statistics of the operand: the RMSNorm factor (normed GEMMs: the operand is
+    // h = x * r * gain) and, for the fp16 path, a power-of-two scale that keeps the row in range.
+    float rnorm = 1.f, xscale = 1.f;
+    float xsum = 0.f;   // this lane's share of sum_k x_k over the whole contraction (fp16 operand values)
     uint4 xr[kXr];
     bool have_x = false;
-    if (normed) {
-      float ss = 0.f;
+#ifdef QUASAR_GEMM_TIMER
+    const long long c_stats0 = clock64();
+#endif
+    if (normed || W_INT8) {
+      float ss = 0.f, amax = 0.f;
       for (int kc = 0; kc < v.nchunks; ++kc) {
-        load_x_raw<W_INT8>(xr, xsrc, ld, M, jb.K, kc * kChunk + warp * kSlice, g, t);
-        ss += sumsq(xr);
+        load_x_raw<W_INT8>(xr, xsrc, ld, M, jb.K, kc * kChunk, warp, g, t);
+        x_stats<W_INT8>(xr, jb.gain, jb.K, kc * kChunk, warp, t, ss, amax);
       }
       ss += __shfl_xor_sync(0xffffffffu, ss, 1);
       ss += __shfl_xor_sync(0xffffffffu, ss, 2);
-      if (t == 0) misc[warp * 8 + g] = ss;
-      __syncthreads();
-      float tot = 0.f;
+      amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
+      amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
+      if (t == 0) {
+        misc[kMiscRowSum + warp * 8 + g] = ss;
+        misc[kMiscCand + warp * 8 + g] = amax;
+      }
+      cbar();
+      float tot = 0.f, mx = 0.f;
 #pragma unroll
-      for (int w = 0; w < NW; ++w) tot += misc[w * 8 + g];
-      rnorm = 1.0f / sqrtf(tot / (float)jb.K + p.rms_eps);
-      __syncthreads();
+      for (int w = 0; w < NW; ++w) {
+        tot += misc[kMiscRowSum + w * 8 + g];
+        mx = fmaxf(mx, misc[kMiscCand + w * 8 + g]);
+      }
+      if (normed) {
+        rnorm = 1.0f / sqrtf(tot / (float)jb.K + p.rms_eps);
+        mx *= rnorm * 1.01f;
+      }
+      float inv = 1.f;
+      if (W_INT8 && mx > 32768.f && mx < 3.0e38f) {
+        int e;
+        (void)frexpf(mx, &e);               // mx = f * 2^e, f in [0.5, 1)
+        xscale = ldexpf(1.f, 15 - e);       // scaled row maximum <= 2^15
+        inv = ldexpf(1.f, e - 15);
+      }
+      cbar();                               // everyone has read the per-warp partials
+      if (warp == 0 && t == 0) misc[kMiscInvScale + g] = inv;
       if (v.nchunks == 1) {
-        apply_norm<W_INT8>(xr, jb.gain, rnorm, jb.K, warp * kSlice, t);
+        if (normed) apply_norm<W_INT8>(xr, jb.gain, rnorm, jb.K, 0, warp, t);
+        if (W_INT8) xsum = to_f16(xr, xscale);
         have_x = true;
       }
+    } else if (warp == 0 && t == 0) {
+      misc[kMiscInvScale + g] = 1.f;
     }
 
-    // per-CTA arg-max state of the LM head (thread tid < 8*... handled in the epilogue)
+#ifdef QUASAR_GEMM_TIMER
+    if (threadIdx.x == 0) g_gemm_clk[blockIdx.x][1] += clock64() - c_stats0;
+#endif
     for (int tg = 0; tg < v.ngroups; ++tg) {
       const int gt = min(GT, v.tiles - tg * GT);
       float acc[GT][4];
@@ -363,21 +566,49 @@ struct GemmPhase {
       for (int i = 0; i < GT; ++i) acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.f;
       for (int kc = 0; kc < v.nchunks; ++kc) {
         if (!have_x) {
-          load_x_raw<W_INT8>(xr, xsrc, ld, M, jb.K, kc * kChunk + warp * kSlice, g, t);
-          if (normed) apply_norm<W_INT8>(xr, jb.gain, rnorm, jb.K, kc * kChunk + warp * kSlice, t);
+          load_x_raw<W_INT8>(xr, xsrc, ld, M, jb.K, kc * kChunk, warp, g, t);
+          if (normed) apply_norm<W_INT8>(xr, jb.gain, rnorm, jb.K, kc * kChunk, warp, t);
+          if (W_INT8) {
+            const float part = to_f16(xr, xscale);
+            if (tg == 0) xsum += part;       // every chunk is visited once per tile group
+          }
           have_x = (v.nchunks == 1);
         }
+        const int kbase = kc * kChunk;
+        const int cb = min(kChunk, jb.K - kbase) * kElemBytes;        // bytes of a weight row in this chunk
+        const int pb_last = cb - (cb - 1) / kRowBytes * kRowBytes;    // bytes of its last piece
 #pragma unroll
         for (int tile = 0; tile < GT; ++tile) {
           if (tile < gt) {
+            // block rows behind MMA rows g and g + 8 (rows past the tile stay inside the stage and feed
+            // accumulator rows that are never stored)
+            const int ra = g;
+            const int rb = v.kind == kJobGateUp ? tile_units(v, tg * GT + tile) + g : g + 8;
+            const int oa_full = block_offset(ra, kRowBytes, warp, t), ob_full = block_offset(rb, kRowBytes, warp, t);
+            const int oa_last = block_offset(ra, pb_last, warp, t), ob_last = block_offset(rb, pb_last, warp, t);
+            float ch[4][4];
 #pragma unroll
-            for (int kb = 0; kb < KB; ++kb) {
-              cp_async_wait<kStages - 2>();
-              __syncwarp();
-              prod.fetch(ring + ((cstage + kStages - 1) % kStages) * kStageBytes);
-              consume_stage<W_INT8>(ring + (cstage % kStages) * kStageBytes, kb, xr, acc[tile], g, t);
-              ++cstage;
+            for (int i = 0; i < 4; ++i) ch[i][0] = ch[i][1] = ch[i][2] = ch[i][3] = 0.f;
+#pragma unroll
+            for (int s = 0; s < SPC; ++s) {
+              const int b0 = s * kRowBytes;
+              if (b0 < cb) {
+                const bool last = b0 + kRowBytes >= cb;
+                const bool lane_valid = b0 + warp * 64 + t * 16 < cb;
+                bool got;
+                GEMM_CLK(0, got = mbar_wait(pipe.full + slot, phase, pipe.abort_flag, pipe.status));
+                if (!got) return false;
+                // a lane past the end of a short piece reads inside the stage (offset < 16 KB) but not its own data
+                const int oa = last ? (lane_valid ? oa_last : 0) : oa_full;
+                const int ob = last ? (lane_valid ? ob_last : 0) : ob_full;
+                GEMM_CLK(3, consume_stage<W_INT8>(pipe.ring + slot * kStageBytes, s, oa, ob, lane_valid, xr, ch);
+                         __syncwarp();
+                         if (lane == 0) mbar_arrive(pipe.empty + slot));
+                if (++slot == kStages) { slot = 0; phase ^= 1u; }
+              }
             }
+#pragma unroll
+            for (int i = 0; i < 4; ++i) acc[tile][i] += (ch[0][i] + ch[1][i]) + (ch[2][i] + ch[3][i]);
           }
         }
       }
@@ -388,12 +619,17 @@ struct GemmPhase {
         *reinterpret_cast<float2*>(r + g * 8 + 2 * t) = make_float2(acc[tile][0], acc[tile][1]);
         *reinterpret_cast<float2*>(r + (g + 8) * 8 + 2 * t) = make_float2(acc[tile][2], acc[tile][3]);
       }
-      __syncthreads();
-      epilogue(p, jb, v, tg, gt, red, misc);
-      __syncthreads();
+      if (W_INT8 && tg == 0) {   // per-warp share of sum_k x_k of operand row g
+        float xs = xsum;
+        xs += __shfl_xor_sync(0xffffffffu, xs, 1);
+        xs += __shfl_xor_sync(0xffffffffu, xs, 2);
+        if (t == 0) misc[kMiscRowSum + warp * 8 + g] = xs;
+      }
+      GEMM_CLK(2, cbar(); epilogue(p, jb, v, tg, gt, red, misc); cbar());
     }
-    prod_io = prod;
-    cstage_io = cstage;
+    slot_io = slot;
+    phase_io = phase;
+    return true;
   }
 
   __device__ static float reduce_at(const float* red, int tile, int row, int col) {
@@ -406,15 +642,26 @@ struct GemmPhase {
   __device__ static void epilogue(const MegaParams& p, const MegaJob& jb, const JobView& v, int tg, int gt,
                                   const float* red, float* misc) {
     const int M = p.M;
+    // A thread always meets the same operand row `col` (kCT is a multiple of 128).  out = (sum - corr) * unit:
+    // corr removes the weights' offset, unit undoes the operand's scale and the 2^-24 of the byte trick.
+    const int my_col = jb.kind == kJobGateUp ? (threadIdx.x >> 3) & 7 : (threadIdx.x >> 4) & 7;
+    float corr = 0.f, unit = 1.f;
+    if (W_INT8) {
+      float xs = 0.f;
+#pragma unroll
+      for (int w = 0; w < NW; ++w) xs += misc[kMiscRowSum + w * 8 + my_col];
+      corr = kWeightOffset * xs;
+      unit = kWeightUnit * misc[kMiscInvScale + my_col];
+    }
     if (jb.kind == kJobGateUp) {
       const int F = v.units;
-      for (int e = threadIdx.x; e < gt * 8 * 8; e += kThreads) {
+      for (int e = threadIdx.x; e < gt * 8 * 8; e += kCT) {
         const int r = e & 7, col = (e >> 3) & 7, tile = e >> 6;
         const int pair = v.u0 + (tg * GT + tile) * 8 + r;
         if (pair >= v.u1 || col >= M) continue;
         const float dg = jb.delta ? jb.delta[pair] : 1.f, du = jb.delta ? jb.delta[F + pair] : 1.f;
-        const float gate = bf16_round_f(reduce_at(red, tile, r, col) * dg);
-        const float up = bf16_round_f(reduce_at(red, tile, r + 8, col) * du);
+        const float gate = bf16_round_f((reduce_at(red, tile, r, col) - corr) * unit * dg);
+        const float up = bf16_round_f((reduce_at(red, tile, r + 8, col) - corr) * unit * du);
         p.act[(size_t)col * F + pair] = __float2bfloat16_rn(gate / (1.0f + expf(-gate)) * up);
       }
       return;
@@ -422,17 +669,17 @@ struct GemmPhase {
     const int N = jb.N;
     float best = -INFINITY;
     int best_i = 0x7fffffff;
-    for (int e = threadIdx.x; e < gt * 16 * 8; e += kThreads) {
+    for (int e = threadIdx.x; e < gt * 16 * 8; e += kCT) {
       const int r = e & 15, col = (e >> 4) & 7, tile = e >> 7;
       const int n = v.u0 + (tg * GT + tile) * 16 + r;
       if (n >= v.u1 || col >= M) continue;
-      const float val = reduce_at(red, tile, r, col) * (jb.delta ? jb.delta[n] : 1.f);
+      const float val = (reduce_at(red, tile, r, col) - corr) * unit * (jb.delta ? jb.delta[n] : 1.f);
       const size_t idx = (size_t)col * N + n;
       if (jb.kind == kJobQkv) {
         p.qkv[idx] = __float2bfloat16_rn(val);
       } else if (jb.kind == kJobLm) {
         if (p.logits) p.logits[idx] = val;
-        // e -> (tile, col, r): a thread sees a single col when kThreads % 128 == 0
+        // e -> (tile, col, r): a thread sees a single col because kCT % 128 == 0
         if (val > best || (val == best && n < best_i)) { best = val; best_i = n; }
       } else {  // o / down: residual add into the stream
         const float xv = __bfloat162float(__ldcg(p.x + idx));
@@ -440,8 +687,6 @@ struct GemmPhase {
       }
     }
     if (jb.kind == kJobLm) {
-      // running arg-max of this CTA's vocabulary range: misc[128 + col*2] (value), [.. + 1] (index)
-      const int col = (threadIdx.x >> 4) & 7;
       // combine the 16 lanes that share a col (lanes differ in r), then the 4 such groups per col in the CTA
 #pragma unroll
       for (int o = 8; o > 0; o >>= 1) {
@@ -449,19 +694,19 @@ struct GemmPhase {
         const int oi = __shfl_xor_sync(0xffffffffu, best_i, o);
         if (ob > best || (ob == best && oi < best_i)) { best = ob; best_i = oi; }
       }
-      float* cand_v = misc + 256;
-      int* cand_i = reinterpret_cast<int*>(misc + 256 + 64);
+      float* cand_v = misc + kMiscCand;
+      int* cand_i = reinterpret_cast<int*>(misc + kMiscCand + 64);
       if ((threadIdx.x & 15) == 0) {
         cand_v[threadIdx.x >> 4] = best;
         cand_i[threadIdx.x >> 4] = best_i;
       }
-      __syncthreads();
+      cbar();
       if (threadIdx.x < 8) {
-        float* run_v = misc + 128;
-        int* run_i = reinterpret_cast<int*>(misc + 128 + 8);
+        float* run_v = misc + kMiscRunV;
+        int* run_i = reinterpret_cast<int*>(misc + kMiscRunI);
         float bv = run_v[threadIdx.x];
         int bi = run_i[threadIdx.x];
-        for (int q = 0; q < kThreads / 16; ++q) {
+        for (int q = 0; q < kCT / 16; ++q) {
           if (((q & 7) == (int)threadIdx.x)) {
             const float ov = cand_v[q];
             const int oi = cand_i[q];
@@ -471,7 +716,6 @@ struct GemmPhase {
         run_v[threadIdx.x] = bv;
         run_i[threadIdx.x] = bi;
       }
-      (void)col;
     }
   }
 };
@@ -505,7 +749,7 @@ __device__ void prep_phase(const MegaParams& p, int cta, int ncta) {
   }
   // embedding rows, 16 bytes per thread, spread over the grid
   const int chunks = p.H / 8;
-  for (int i = cta * kThreads + threadIdx.x; i < p.M * chunks; i += ncta * kThreads) {
+  for (int i = cta * kCT + threadIdx.x; i < p.M * chunks; i += ncta * kCT) {
     const int m = i / chunks, c = i % chunks;
     const int tok = p.tokens[m];
     const bool ok = tok >= 0 && tok < p.vocab;
@@ -574,7 +818,7 @@ __device__ void attention_phase(const MegaParams& p, int layer, __nv_bfloat16* k
     __nv_bfloat16* kbase = kc_l + ((size_t)b * p.Hkv + hk) * (size_t)p.s_max * D;
     __nv_bfloat16* vbase = vc_l + ((size_t)b * p.Hkv + hk) * (size_t)p.s_max * D;
     const int R = G * T;
-    __syncthreads();  // shared tiles of the previous item are no longer read
+    cbar();  // shared tiles of the previous item are no longer read
 
     // (a) rotate this kv head's query rows into shared memory; the item that owns a block row's
     //     cache slot also rotates its K row and stores K and V there
@@ -597,10 +841,10 @@ __device__ void attention_phase(const MegaParams& p, int layer, __nv_bfloat16* k
         }
       }
     }
-    __syncthreads();  // block-level visibility of the K/V rows just stored and of q_s
+    cbar();  // block-level visibility of the K/V rows just stored and of q_s
 
     // (b) stage the K / V tile (zero beyond the end of the sequence)
-    for (int i = threadIdx.x; i < kKeyTile * (D / 8); i += kThreads) {
+    for (int i = threadIdx.x; i < kKeyTile * (D / 8); i += kCT) {
       const int key = i / (D / 8), ch = i % (D / 8);
       uint4 kv4 = make_uint4(0, 0, 0, 0), vv4 = make_uint4(0, 0, 0, 0);
       if (key_begin + key < key_end) {
@@ -610,7 +854,7 @@ __device__ void attention_phase(const MegaParams& p, int layer, __nv_bfloat16* k
       *reinterpret_cast<uint4*>(k_s + key * kStride + ch * 8) = kv4;
       *reinterpret_cast<uint4*>(v_s + key * kStride + ch * 8) = vv4;
     }
-    __syncthreads();
+    cbar();
 
     // (c) one warp per 16 query rows
     const int row_tiles = (R + 15) / 16;
@@ -637,8 +881,8 @@ __device__ void attention_phase(const MegaParams& p, int layer, __nv_bfloat16* k
 #pragma unroll
         for (int kd = 0; kd < kDSteps; ++kd) {
           const __nv_bfloat16* kr = k_s + (8 * j + g) * kStride + kd * 16 + 2 * t;
-          mma16816(s[j], qf[kd][0], qf[kd][1], qf[kd][2], qf[kd][3], *reinterpret_cast<const uint32_t*>(kr),
-                   *reinterpret_cast<const uint32_t*>(kr + 8));
+          mma16816_bf16(s[j], qf[kd][0], qf[kd][1], qf[kd][2], qf[kd][3], *reinterpret_cast<const uint32_t*>(kr),
+                        *reinterpret_cast<const uint32_t*>(kr + 8));
         }
       }
       float row_max[2] = {-INFINITY, -INFINITY}, row_sum[2] = {0.f, 0.f};
@@ -696,10 +940,10 @@ __device__ void attention_phase(const MegaParams& p, int layer, __nv_bfloat16* k
             const int mat = lane >> 3, r = lane & 7;
             ldmatrix_x4_trans(b0, b1, b2, b3, v_s + (kk * 16 + (mat & 1) * 8 + r) * kStride + half * (D / 2) +
                                                   dt * 16 + (mat >> 1) * 8);
-            mma16816(o[2 * dt], ah[0], ah[1], ah[2], ah[3], b0, b1);
-            mma16816(o[2 * dt], al[0], al[1], al[2], al[3], b0, b1);
-            mma16816(o[2 * dt + 1], ah[0], ah[1], ah[2], ah[3], b2, b3);
-            mma16816(o[2 * dt + 1], al[0], al[1], al[2], al[3], b2, b3);
+            mma16816_bf16(o[2 * dt], ah[0], ah[1], ah[2], ah[3], b0, b1);
+            mma16816_bf16(o[2 * dt], al[0], al[1], al[2], al[3], b0, b1);
+            mma16816_bf16(o[2 * dt + 1], ah[0], ah[1], ah[2], ah[3], b2, b3);
+            mma16816_bf16(o[2 * dt + 1], al[0], al[1], al[2], al[3], b2, b3);
           }
         }
 #pragma unroll
@@ -792,7 +1036,7 @@ __device__ void accept_phase(const MegaParams& p, int ncta) {
     }
     if (lane == 0) p.top1[m] = bi == 0x7fffffff ? 0 : bi;
   }
-  __syncthreads();
+  cbar();
   if ((int)threadIdx.x < p.B) {
     const int b = threadIdx.x, base = b * p.T_max;
     if (!p.bi.valid[b]) {
@@ -826,60 +1070,125 @@ template <bool W_INT8, int D>
 __global__ void __launch_bounds__(kThreads, 1) verify_megakernel(const MegaParams p) {
   extern __shared__ __align__(128) unsigned char smem[];
   const int cta = blockIdx.x, ncta = gridDim.x;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  unsigned char* ring = smem + (size_t)warp * kStages * kStageBytes;
+  const int warp = threadIdx.x >> 5;
   unsigned char* uni = smem + kRingBytes;
   float* red = reinterpret_cast<float*>(uni);
   __nv_bfloat16* k_s = reinterpret_cast<__nv_bfloat16*>(uni);
   __nv_bfloat16* v_s = reinterpret_cast<__nv_bfloat16*>(uni + kKvTileBytes);
   __nv_bfloat16* q_s = reinterpret_cast<__nv_bfloat16*>(uni + kUnionBytes);
   float* misc = reinterpret_cast<float*>(uni + kUnionBytes + kQTileBytes);
-  int* abort_flag = reinterpret_cast<int*>(misc + 200);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + kMiscAbort);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<unsigned char*>(misc) + kMiscBarBytes);
+  Pipe pipe{smem, bars, bars + kStages, abort_flag, p.status};
 
-  if (threadIdx.x == 0) *abort_flag = 0;
+  if (threadIdx.x == 0) {
+    *abort_flag = 0;
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(pipe.full + s, 1);     // the producer's arrive.expect_tx; the bytes complete the phase
+      mbar_init(pipe.empty + s, NW);   // one arrival per consumer warp
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+  }
   if (threadIdx.x < 8) {  // running arg-max of this CTA
-    misc[128 + threadIdx.x] = -INFINITY;
-    reinterpret_cast<int*>(misc + 128 + 8)[threadIdx.x] = 0x7fffffff;
+    misc[kMiscRunV + threadIdx.x] = -INFINITY;
+    reinterpret_cast<int*>(misc + kMiscRunI)[threadIdx.x] = 0x7fffffff;
   }
   __syncthreads();
 
-  // start the weight stream: the first kStages-1 stages of this warp's schedule
-  Producer<W_INT8> prod;
-  prod.init(p.jobs, p.n_jobs, cta, ncta, warp, lane);
-  unsigned cstage = 0;
-#pragma unroll 1
-  for (int s = 0; s < kStages - 1; ++s) prod.fetch(ring + s * kStageBytes);
+  if (warp >= NW) {  // the weight stream; hands most of its registers to the consumer warps
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;\n" ::"n"(kProducerRegs));
+    if (warp == NW) producer_loop<W_INT8>(p, pipe, cta, ncta);
+    return;
+  }
+  asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;\n" ::"n"(kConsumerRegs));
 
+  int slot = 0;
+  uint32_t phase = 0;
   GridSync gs{p.barrier, p.status, (unsigned)ncta, 0u, abort_flag};
   bool ok = true;
+#ifdef QUASAR_PHASE_TIMER
+  int mark_n = 0;
+#endif
 
+  PHASE_MARK();
   prep_phase(p, cta, ncta);
+  PHASE_MARK();
   ok = gs.sync();
-  for (int l = 0; l < p.L && ok; ++l) {
-    GemmPhase<W_INT8>::run(p, 4 * l + 0, prod, ring, cstage, red, misc, cta, ncta);
+  PHASE_MARK();
+  // the GEMMs of the pass in order (qkv, o, gate+up, down per layer, then the LM head); attention follows every qkv
+  for (int job = 0; job < p.n_jobs && ok; ++job) {
+    if (!(ok = GemmPhase<W_INT8>::run(p, job, pipe, slot, phase, red, misc, cta, ncta))) break;
+    PHASE_MARK();
+    if (job == p.n_jobs - 1) break;   // the LM head is followed by the candidate exchange below
     if (!(ok = gs.sync())) break;
-    attention_phase<D>(p, l, k_s, v_s, q_s, cta, ncta);
-    if (!(ok = gs.sync())) break;
-    merge_phase<D>(p, cta, ncta);
-    if (!(ok = gs.sync())) break;
-    GemmPhase<W_INT8>::run(p, 4 * l + 1, prod, ring, cstage, red, misc, cta, ncta);
-    if (!(ok = gs.sync())) break;
-    GemmPhase<W_INT8>::run(p, 4 * l + 2, prod, ring, cstage, red, misc, cta, ncta);
-    if (!(ok = gs.sync())) break;
-    GemmPhase<W_INT8>::run(p, 4 * l + 3, prod, ring, cstage, red, misc, cta, ncta);
-    if (!(ok = gs.sync())) break;
+    PHASE_MARK();
+    if ((job & 3) == 0) {
+      attention_phase<D>(p, job >> 2, k_s, v_s, q_s, cta, ncta);
+      PHASE_MARK();
+      if (!(ok = gs.sync())) break;
+      PHASE_MARK();
+      merge_phase<D>(p, cta, ncta);
+      PHASE_MARK();
+      if (!(ok = gs.sync())) break;
+      PHASE_MARK();
+    }
   }
   if (ok) {
-    GemmPhase<W_INT8>::run(p, 4 * p.L, prod, ring, cstage, red, misc, cta, ncta);
-    __syncthreads();
+    cbar();
     if (threadIdx.x < 8) {
-      p.cand_val[(size_t)cta * 8 + threadIdx.x] = misc[128 + threadIdx.x];
-      p.cand_idx[(size_t)cta * 8 + threadIdx.x] = reinterpret_cast<int*>(misc + 128 + 8)[threadIdx.x];
+      p.cand_val[(size_t)cta * 8 + threadIdx.x] = misc[kMiscRunV + threadIdx.x];
+      p.cand_idx[(size_t)cta * 8 + threadIdx.x] = reinterpret_cast<int*>(misc + kMiscRunI)[threadIdx.x];
     }
     ok = gs.sync();
+    PHASE_MARK();
     if (ok && cta == 0) accept_phase(p, ncta);
   }
-  cp_async_wait<0>();  // nothing of ours is in flight when the CTA leaves
+#ifdef QUASAR_PHASE_TIMER
+  if (threadIdx.x == 0) g_phase_n[blockIdx.x] = mark_n;
+#endif
+  if (!ok && threadIdx.x == 0) *abort_flag = 1;  // tells the producer to stop issuing
+}
+
+// ---- model creation: permute every CTA's row range into its consumption order ------------------
+// One thread block per (tile, CTA).  The destination has the size of the source and every CTA's
+// range starts where its rows start in the source; inside the range the blocks follow the
+// schedule above.  int8 weights get their sign bits flipped (see u8x4_to_f16x4).
+template <bool W_INT8>
+__global__ void __launch_bounds__(256) repack_kernel(const unsigned char* __restrict__ w, unsigned char* __restrict__ wp,
+                                                     int N, int K, int kind, int ncta) {
+  constexpr int kElemBytes = W_INT8 ? 1 : 2;
+  constexpr int kChunkBytes = kChunk * kElemBytes;
+  const int cta = blockIdx.y, tile_g = blockIdx.x;
+  JobView v;
+  job_split(kind, N, K, cta, ncta, v);
+  if (tile_g >= v.tiles) return;
+  const int mult = kind == kJobGateUp ? 2 : 1;
+  const int tg = tile_g / GT, tile = tile_g % GT;
+  const int gt = min(GT, v.tiles - tg * GT);
+  int rows_in_group = 0;
+  for (int i = 0; i < gt; ++i) rows_in_group += tile_rows(v, tg * GT + i);
+  const size_t rows_before_group = (size_t)mult * tg * GT * v.rows_per_tile;   // every earlier tile is full
+  const size_t rows_before_in_group = (size_t)mult * tile * v.rows_per_tile;
+  const int nr = tile_rows(v, tile_g);
+  const size_t kbytes = (size_t)K * kElemBytes;
+  unsigned char* region = wp + (size_t)mult * v.u0 * kbytes;
+  for (int kc = 0; kc < v.nchunks; ++kc) {
+    const int cb = (int)min((size_t)kChunkBytes, kbytes - (size_t)kc * kChunkBytes);
+    const size_t chunk_off = rows_before_group * kbytes + (size_t)rows_in_group * kc * kChunkBytes + rows_before_in_group * cb;
+    for (int b0 = 0; b0 < cb; b0 += kRowBytes) {
+      const int pb = min(kRowBytes, cb - b0);
+      unsigned char* blk = region + chunk_off + (size_t)nr * b0;
+      const int per_row = pb / 16;
+      for (int idx = threadIdx.x; idx < nr * per_row; idx += blockDim.x) {
+        const int row = idx / per_row, ch = idx % per_row;
+        const int n = block_row_to_global(v, tile_g, row);
+        uint4 val = __ldg(reinterpret_cast<const uint4*>(w + (size_t)n * kbytes + (size_t)kc * kChunkBytes + b0) + ch);
+        if (W_INT8) { val.x ^= 0x80808080u; val.y ^= 0x80808080u; val.z ^= 0x80808080u; val.w ^= 0x80808080u; }
+        const int dch = (pb & 127) == 0 ? ch ^ ((row & 1) << 2) : ch;
+        *reinterpret_cast<uint4*>(blk + (size_t)row * pb + dch * 16) = val;
+      }
+    }
+  }
 }
 
 template <bool W_INT8, int D>
@@ -898,6 +1207,37 @@ int launch_variant(const MegaParams& p, int ncta, cudaStream_t stream) {
 }
 
 }  // namespace
+
+#ifdef QUASAR_PHASE_TIMER
+extern "C" int quasar_debug_phase_marks(long long* clk_host, int* n_host) {
+  if (cudaMemcpyFromSymbol(clk_host, g_phase_clk, sizeof(long long) * 160 * kMaxMarks) != cudaSuccess) return -1;
+  if (cudaMemcpyFromSymbol(n_host, g_phase_n, sizeof(int) * 160) != cudaSuccess) return -1;
+  return kMaxMarks;
+}
+extern "C" int quasar_debug_gemm_clocks(long long* host, int reset) {
+  if (cudaMemcpyFromSymbol(host, g_gemm_clk, sizeof(long long) * 160 * 4) != cudaSuccess) return -1;
+  if (reset) {
+    static long long zero[160 * 4];
+    if (cudaMemcpyToSymbol(g_gemm_clk, zero, sizeof(zero)) != cudaSuccess) return -1;
+  }
+  return 0;
+}
+#endif
+
+int launch_repack(const void* w, void* wp, int N, int K, int kind, int weight_dtype, int ncta, cudaStream_t stream) {
+  const int units = kind == kJobGateUp ? N / 2 : N;
+  const int rpt = kind == kJobGateUp ? 8 : 16;
+  const int max_units = (units + ncta - 1) / ncta;
+  dim3 grid((max_units + rpt - 1) / rpt, ncta);
+  if (weight_dtype == QUASAR_W_INT8)
+    repack_kernel<true><<<grid, 256, 0, stream>>>(reinterpret_cast<const unsigned char*>(w),
+                                                  reinterpret_cast<unsigned char*>(wp), N, K, kind, ncta);
+  else
+    repack_kernel<false><<<grid, 256, 0, stream>>>(reinterpret_cast<const unsigned char*>(w),
+                                                   reinterpret_cast<unsigned char*>(wp), N, K, kind, ncta);
+  QUASAR_LAUNCH_CHECK();
+  return QUASAR_OK;
+}
 
 bool mega_supported(int M, int T_max, int Hq, int Hkv, int D) {
   return M <= 8 && (Hq / Hkv) * T_max <= kMaxRowsAttn && (D == 64 || D == 128);

@@ -11,7 +11,7 @@ enum MegaJobKind { kJobQkv = 0, kJobO = 1, kJobGateUp = 2, kJobDown = 3, kJobLm 
 
 // One GEMM of the pass, in execution order: per layer qkv, o, gate+up, down; then the LM head.
 struct MegaJob {
-  const void* w;               // [N][K] int8 or bf16
+  const void* wp;              // [N][K] int8 or bf16, every CTA's row range permuted into its consumption order
   const float* delta;          // [N] or nullptr
   const __nv_bfloat16* gain;   // RMSNorm gain fused into the operand load, or nullptr
   int N, K, kind, pad;
@@ -49,6 +49,8 @@ bool mega_supported(int M, int T_max, int Hq, int Hkv, int D);
 int mega_attn_nchunk(int s_max);
 int mega_attn_rpad(int T_max, int Hq, int Hkv);
 int mega_grid_size(int weight_dtype, int D, int* ncta_out);
+// Writes the permuted copy of one weight matrix for a grid of `ncta` CTAs (same size as the source).
+int launch_repack(const void* w, void* wp, int N, int K, int kind, int weight_dtype, int ncta, cudaStream_t stream);
 int launch_verify_mega(const MegaParams& p, int weight_dtype, int D, int ncta, cudaStream_t stream);
 
 }  // namespace quasar
