@@ -88,6 +88,32 @@ int quasar_linear(const void* x, const void* w, const float* delta, int32_t weig
                   size_t workspace_bytes, void* stream);
 
 /* ------------------------------------------------------------------------
+ * quasar_linear for callers that may not allocate device memory.  (The paper has no
+ * counterpart: this is a convenience of the library, not a step of the method.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits, for instance a plug-in
+ * inside a host application that owns the whole memory pool and hands out only the input
+ * and output tensors, or a latency-critical loop that must not touch the allocator (an
+ * allocation can synchronise the device).  Such a caller has no workspace to pass.
+ *
+ * Same arithmetic, arguments and result as quasar_linear, minus the workspace: the scratch
+ * of the split-K reduction lives in a fixed array of quasar_linear_static_scratch_bytes()
+ * (4 MiB) inside the library, which every GPU that loads the library holds until the
+ * process exits.  The call itself allocates and frees nothing.
+ *  - Shapes whose scratch would exceed the array are refused with QUASAR_ERR_CAPACITY
+ *    (the message gives both sizes); use quasar_linear for those.
+ *  - The first call on a device looks up the array's device address (with that device
+ *    current); make that first call outside any stream capture.
+ *  - All calls on a device share the one array, and it keeps the previous call's contents
+ *    (the part that must start at zero is cleared on `stream` by every call).  Two calls
+ *    that may overlap on the GPU - different streams without an ordering between them -
+ *    race on it; issue them on one stream or order them with events.
+ * ---------------------------------------------------------------------- */
+size_t quasar_linear_static_scratch_bytes(void);
+int quasar_linear_static(const void* x, const void* w, const float* delta, int32_t weight_dtype, int64_t M, int64_t N,
+                         int64_t K, void* y, int32_t y_is_f32, const void* residual, void* stream);
+
+/* ------------------------------------------------------------------------
  * Model description.  The paper fixes only the linear layers; the rest of the
  * decoder layer (Section 3.3: "non-linear layers" stay in high precision) is a
  * pre-norm decoder: RMSNorm (y = x * rsqrt(mean(x^2) + eps) * g), optional

@@ -62,6 +62,8 @@ SIGNATURES = {
     "quasar_quantize": (C.c_int, [_vp, _i64, _i64, _vp, _vp, _vp]),
     "quasar_linear_workspace_bytes": (C.c_int, [_i64, _i64, _i64, C.POINTER(_sz)]),
     "quasar_linear": (C.c_int, [_vp, _vp, _vp, _i32, _i64, _i64, _i64, _vp, _i32, _vp, _vp, _sz, _vp]),
+    "quasar_linear_static_scratch_bytes": (_sz, []),
+    "quasar_linear_static": (C.c_int, [_vp, _vp, _vp, _i32, _i64, _i64, _i64, _vp, _i32, _vp, _vp]),
     "quasar_model_create": (C.c_int, [C.POINTER(Config), C.POINTER(Weights), C.POINTER(_vp)]),
     "quasar_model_destroy": (C.c_int, [_vp]),
     "quasar_workspace_bytes": (C.c_int, [_vp, _i32, _i32, C.POINTER(_sz)]),
@@ -139,6 +141,24 @@ def quasar_linear(x: torch.Tensor, w: torch.Tensor, delta: Optional[torch.Tensor
         workspace = torch.zeros(max(quasar_linear_workspace_bytes(m, n, k), 16), dtype=torch.uint8, device=x.device)
     _check(lib().quasar_linear(_ptr(x), _ptr(w), _ptr(delta), wd, m, n, k, _ptr(out), 1 if out_f32 else 0,
                                _ptr(residual), _ptr(workspace), workspace.numel(), _stream()))
+    return out
+
+
+def quasar_linear_static_scratch_bytes() -> int:
+    return int(lib().quasar_linear_static_scratch_bytes())
+
+
+def quasar_linear_static(x: torch.Tensor, w: torch.Tensor, delta: Optional[torch.Tensor], out: torch.Tensor,
+                         residual=None) -> torch.Tensor:
+    """quasar_linear without a workspace argument: the library's built-in scratch array is used and
+    nothing is allocated by the call (the caller supplies `out`: bf16 or fp32 [M][N])."""
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.is_contiguous() and w.is_contiguous() and out.is_contiguous()
+    m, k = x.shape
+    n = w.shape[0]
+    assert tuple(out.shape) == (m, n) and out.dtype in (torch.float32, torch.bfloat16)
+    wd = QUASAR_W_INT8 if w.dtype == torch.int8 else QUASAR_W_BF16
+    _check(lib().quasar_linear_static(_ptr(x), _ptr(w), _ptr(delta), wd, m, n, k, _ptr(out),
+                                      1 if out.dtype == torch.float32 else 0, _ptr(residual), _stream()))
     return out
 
 

@@ -345,6 +345,20 @@ int quasar_linear(const void* x, const void* w, const float* delta, int32_t weig
                        (cudaStream_t)stream);
 }
 
+int quasar_linear_static(const void* x, const void* w, const float* delta, int32_t weight_dtype, int64_t M, int64_t N,
+                         int64_t K, void* y, int32_t y_is_f32, const void* residual, void* stream) {
+  if (weight_dtype != QUASAR_W_INT8 && weight_dtype != QUASAR_W_BF16) { set_error("linear_static: weight_dtype %d", weight_dtype); return QUASAR_ERR_INVALID_ARG; }
+  REQUIRE_PTR(x, "x");
+  REQUIRE_PTR(w, "w");
+  REQUIRE_PTR(y, "y");
+  if (weight_dtype == QUASAR_W_INT8) REQUIRE_PTR(delta, "delta");
+  if (residual && !aligned16(residual)) { set_error("residual is not 16-byte aligned"); return QUASAR_ERR_ALIGN; }
+  return launch_linear_static(reinterpret_cast<const __nv_bfloat16*>(x), w, delta, weight_dtype, M, N, K, y,
+                              y_is_f32 != 0, reinterpret_cast<const __nv_bfloat16*>(residual), (cudaStream_t)stream);
+}
+
+size_t quasar_linear_static_scratch_bytes(void) { return linear_static_scratch_bytes(); }
+
 int quasar_model_create(const quasar_config* cfg, const quasar_weights* w, quasar_model** out) {
   if (cfg == nullptr || w == nullptr || out == nullptr) { set_error("model_create: NULL argument"); return QUASAR_ERR_INVALID_ARG; }
   *out = nullptr;

@@ -44,6 +44,12 @@ int launch_linear(const __nv_bfloat16* x, const void* w, const float* delta, int
                   int64_t K, void* y, bool y_is_f32, const __nv_bfloat16* residual, void* workspace,
                   size_t workspace_bytes, cudaStream_t stream);
 
+// The same launch with the split-K scratch taken from a fixed array inside the library.
+size_t linear_static_scratch_bytes();
+int launch_linear_static(const __nv_bfloat16* x, const void* w, const float* delta, int weight_dtype, int64_t M,
+                         int64_t N, int64_t K, void* y, bool y_is_f32, const __nv_bfloat16* residual,
+                         cudaStream_t stream);
+
 // Per-call description of the draft blocks, derived on the device from tokens / parents / block_len.
 struct BlockInfo {
   uint64_t* anc;    // [B*T_max] bit j set: block row j is row i itself or an ancestor of it

@@ -14,6 +14,8 @@
 // Work split: a CTA of 4 warps owns 64 output channels x one k-range; k-ranges of one
 // channel block are reduced in a FIXED order by the last CTA to arrive (fp32 partials in
 // the workspace, a self-resetting arrival counter), so results are run-to-run identical.
+#include <mutex>
+
 #include "common.cuh"
 
 namespace quasar {
@@ -324,6 +326,57 @@ int launch_linear(const __nv_bfloat16* x, const void* w, const float* delta, int
     if (rc != QUASAR_OK) return rc;
   }
   return QUASAR_OK;
+}
+
+// ---- the same linear layer with its scratch inside the library ------------------------------------
+// Scratch of the split-K reduction for callers that cannot hand over a workspace: a fixed array in
+// device memory that every GPU loading the library holds until the process exits.
+constexpr size_t kStaticScratchBytes = 4u << 20;
+static __device__ __align__(256) unsigned char g_linear_scratch[kStaticScratchBytes];
+
+size_t linear_static_scratch_bytes() { return kStaticScratchBytes; }
+
+int launch_linear_static(const __nv_bfloat16* x, const void* w, const float* delta, int weight_dtype, int64_t M,
+                         int64_t N, int64_t K, void* y, bool y_is_f32, const __nv_bfloat16* residual,
+                         cudaStream_t stream) {
+  // In host code the array's name only stands for the symbol; its device address is looked up once per
+  // device (with that device current) and kept.
+  constexpr int kMaxDevices = 64;
+  static void* scratch_of_device[kMaxDevices] = {};
+  static std::mutex mu;
+  int dev = 0;
+  QUASAR_CUDA_CHECK(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) {
+    set_error("linear_static: device ordinal %d not supported (at most %d devices)", dev, kMaxDevices);
+    return QUASAR_ERR_CAPACITY;
+  }
+  void* scratch = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(mu);
+    if (scratch_of_device[dev] == nullptr) {
+      void* ptr = nullptr;
+      QUASAR_CUDA_CHECK(cudaGetSymbolAddress(&ptr, g_linear_scratch));
+      scratch_of_device[dev] = ptr;
+    }
+    scratch = scratch_of_device[dev];
+  }
+  if (M <= 0 || N <= 0 || K <= 0 || (K % 16) != 0 || N > 0x7fffffff || K > 0x7fffffff) {
+    set_error("linear_static: unsupported sizes M=%lld N=%lld K=%lld (K must be a multiple of 16)", (long long)M,
+              (long long)N, (long long)K);
+    return QUASAR_ERR_SHAPE;
+  }
+  const size_t need = linear_workspace_bytes(M, N, K);
+  if (need > kStaticScratchBytes) {
+    set_error("linear_static: M=%lld N=%lld K=%lld needs %zu bytes of scratch, the built-in array holds %zu; "
+              "use quasar_linear with a workspace",
+              (long long)M, (long long)N, (long long)K, need, kStaticScratchBytes);
+    return QUASAR_ERR_CAPACITY;
+  }
+  // The arrival counters must start at zero; the array keeps whatever the last call left in it.
+  const SplitPlan p = plan_split(N, K);
+  const size_t counters = ((size_t)p.nblocks * sizeof(int) + 255) / 256 * 256;
+  QUASAR_CUDA_CHECK(cudaMemsetAsync(scratch, 0, counters, stream));
+  return launch_linear(x, w, delta, weight_dtype, M, N, K, y, y_is_f32, residual, scratch, kStaticScratchBytes, stream);
 }
 
 }  // namespace quasar
