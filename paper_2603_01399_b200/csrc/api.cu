@@ -1,5 +1,6 @@
 // C ABI of the library: argument checks, the model object, and the sequence of launches
 // that makes up one verification pass (Section 3.1 "Verification", Section 3.3).
+#include <math.h>
 #include <stdarg.h>
 #include <stdio.h>
 #include <string.h>
@@ -64,7 +65,7 @@ size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
 
 // Layout of the verify workspace; every offset is a multiple of 256 bytes.
 struct Workspace {
-  size_t x, h, qkv, attn, gu, act, logits, top1, anc, depth, valid, lin, att, cand, barrier, total;
+  size_t x, h, qkv, attn, gu, act, logits, top1, anc, depth, valid, lin, att, cand, ss_part, amax, barrier, total;
   size_t lin_bytes, att_bytes;
 };
 
@@ -107,6 +108,8 @@ Workspace layout(const quasar_config& c, int B, int T_max, int s_max) {
   }
   w.att = take(w.att_bytes);
   w.cand = take((size_t)kMaxGrid * 8 * 2 * sizeof(float));
+  w.ss_part = take((size_t)kMaxGrid * 8 * sizeof(float));
+  w.amax = take((size_t)(4 * c.n_layers + 1) * 8 * sizeof(unsigned));
   w.barrier = take(256);
   w.total = off;
   return w;
@@ -252,6 +255,8 @@ int verify_impl(quasar_model* m, const quasar_kv* kv, const int32_t* tokens, con
     p.ml_part = p.o_part + rows * D;
     p.cand_val = reinterpret_cast<float*>(wsp + ws.cand);
     p.cand_idx = reinterpret_cast<int*>(wsp + ws.cand + (size_t)kMaxGrid * 8 * sizeof(float));
+    p.ss_part = reinterpret_cast<float*>(wsp + ws.ss_part);
+    p.amax_buf = reinterpret_cast<unsigned*>(wsp + ws.amax);
     p.barrier = reinterpret_cast<unsigned*>(wsp + ws.barrier);
     p.accept_len = accept_len; p.bonus = bonus; p.accept_path = accept_path; p.status = status;
     QUASAR_CUDA_CHECK(cudaMemsetAsync(p.barrier, 0, 256, stream));
@@ -419,22 +424,50 @@ int quasar_model_create(const quasar_config* cfg, const quasar_weights* w, quasa
     for (int l = 0; l < cfg->n_layers; ++l) {
       const quasar_layer_weights& L = m->layers[l];
       jobs.push_back({nullptr, q ? L.qkv_delta : nullptr, reinterpret_cast<const __nv_bfloat16*>(L.attn_norm), qkv_w,
-                      cfg->hidden, kJobQkv, 0});
+                      cfg->hidden, kJobQkv, 1.f});
       src.push_back(L.qkv_w);
-      jobs.push_back({nullptr, q ? L.o_delta : nullptr, nullptr, cfg->hidden, cfg->n_q_heads * cfg->head_dim, kJobO, 0});
+      jobs.push_back({nullptr, q ? L.o_delta : nullptr, nullptr, cfg->hidden, cfg->n_q_heads * cfg->head_dim, kJobO, 1.f});
       src.push_back(L.o_w);
       jobs.push_back({nullptr, q ? L.gateup_delta : nullptr, reinterpret_cast<const __nv_bfloat16*>(L.mlp_norm),
-                      2 * cfg->ffn, cfg->hidden, kJobGateUp, 0});
+                      2 * cfg->ffn, cfg->hidden, kJobGateUp, 1.f});
       src.push_back(L.gateup_w);
-      jobs.push_back({nullptr, q ? L.down_delta : nullptr, nullptr, cfg->hidden, cfg->ffn, kJobDown, 0});
+      jobs.push_back({nullptr, q ? L.down_delta : nullptr, nullptr, cfg->hidden, cfg->ffn, kJobDown, 1.f});
       src.push_back(L.down_w);
       mls.push_back({reinterpret_cast<const __nv_bfloat16*>(cfg->qk_norm ? L.q_norm : nullptr),
                      reinterpret_cast<const __nv_bfloat16*>(cfg->qk_norm ? L.k_norm : nullptr)});
     }
     jobs.push_back({nullptr, q ? w->lm_delta : nullptr, reinterpret_cast<const __nv_bfloat16*>(w->final_norm),
-                    cfg->vocab, cfg->hidden, kJobLm, 0});
+                    cfg->vocab, cfg->hidden, kJobLm, 1.f});
     src.push_back(w->lm_w);
     if (mls.empty()) mls.push_back({nullptr, nullptr});
+    // Normed GEMMs feed h = x * r * gain with |x r| <= sqrt(K): a static power-of-two scale keeps h
+    // inside the fp16 range whatever the activations are (1 unless a gain is in the hundreds).
+    {
+      std::vector<uint16_t> gh;
+      for (auto& j : jobs) {
+        if (j.gain == nullptr) continue;
+        gh.resize(j.K);
+        if (cudaMemcpy(gh.data(), j.gain, (size_t)j.K * 2, cudaMemcpyDeviceToHost) != cudaSuccess) {
+          set_error("model_create: reading a norm gain failed: %s", cudaGetErrorString(cudaGetLastError()));
+          quasar_model_destroy(m);
+          return QUASAR_ERR_CUDA;
+        }
+        float gmax = 0.f;
+        for (int k = 0; k < j.K; ++k) {
+          const uint32_t bits = (uint32_t)gh[k] << 16;
+          float f;
+          memcpy(&f, &bits, 4);
+          f = f < 0 ? -f : f;
+          if (f > gmax) gmax = f;
+        }
+        const float bound = gmax * sqrtf((float)j.K) * 1.01f;
+        if (bound > 32768.f && bound < 3.0e38f) {
+          int e;
+          (void)frexpf(bound, &e);
+          j.xscale = ldexpf(1.f, 15 - e);
+        }
+      }
+    }
     const size_t esz = q ? 1 : 2;
     size_t total = 0;
     std::vector<size_t> offs;

@@ -44,9 +44,7 @@ namespace {
 
 constexpr int NW = kMegaWarps;             // consumer warps per CTA
 constexpr int kCT = NW * 32;               // consumer threads
-constexpr int kThreads = kCT + 128;        // + the producer's warp group (one of its warps issues the copies)
-constexpr int kConsumerRegs = 112;         // registers per thread after the split (setmaxnreg): 16 consumer warps
-constexpr int kProducerRegs = 40;          // ... and the 4 warps of the producer's group
+constexpr int kThreads = kCT + 32;         // + the producer warp (17 warps: 5 on one SM sub-partition, so 96 registers per thread)
 constexpr int kRowBytes = 1024;            // bytes of one weight row per stage
 constexpr int kStageBytes = 16 * kRowBytes;  // 16 weight rows
 constexpr int kStages = 10;                // ring depth (160 KB of weights in flight per CTA)
@@ -69,9 +67,9 @@ constexpr int kSmemBytes = kRingBytes + kUnionBytes + kQTileBytes + kMiscBytes;
 static_assert(kSmemBytes <= 227 * 1024, "shared memory budget of one SM");
 
 // misc region (floats): [0,128) per-warp row sums, [128,136) running arg-max values, [136,144) its
-// indices, [144,152) 1/scale of the operand rows, [200] abort flag, [256,512) candidates / per-warp
+// indices, [144,152) 1/scale of the operand rows, [152,184) per-tile sums of squares, [200] abort flag, [256,512) candidates / per-warp
 // row maxima, byte 1536.. the mbarriers.
-constexpr int kMiscRowSum = 0, kMiscRunV = 128, kMiscRunI = 136, kMiscInvScale = 144, kMiscAbort = 200,
+constexpr int kMiscRowSum = 0, kMiscRunV = 128, kMiscRunI = 136, kMiscInvScale = 144, kMiscPart = 152, kMiscAbort = 200,
               kMiscCand = 256, kMiscBarBytes = 1536;
 
 __device__ __forceinline__ void mma16816_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
@@ -100,8 +98,6 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t& r0, uint32_t& r1, ui
 // Four weight bytes -> four fp16 (exact).  The repacked bytes hold u = w + 128 in [1, 255]
 // (sign bit flipped); placed under the high byte 0x64, u reads 1024 + u as fp16 (the spacing of
 // fp16 in [1024, 2048) is 1), and subtracting 1152 leaves w.  lo = bytes 0,1; hi = bytes 2,3.
-constexpr float kWeightUnit = 1.f;
-constexpr float kWeightOffset = 0.f;
 __device__ __forceinline__ void u8x4_to_f16x4(uint32_t u, uint32_t& lo, uint32_t& hi) {
   const uint32_t l = __byte_perm(u, 0x64646464u, 0x4140);
   const uint32_t h = __byte_perm(u, 0x64646464u, 0x4342);
@@ -145,7 +141,9 @@ __device__ __forceinline__ unsigned long long now_ns() {
 constexpr int kMaxMarks = 640;
 __device__ long long g_phase_clk[160][kMaxMarks];
 __device__ int g_phase_n[160];
-__device__ long long g_gemm_clk[160][4];   // warp 0 of every CTA: cycles waiting for stages, in stats, in epilogues, in GEMM phases
+__device__ long long g_gemm_clk[160][8];
+__device__ int g_clk_on_dummy;
+#define g_clk_on (job == p.n_jobs - 1)   // warp 0 of every CTA: cycles waiting for stages, in stats, in epilogues, in GEMM phases
 #define PHASE_MARK()                                                                         \
   do {                                                                                       \
     if (threadIdx.x == 0 && mark_n < kMaxMarks) g_phase_clk[blockIdx.x][mark_n++] = clock64(); \
@@ -155,7 +153,7 @@ __device__ long long g_gemm_clk[160][4];   // warp 0 of every CTA: cycles waitin
   do {                                                              \
     const long long c0__ = clock64();                               \
     expr;                                                           \
-    if (threadIdx.x == 0) g_gemm_clk[blockIdx.x][i] += clock64() - c0__; \
+    if (threadIdx.x == 0 && g_clk_on) g_gemm_clk[blockIdx.x][i] += clock64() - c0__; \
   } while (0)
 #else
 #define GEMM_CLK(i, expr) do { expr; } while (0)
@@ -371,81 +369,46 @@ __device__ __forceinline__ int x_index(int i, int kbase, int warp, int t) {
   return W_INT8 ? (kbase + (i >> 1) * 1024 + warp * 64 + t * 16 + (i & 1) * 8) : (kbase + i * 512 + warp * 32 + t * 8);
 }
 
+// The <= 8 operand rows of this warp's share of chunk `kbase`, ready for the MMA.  Normed GEMMs
+// (gain != null): h = bf16(x * r * gain), the RMSNorm output rounded where the decoder layer rounds
+// it.  int8 weights: the value is then multiplied by the row's power-of-two scale and converted to
+// fp16 (exact unless the scaled value falls below the fp16 normal range).
 template <bool W_INT8>
-__device__ __forceinline__ void load_x_raw(uint4 (&xr)[kXr], const __nv_bfloat16* src, int ld, int M, int K, int kbase,
-                                           int warp, int g, int t) {
+__device__ __forceinline__ void load_operand(uint4 (&xr)[kXr], const __nv_bfloat16* src, int ld, int M, int K, int kbase,
+                                             const __nv_bfloat16* gain, float rnorm, float xscale, int warp, int g,
+                                             int t) {
+  uint4 gv[kXr];
 #pragma unroll
-  for (int i = 0; i < kXr; ++i) {
+  for (int i = 0; i < kXr; ++i) {   // all loads first: one round trip to L2
     const int k = x_index<W_INT8>(i, kbase, warp, t);
     xr[i] = make_uint4(0, 0, 0, 0);
-    if (g < M && k < K) xr[i] = __ldcg(reinterpret_cast<const uint4*>(src + (size_t)g * ld + k));
-  }
-}
-
-// per-row statistics of the raw operand: sum of squares and max |x * gain| (gain may be null)
-template <bool W_INT8>
-__device__ __forceinline__ void x_stats(const uint4 (&xr)[kXr], const __nv_bfloat16* gain, int K, int kbase, int warp,
-                                        int t, float& ss, float& amax) {
-#pragma unroll
-  for (int i = 0; i < kXr; ++i) {
-    const int k = x_index<W_INT8>(i, kbase, warp, t);
+    gv[i] = make_uint4(0, 0, 0, 0);
     if (k < K) {
-      uint4 gv = make_uint4(0x3f803f80u, 0x3f803f80u, 0x3f803f80u, 0x3f803f80u);  // bf16 ones
-      if (gain != nullptr) gv = __ldg(reinterpret_cast<const uint4*>(gain + k));
-      const __nv_bfloat162* xp = reinterpret_cast<const __nv_bfloat162*>(&xr[i]);
-      const __nv_bfloat162* gp = reinterpret_cast<const __nv_bfloat162*>(&gv);
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const float2 xf = __bfloat1622float2(xp[e]);
-        const float2 gf = __bfloat1622float2(gp[e]);
-        ss += xf.x * xf.x + xf.y * xf.y;
-        amax = fmaxf(amax, fmaxf(fabsf(xf.x * gf.x), fabsf(xf.y * gf.y)));
-      }
+      if (g < M) xr[i] = __ldcg(reinterpret_cast<const uint4*>(src + (size_t)g * ld + k));
+      if (gain != nullptr) gv[i] = __ldg(reinterpret_cast<const uint4*>(gain + k));
     }
   }
-}
-
-// h = bf16(x * r * gain) in place (the RMSNorm output, rounded where the decoder layer rounds it)
-template <bool W_INT8>
-__device__ __forceinline__ void apply_norm(uint4 (&xr)[kXr], const __nv_bfloat16* gain, float r, int K, int kbase,
-                                           int warp, int t) {
-#pragma unroll
-  for (int i = 0; i < kXr; ++i) {
-    const int k = x_index<W_INT8>(i, kbase, warp, t);
-    if (k < K) {
-      const uint4 gv = __ldg(reinterpret_cast<const uint4*>(gain + k));
-      const __nv_bfloat162* xp = reinterpret_cast<const __nv_bfloat162*>(&xr[i]);
-      const __nv_bfloat162* gp = reinterpret_cast<const __nv_bfloat162*>(&gv);
-      uint32_t o[4];
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const float2 xf = __bfloat1622float2(xp[e]);
-        const float2 gf = __bfloat1622float2(gp[e]);
-        o[e] = pack_bf16(xf.x * r * gf.x, xf.y * r * gf.y);
-      }
-      xr[i] = make_uint4(o[0], o[1], o[2], o[3]);
-    }
-  }
-}
-
-// bf16 -> fp16 in place after multiplying by the row's power-of-two scale (exact unless the
-// scaled value falls below the fp16 normal range).  Returns the sum of the fp16 values written
-// (the epilogue needs sum_k x_k to remove the weights' offset).
-__device__ __forceinline__ float to_f16(uint4 (&xr)[kXr], float scale) {
-  float sum = 0.f;
+  if (!W_INT8 && gain == nullptr) return;   // bf16 operand as stored
 #pragma unroll
   for (int i = 0; i < kXr; ++i) {
     uint32_t* w = reinterpret_cast<uint32_t*>(&xr[i]);
+    const __nv_bfloat162* gp = reinterpret_cast<const __nv_bfloat162*>(&gv[i]);
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
-      const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w[e]));
-      const __half2 h = __floats2half2_rn(f.x * scale, f.y * scale);
-      const float2 b = __half22float2(h);
-      sum += b.x + b.y;
-      w[e] = *reinterpret_cast<const uint32_t*>(&h);
+      float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w[e]));
+      if (gain != nullptr) {
+        const float2 gf = __bfloat1622float2(gp[e]);
+        f.x = bf16_round_f(f.x * rnorm * gf.x);
+        f.y = bf16_round_f(f.y * rnorm * gf.y);
+      }
+      if (W_INT8) {
+        const __half2 h = __floats2half2_rn(f.x * xscale, f.y * xscale);
+        w[e] = *reinterpret_cast<const uint32_t*>(&h);
+      } else {
+        w[e] = pack_bf16(f.x, f.y);
+      }
     }
   }
-  return sum;
 }
 
 // One stage = one block [rows][pb bytes].  MMA row g of the tile is block row ra, MMA row g + 8
@@ -491,9 +454,10 @@ struct GemmPhase {
   static constexpr int kElemBytes = W_INT8 ? 1 : 2;
   static constexpr int kStageElems = kRowBytes / kElemBytes;
   static constexpr int SPC = kChunk / kStageElems;   // stages per chunk: 4 (int8) or 8 (bf16)
+  static_assert(kCT == GT * 128, "one epilogue element per consumer thread and tile group");
 
   __device__ __forceinline__ static bool run(const MegaParams& p, int job, const Pipe& pipe, int& slot_io,
-                                          uint32_t& phase_io, float* red, float* misc, int cta, int ncta) {
+                                             uint32_t& phase_io, float* red, float* misc, int cta, int ncta) {
     int slot = slot_io;
     uint32_t phase = phase_io;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
@@ -501,193 +465,194 @@ struct GemmPhase {
     const MegaJob jb = p.jobs[job];
     const int M = p.M;
     const bool normed = jb.gain != nullptr;
+    const bool residual = jb.kind == kJobO || jb.kind == kJobDown;
     const __nv_bfloat16* xsrc = jb.kind == kJobO ? p.attn : (jb.kind == kJobDown ? p.act : p.x);
     const int ld = jb.K;
 
-    // Row statistics of the operand: the RMSNorm factor (normed GEMMs: the operand is
-    // h = x * r * gain) and, for the fp16 path, a power-of-two scale that keeps the row in range.
-    float rnorm = 1.f, xscale = 1.f;
-    float xsum = 0.f;   // this lane's share of sum_k x_k over the whole contraction (fp16 operand values)
-    uint4 xr[kXr];
-    bool have_x = false;
+    // Per-row factors of the operand, computed by every warp for itself (no CTA barrier, one round
+    // trip to L2).  Normed GEMMs: the RMSNorm factor from the per-CTA sums of squares that the phase
+    // which wrote x left behind, added in a fixed order; the fp16 scale is the job's static one
+    // (|h| <= sqrt(K) * max|gain|).  Other GEMMs with int8 weights: a power-of-two scale from the
+    // row maximum gathered while the operand was written.
 #ifdef QUASAR_GEMM_TIMER
-    const long long c_stats0 = clock64();
+    const long long c_f0 = clock64();
 #endif
-    if (normed || W_INT8) {
-      float ss = 0.f, amax = 0.f;
-      for (int kc = 0; kc < v.nchunks; ++kc) {
-        load_x_raw<W_INT8>(xr, xsrc, ld, M, jb.K, kc * kChunk, warp, g, t);
-        x_stats<W_INT8>(xr, jb.gain, jb.K, kc * kChunk, warp, t, ss, amax);
-      }
+    float rnorm = 1.f, xscale = 1.f, inv = 1.f;
+    if (normed) {
+      float ss = 0.f;
+#pragma unroll 8
+      for (int c = t; c < ncta; c += 4) ss += __ldcg(p.ss_part + c * 8 + g);
       ss += __shfl_xor_sync(0xffffffffu, ss, 1);
       ss += __shfl_xor_sync(0xffffffffu, ss, 2);
-      amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
-      amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
-      if (t == 0) {
-        misc[kMiscRowSum + warp * 8 + g] = ss;
-        misc[kMiscCand + warp * 8 + g] = amax;
-      }
-      cbar();
-      float tot = 0.f, mx = 0.f;
-#pragma unroll
-      for (int w = 0; w < NW; ++w) {
-        tot += misc[kMiscRowSum + w * 8 + g];
-        mx = fmaxf(mx, misc[kMiscCand + w * 8 + g]);
-      }
-      if (normed) {
-        rnorm = 1.0f / sqrtf(tot / (float)jb.K + p.rms_eps);
-        mx *= rnorm * 1.01f;
-      }
-      float inv = 1.f;
-      if (W_INT8 && mx > 32768.f && mx < 3.0e38f) {
+      rnorm = 1.0f / sqrtf(ss / (float)jb.K + p.rms_eps);
+      if (W_INT8) { xscale = jb.xscale; inv = 1.0f / xscale; }
+    } else if (W_INT8) {
+      const float mx = __uint_as_float(__ldcg(p.amax_buf + job * 8 + g));
+      if (mx > 32768.f && mx < 3.0e38f) {
         int e;
         (void)frexpf(mx, &e);               // mx = f * 2^e, f in [0.5, 1)
         xscale = ldexpf(1.f, 15 - e);       // scaled row maximum <= 2^15
         inv = ldexpf(1.f, e - 15);
       }
-      cbar();                               // everyone has read the per-warp partials
-      if (warp == 0 && t == 0) misc[kMiscInvScale + g] = inv;
-      if (v.nchunks == 1) {
-        if (normed) apply_norm<W_INT8>(xr, jb.gain, rnorm, jb.K, 0, warp, t);
-        if (W_INT8) xsum = to_f16(xr, xscale);
-        have_x = true;
-      }
-    } else if (warp == 0 && t == 0) {
-      misc[kMiscInvScale + g] = 1.f;
     }
+    if (warp == 0 && t == 0) misc[kMiscInvScale + g] = inv;   // read in the epilogues, behind a CTA barrier
 
 #ifdef QUASAR_GEMM_TIMER
-    if (threadIdx.x == 0) g_gemm_clk[blockIdx.x][1] += clock64() - c_stats0;
+    if (threadIdx.x == 0 && rnorm != 123.f && g_clk_on) g_gemm_clk[blockIdx.x][1] += clock64() - c_f0;
 #endif
+    uint4 xr[kXr];
+    bool have_x = false;
+    float ss_run = 0.f;   // threads 0..7 (o / down): sum of squares of the row of x this CTA has written
+
     for (int tg = 0; tg < v.ngroups; ++tg) {
       const int gt = min(GT, v.tiles - tg * GT);
-      float acc[GT][4];
-#pragma unroll
-      for (int i = 0; i < GT; ++i) acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.f;
+      // The element this thread finishes in the group's epilogue; its step sizes and residual are
+      // fetched now so that the epilogue does not wait for L2.
+      const int e_tile = jb.kind == kJobGateUp ? (int)threadIdx.x >> 6 : (int)threadIdx.x >> 7;
+      const int e_col = jb.kind == kJobGateUp ? ((int)threadIdx.x >> 3) & 7 : ((int)threadIdx.x >> 4) & 7;
+      const int e_row = jb.kind == kJobGateUp ? (int)threadIdx.x & 7 : (int)threadIdx.x & 15;
+      const int e_unit = v.u0 + (tg * GT + e_tile) * v.rows_per_tile + e_row;   // output channel, or gate/up pair
+      const bool e_ok = e_tile < gt && e_unit < v.u1 && e_col < M;
+      float d0 = 1.f, d1 = 1.f, resid = 0.f;
+      if (e_ok) {
+        if (jb.delta != nullptr) {
+          d0 = __ldg(jb.delta + e_unit);
+          if (jb.kind == kJobGateUp) d1 = __ldg(jb.delta + v.units + e_unit);
+        }
+        if (residual) resid = __bfloat162float(__ldcg(p.x + (size_t)e_col * jb.N + e_unit));
+      }
+
+      // Accumulators live for one tile and one chunk; each warp then parks them in its own part of
+      // `red` (summing over the chunks of a long contraction), where the epilogue adds the 16 warps up.
+#ifdef QUASAR_GEMM_TIMER
+      const long long c_t0 = clock64();
+#endif
       for (int kc = 0; kc < v.nchunks; ++kc) {
         if (!have_x) {
-          load_x_raw<W_INT8>(xr, xsrc, ld, M, jb.K, kc * kChunk, warp, g, t);
-          if (normed) apply_norm<W_INT8>(xr, jb.gain, rnorm, jb.K, kc * kChunk, warp, t);
-          if (W_INT8) {
-            const float part = to_f16(xr, xscale);
-            if (tg == 0) xsum += part;       // every chunk is visited once per tile group
-          }
+          GEMM_CLK(4, load_operand<W_INT8>(xr, xsrc, ld, M, jb.K, kc * kChunk, jb.gain, rnorm, xscale, warp, g, t); if (xr[0].x == 0x12345u) slot ^= 0);
           have_x = (v.nchunks == 1);
         }
         const int kbase = kc * kChunk;
         const int cb = min(kChunk, jb.K - kbase) * kElemBytes;        // bytes of a weight row in this chunk
         const int pb_last = cb - (cb - 1) / kRowBytes * kRowBytes;    // bytes of its last piece
+#pragma unroll 1
+        for (int tile = 0; tile < gt; ++tile) {
+          // block rows behind MMA rows g and g + 8 (rows past the tile stay inside the stage and feed
+          // accumulator rows that are never stored)
+          const int ra = g;
+          const int rb = v.kind == kJobGateUp ? tile_units(v, tg * GT + tile) + g : g + 8;
+          const int oa_full = block_offset(ra, kRowBytes, warp, t), ob_full = block_offset(rb, kRowBytes, warp, t);
+          const int oa_last = block_offset(ra, pb_last, warp, t), ob_last = block_offset(rb, pb_last, warp, t);
+          float ch[4][4];
 #pragma unroll
-        for (int tile = 0; tile < GT; ++tile) {
-          if (tile < gt) {
-            // block rows behind MMA rows g and g + 8 (rows past the tile stay inside the stage and feed
-            // accumulator rows that are never stored)
-            const int ra = g;
-            const int rb = v.kind == kJobGateUp ? tile_units(v, tg * GT + tile) + g : g + 8;
-            const int oa_full = block_offset(ra, kRowBytes, warp, t), ob_full = block_offset(rb, kRowBytes, warp, t);
-            const int oa_last = block_offset(ra, pb_last, warp, t), ob_last = block_offset(rb, pb_last, warp, t);
-            float ch[4][4];
+          for (int i = 0; i < 4; ++i) ch[i][0] = ch[i][1] = ch[i][2] = ch[i][3] = 0.f;
 #pragma unroll
-            for (int i = 0; i < 4; ++i) ch[i][0] = ch[i][1] = ch[i][2] = ch[i][3] = 0.f;
-#pragma unroll
-            for (int s = 0; s < SPC; ++s) {
-              const int b0 = s * kRowBytes;
-              if (b0 < cb) {
-                const bool last = b0 + kRowBytes >= cb;
-                const bool lane_valid = b0 + warp * 64 + t * 16 < cb;
-                bool got;
-                GEMM_CLK(0, got = mbar_wait(pipe.full + slot, phase, pipe.abort_flag, pipe.status));
-                if (!got) return false;
-                // a lane past the end of a short piece reads inside the stage (offset < 16 KB) but not its own data
-                const int oa = last ? (lane_valid ? oa_last : 0) : oa_full;
-                const int ob = last ? (lane_valid ? ob_last : 0) : ob_full;
-                GEMM_CLK(3, consume_stage<W_INT8>(pipe.ring + slot * kStageBytes, s, oa, ob, lane_valid, xr, ch);
-                         __syncwarp();
-                         if (lane == 0) mbar_arrive(pipe.empty + slot));
-                if (++slot == kStages) { slot = 0; phase ^= 1u; }
-              }
+          for (int s = 0; s < SPC; ++s) {
+            const int b0 = s * kRowBytes;
+            if (b0 < cb) {
+              const bool last = b0 + kRowBytes >= cb;
+              const bool lane_valid = b0 + warp * 64 + t * 16 < cb;
+              bool got;
+              GEMM_CLK(0, got = mbar_wait(pipe.full + slot, phase, pipe.abort_flag, pipe.status));
+              if (!got) return false;
+              // a lane past the end of a short piece reads inside the stage (offset < 16 KB) but not its own data
+              const int oa = last ? (lane_valid ? oa_last : 0) : oa_full;
+              const int ob = last ? (lane_valid ? ob_last : 0) : ob_full;
+              GEMM_CLK(3, consume_stage<W_INT8>(pipe.ring + slot * kStageBytes, s, oa, ob, lane_valid, xr, ch);
+                       __syncwarp();
+                       if (lane == 0) mbar_arrive(pipe.empty + slot));
+              if (++slot == kStages) { slot = 0; phase ^= 1u; }
             }
-#pragma unroll
-            for (int i = 0; i < 4; ++i) acc[tile][i] += (ch[0][i] + ch[1][i]) + (ch[2][i] + ch[3][i]);
           }
+          float* r = red + ((warp * GT + tile) * 16) * 8;
+          float2 lo = make_float2((ch[0][0] + ch[1][0]) + (ch[2][0] + ch[3][0]), (ch[0][1] + ch[1][1]) + (ch[2][1] + ch[3][1]));
+          float2 hi = make_float2((ch[0][2] + ch[1][2]) + (ch[2][2] + ch[3][2]), (ch[0][3] + ch[1][3]) + (ch[2][3] + ch[3][3]));
+          float2* plo = reinterpret_cast<float2*>(r + g * 8 + 2 * t);
+          float2* phi = reinterpret_cast<float2*>(r + (g + 8) * 8 + 2 * t);
+          if (kc > 0) {   // only this thread touches these two slots
+            const float2 a = *plo, b = *phi;
+            lo.x += a.x; lo.y += a.y; hi.x += b.x; hi.y += b.y;
+          }
+          *plo = lo;
+          *phi = hi;
         }
       }
+#ifdef QUASAR_GEMM_TIMER
+      if (threadIdx.x == 0 && g_clk_on) g_gemm_clk[blockIdx.x][5] += clock64() - c_t0;
+#endif
       // ---- cross-warp reduction in a fixed order, then the fused epilogue ----
-#pragma unroll
-      for (int tile = 0; tile < GT; ++tile) {
-        float* r = red + ((warp * GT + tile) * 16) * 8;
-        *reinterpret_cast<float2*>(r + g * 8 + 2 * t) = make_float2(acc[tile][0], acc[tile][1]);
-        *reinterpret_cast<float2*>(r + (g + 8) * 8 + 2 * t) = make_float2(acc[tile][2], acc[tile][3]);
+      GEMM_CLK(2, cbar();
+               epilogue(p, jb, v, job, e_ok, e_tile, e_row, e_col, e_unit, d0, d1, resid, red, misc);
+               cbar());
+      if (residual && threadIdx.x < 8) {   // fixed order: tiles of the group, groups of the phase
+        for (int tile = 0; tile < gt; ++tile) ss_run += misc[kMiscPart + tile * 8 + threadIdx.x];
       }
-      if (W_INT8 && tg == 0) {   // per-warp share of sum_k x_k of operand row g
-        float xs = xsum;
-        xs += __shfl_xor_sync(0xffffffffu, xs, 1);
-        xs += __shfl_xor_sync(0xffffffffu, xs, 2);
-        if (t == 0) misc[kMiscRowSum + warp * 8 + g] = xs;
-      }
-      GEMM_CLK(2, cbar(); epilogue(p, jb, v, tg, gt, red, misc); cbar());
     }
+    if (residual && threadIdx.x < 8) p.ss_part[cta * 8 + threadIdx.x] = ss_run;
     slot_io = slot;
     phase_io = phase;
     return true;
   }
 
-  __device__ static float reduce_at(const float* red, int tile, int row, int col) {
+  __device__ __forceinline__ static float reduce_at(const float* red, int tile, int row, int col) {
     float s = 0.f;
 #pragma unroll
     for (int w = 0; w < NW; ++w) s += red[((w * GT + tile) * 16 + row) * 8 + col];
     return s;
   }
 
-  __device__ static void epilogue(const MegaParams& p, const MegaJob& jb, const JobView& v, int tg, int gt,
-                                  const float* red, float* misc) {
-    const int M = p.M;
-    // A thread always meets the same operand row `col` (kCT is a multiple of 128).  out = (sum - corr) * unit:
-    // corr removes the weights' offset, unit undoes the operand's scale and the 2^-24 of the byte trick.
-    const int my_col = jb.kind == kJobGateUp ? (threadIdx.x >> 3) & 7 : (threadIdx.x >> 4) & 7;
-    float corr = 0.f, unit = 1.f;
-    if (W_INT8) {
-      float xs = 0.f;
-#pragma unroll
-      for (int w = 0; w < NW; ++w) xs += misc[kMiscRowSum + w * 8 + my_col];
-      corr = kWeightOffset * xs;
-      unit = kWeightUnit * misc[kMiscInvScale + my_col];
-    }
+  // One output element per thread: sum the 16 warps' partials, apply the step size (and the operand's
+  // scale), then what the step of the pass asks for.
+  __device__ __forceinline__ static void epilogue(const MegaParams& p, const MegaJob& jb, const JobView& v, int job,
+                                                  bool ok, int tile, int row, int col, int unit_idx, float d0, float d1,
+                                                  float resid, const float* red, float* misc) {
+    const int lane = threadIdx.x & 31;
+    const float unit = W_INT8 ? misc[kMiscInvScale + col] : 1.f;
     if (jb.kind == kJobGateUp) {
-      const int F = v.units;
-      for (int e = threadIdx.x; e < gt * 8 * 8; e += kCT) {
-        const int r = e & 7, col = (e >> 3) & 7, tile = e >> 6;
-        const int pair = v.u0 + (tg * GT + tile) * 8 + r;
-        if (pair >= v.u1 || col >= M) continue;
-        const float dg = jb.delta ? jb.delta[pair] : 1.f, du = jb.delta ? jb.delta[F + pair] : 1.f;
-        const float gate = bf16_round_f((reduce_at(red, tile, r, col) - corr) * unit * dg);
-        const float up = bf16_round_f((reduce_at(red, tile, r + 8, col) - corr) * unit * du);
-        p.act[(size_t)col * F + pair] = __float2bfloat16_rn(gate / (1.0f + expf(-gate)) * up);
+      // SwiGLU: act = silu(gate) * up, gate and up rounded to bf16 first (they are tensors of the layer)
+      float a = 0.f;
+      if (ok) {
+        const float gate = bf16_round_f(reduce_at(red, tile, row, col) * unit * d0);
+        const float up = bf16_round_f(reduce_at(red, tile, row + 8, col) * unit * d1);
+        const __nv_bfloat16 av = __float2bfloat16_rn(gate / (1.0f + expf(-gate)) * up);
+        p.act[(size_t)col * v.units + unit_idx] = av;
+        a = fabsf(__bfloat162float(av));
+      }
+      if (W_INT8) {   // row maximum of the next GEMM's operand (8 consecutive lanes share a row)
+        a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 1));
+        a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 2));
+        a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 4));
+        if ((lane & 7) == 0 && a > 0.f) atomicMax(p.amax_buf + (job + 1) * 8 + col, __float_as_uint(a));
       }
       return;
     }
-    const int N = jb.N;
     float best = -INFINITY;
     int best_i = 0x7fffffff;
-    for (int e = threadIdx.x; e < gt * 16 * 8; e += kCT) {
-      const int r = e & 15, col = (e >> 4) & 7, tile = e >> 7;
-      const int n = v.u0 + (tg * GT + tile) * 16 + r;
-      if (n >= v.u1 || col >= M) continue;
-      const float val = (reduce_at(red, tile, r, col) - corr) * unit * (jb.delta ? jb.delta[n] : 1.f);
-      const size_t idx = (size_t)col * N + n;
+    float sq = 0.f;
+    if (ok) {
+      const float val = reduce_at(red, tile, row, col) * unit * d0;
+      const size_t idx = (size_t)col * jb.N + unit_idx;
       if (jb.kind == kJobQkv) {
         p.qkv[idx] = __float2bfloat16_rn(val);
       } else if (jb.kind == kJobLm) {
         if (p.logits) p.logits[idx] = val;
-        // e -> (tile, col, r): a thread sees a single col because kCT % 128 == 0
-        if (val > best || (val == best && n < best_i)) { best = val; best_i = n; }
+        best = val;
+        best_i = unit_idx;
       } else {  // o / down: residual add into the stream
-        const float xv = __bfloat162float(__ldcg(p.x + idx));
-        p.x[idx] = __float2bfloat16_rn(bf16_round_f(val) + xv);
+        const __nv_bfloat16 xn = __float2bfloat16_rn(bf16_round_f(val) + resid);
+        p.x[idx] = xn;
+        const float xf = __bfloat162float(xn);
+        sq = xf * xf;
       }
     }
+    if (jb.kind == kJobO || jb.kind == kJobDown) {
+      // sum of squares of what this CTA adds to each row of x (16 consecutive lanes share tile and row)
+#pragma unroll
+      for (int o = 8; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+      if ((lane & 15) == 0) misc[kMiscPart + tile * 8 + col] = sq;
+    }
     if (jb.kind == kJobLm) {
-      // combine the 16 lanes that share a col (lanes differ in r), then the 4 such groups per col in the CTA
+      // combine the 16 lanes that share a col (lanes differ in row), then the 4 such groups per col in the CTA
 #pragma unroll
       for (int o = 8; o > 0; o >>= 1) {
         const float ob = __shfl_xor_sync(0xffffffffu, best, o);
@@ -721,7 +686,7 @@ struct GemmPhase {
 };
 
 // ---- block bookkeeping + embedding gather (phase 0) -------------------------------------------
-__device__ void prep_phase(const MegaParams& p, int cta, int ncta) {
+__device__ void prep_phase(const MegaParams& p, float* misc, int cta, int ncta) {
   // one thread per sequence validates the block and derives ancestor masks / depths
   if (cta == 0 && (int)threadIdx.x < p.B) {
     const int b = threadIdx.x;
@@ -747,15 +712,37 @@ __device__ void prep_phase(const MegaParams& p, int cta, int ncta) {
     p.bi.valid[b] = err ? 0 : 1;
     if (err) atomicMin(p.status, err);
   }
-  // embedding rows, 16 bytes per thread, spread over the grid
-  const int chunks = p.H / 8;
-  for (int i = cta * kCT + threadIdx.x; i < p.M * chunks; i += ncta * kCT) {
-    const int m = i / chunks, c = i % chunks;
+  // row maxima of the un-normed GEMM operands start at zero (gathered with atomicMax during the pass)
+  for (int i = cta * kCT + threadIdx.x; i < p.n_jobs * 8; i += ncta * kCT) p.amax_buf[i] = 0u;
+  // Embedding rows: CTA m gathers row m and leaves its sum of squares for the first RMSNorm; every
+  // CTA leaves a (possibly zero) entry per row, the layout the later phases use too.
+  float* wsum = misc + kMiscRowSum;
+  const int m = cta;   // the grid has at least 8 CTAs
+  float ss = 0.f;
+  if (m < p.M) {
     const int tok = p.tokens[m];
     const bool ok = tok >= 0 && tok < p.vocab;
-    uint4 v = make_uint4(0, 0, 0, 0);
-    if (ok) v = __ldg(reinterpret_cast<const uint4*>(p.embed + (size_t)tok * p.H) + c);
-    reinterpret_cast<uint4*>(p.x + (size_t)m * p.H)[c] = v;
+    for (int c = threadIdx.x; c < p.H / 8; c += kCT) {
+      uint4 v = make_uint4(0, 0, 0, 0);
+      if (ok) v = __ldg(reinterpret_cast<const uint4*>(p.embed + (size_t)tok * p.H) + c);
+      reinterpret_cast<uint4*>(p.x + (size_t)m * p.H)[c] = v;
+      const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&v);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float2 f = __bfloat1622float2(h[e]);
+        ss += f.x * f.x + f.y * f.y;
+      }
+    }
+  }
+  ss = warp_sum(ss);
+  if ((threadIdx.x & 31) == 0) wsum[threadIdx.x >> 5] = ss;
+  cbar();
+  if (threadIdx.x < 8) {
+    float tot = 0.f;
+    if ((int)threadIdx.x == m && m < p.M) {
+      for (int w = 0; w < NW; ++w) tot += wsum[w];
+    }
+    p.ss_part[cta * 8 + threadIdx.x] = tot;
   }
 }
 
@@ -793,7 +780,7 @@ __device__ void rope_vec(const __nv_bfloat16* src, const __nv_bfloat16* gain, co
 }
 
 template <int D>
-__device__ void attention_phase(const MegaParams& p, int layer, __nv_bfloat16* k_s, __nv_bfloat16* v_s,
+__device__ __noinline__ void attention_phase(const MegaParams& p, int layer, __nv_bfloat16* k_s, __nv_bfloat16* v_s,
                                 __nv_bfloat16* q_s, int cta, int ncta) {
   constexpr int kStride = D + 8;
   constexpr int kDSteps = D / 16;
@@ -971,7 +958,7 @@ __device__ void attention_phase(const MegaParams& p, int layer, __nv_bfloat16* k
 
 // merge the chunk partials of every (row, query head) in chunk order: one warp per item
 template <int D>
-__device__ void merge_phase(const MegaParams& p, int cta, int ncta) {
+__device__ __noinline__ void merge_phase(const MegaParams& p, int layer, bool want_amax, int cta, int ncta) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   constexpr int kPer = D / 32;
   const int G = p.Hq / p.Hkv;
@@ -1012,8 +999,18 @@ __device__ void merge_phase(const MegaParams& p, int cta, int ncta) {
       }
     }
     const float inv = 1.0f / den;
+    float amax = 0.f;
 #pragma unroll
-    for (int e = 0; e < kPer; ++e) dst[lane * kPer + e] = __float2bfloat16_rn(acc[e] * inv);
+    for (int e = 0; e < kPer; ++e) {
+      const __nv_bfloat16 ov = __float2bfloat16_rn(acc[e] * inv);
+      dst[lane * kPer + e] = ov;
+      amax = fmaxf(amax, fabsf(__bfloat162float(ov)));
+    }
+    if (want_amax) {   // row maximum of the o projection's operand
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+      if (lane == 0 && amax > 0.f) atomicMax(p.amax_buf + (4 * layer + 1) * 8 + m, __float_as_uint(amax));
+    }
   }
 }
 
@@ -1095,12 +1092,10 @@ __global__ void __launch_bounds__(kThreads, 1) verify_megakernel(const MegaParam
   }
   __syncthreads();
 
-  if (warp >= NW) {  // the weight stream; hands most of its registers to the consumer warps
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;\n" ::"n"(kProducerRegs));
-    if (warp == NW) producer_loop<W_INT8>(p, pipe, cta, ncta);
+  if (warp == NW) {  // the weight stream
+    producer_loop<W_INT8>(p, pipe, cta, ncta);
     return;
   }
-  asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;\n" ::"n"(kConsumerRegs));
 
   int slot = 0;
   uint32_t phase = 0;
@@ -1111,7 +1106,7 @@ __global__ void __launch_bounds__(kThreads, 1) verify_megakernel(const MegaParam
 #endif
 
   PHASE_MARK();
-  prep_phase(p, cta, ncta);
+  prep_phase(p, misc, cta, ncta);
   PHASE_MARK();
   ok = gs.sync();
   PHASE_MARK();
@@ -1127,7 +1122,7 @@ __global__ void __launch_bounds__(kThreads, 1) verify_megakernel(const MegaParam
       PHASE_MARK();
       if (!(ok = gs.sync())) break;
       PHASE_MARK();
-      merge_phase<D>(p, cta, ncta);
+      merge_phase<D>(p, job >> 2, W_INT8, cta, ncta);
       PHASE_MARK();
       if (!(ok = gs.sync())) break;
       PHASE_MARK();
@@ -1215,9 +1210,9 @@ extern "C" int quasar_debug_phase_marks(long long* clk_host, int* n_host) {
   return kMaxMarks;
 }
 extern "C" int quasar_debug_gemm_clocks(long long* host, int reset) {
-  if (cudaMemcpyFromSymbol(host, g_gemm_clk, sizeof(long long) * 160 * 4) != cudaSuccess) return -1;
+  if (cudaMemcpyFromSymbol(host, g_gemm_clk, sizeof(long long) * 160 * 8) != cudaSuccess) return -1;
   if (reset) {
-    static long long zero[160 * 4];
+    static long long zero[160 * 8];
     if (cudaMemcpyToSymbol(g_gemm_clk, zero, sizeof(zero)) != cudaSuccess) return -1;
   }
   return 0;
@@ -1257,6 +1252,10 @@ int mega_grid_size(int weight_dtype, int D, int* ncta_out) {
   QUASAR_CUDA_CHECK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, kThreads, (size_t)kSmemBytes));
   if (per_sm < 1) {
     set_error("persistent kernel does not fit on an SM (%d bytes of shared memory)", kSmemBytes);
+    return QUASAR_ERR_CUDA;
+  }
+  if (sms < 8) {
+    set_error("persistent kernel needs at least 8 SMs");
     return QUASAR_ERR_CUDA;
   }
   *ncta_out = sms;

@@ -14,7 +14,8 @@ struct MegaJob {
   const void* wp;              // [N][K] int8 or bf16, every CTA's row range permuted into its consumption order
   const float* delta;          // [N] or nullptr
   const __nv_bfloat16* gain;   // RMSNorm gain fused into the operand load, or nullptr
-  int N, K, kind, pad;
+  int N, K, kind;
+  float xscale;                // normed GEMMs, int8 weights: power-of-two scale keeping h = x r gain inside fp16 (usually 1)
 };
 
 struct MegaLayer {
@@ -41,6 +42,8 @@ struct MegaParams {
   int attn_nchunk, attn_rpad;
   float* cand_val;          // [grid][8] per-CTA arg-max candidates
   int* cand_idx;
+  float* ss_part;           // [grid][8] per-CTA sums of squares of the rows of x, left by the phase that wrote x
+  unsigned* amax_buf;       // [n_jobs][8] row maxima (float bits) of the un-normed GEMM operands
   unsigned* barrier;        // zeroed before every launch
   int32_t *accept_len, *bonus, *accept_path, *status;
 };
