@@ -65,7 +65,7 @@ size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
 
 // Layout of the verify workspace; every offset is a multiple of 256 bytes.
 struct Workspace {
-  size_t x, h, qkv, attn, gu, act, logits, top1, anc, depth, valid, lin, att, cand, ss_part, amax, barrier, total;
+  size_t x, h, qkv, attn, gu, act, logits, top1, anc, depth, valid, lin, att, cand, ss_part, amax, attn_count, barrier, total;
   size_t lin_bytes, att_bytes;
 };
 
@@ -110,6 +110,7 @@ Workspace layout(const quasar_config& c, int B, int T_max, int s_max) {
   w.cand = take((size_t)kMaxGrid * 8 * 2 * sizeof(float));
   w.ss_part = take((size_t)kMaxGrid * 8 * sizeof(float));
   w.amax = take((size_t)(4 * c.n_layers + 1) * 8 * sizeof(unsigned));
+  w.attn_count = take((size_t)(c.n_layers > 0 ? c.n_layers : 1) * B * c.n_kv_heads * sizeof(unsigned));
   w.barrier = take(256);
   w.total = off;
   return w;
@@ -257,6 +258,7 @@ int verify_impl(quasar_model* m, const quasar_kv* kv, const int32_t* tokens, con
     p.cand_idx = reinterpret_cast<int*>(wsp + ws.cand + (size_t)kMaxGrid * 8 * sizeof(float));
     p.ss_part = reinterpret_cast<float*>(wsp + ws.ss_part);
     p.amax_buf = reinterpret_cast<unsigned*>(wsp + ws.amax);
+    p.attn_count = reinterpret_cast<unsigned*>(wsp + ws.attn_count);
     p.barrier = reinterpret_cast<unsigned*>(wsp + ws.barrier);
     p.accept_len = accept_len; p.bonus = bonus; p.accept_path = accept_path; p.status = status;
     QUASAR_CUDA_CHECK(cudaMemsetAsync(p.barrier, 0, 256, stream));

@@ -44,12 +44,14 @@ namespace {
 
 constexpr int NW = kMegaWarps;             // consumer warps per CTA
 constexpr int kCT = NW * 32;               // consumer threads
-constexpr int kThreads = kCT + 32;         // + the producer warp (17 warps: 5 on one SM sub-partition, so 96 registers per thread)
+constexpr int kThreads = kCT + 32;         // + the producer warp (9 warps: at most 3 per SM sub-partition, so 168 registers per thread)
 constexpr int kRowBytes = 1024;            // bytes of one weight row per stage
 constexpr int kStageBytes = 16 * kRowBytes;  // 16 weight rows
-constexpr int kStages = 10;                // ring depth (160 KB of weights in flight per CTA)
+constexpr int kStages = 8;                 // ring depth (128 KB of weights in flight per CTA)
 constexpr int kChunk = 4096;               // contraction elements whose activations a warp keeps in registers
-constexpr int kXr = 8;                     // 16-byte registers holding this thread's share of the operand chunk
+constexpr int kWarpBytes = kRowBytes / NW;   // bytes of a row piece one warp covers (128)
+constexpr int kSub = kWarpBytes / 64;        // 64-byte sub-slices of it: four lanes x 16 bytes each
+constexpr int kXr = 8 * kSub;                // 16-byte registers holding this thread's share of the operand chunk
 constexpr int GT = 4;                      // 16-row tiles accumulated together before a reduction
 constexpr int kKeyTile = 64;
 constexpr int kMaxRowsAttn = 64;           // query rows (heads-in-group x block rows) per kv head
@@ -57,20 +59,28 @@ constexpr float kLog2e = 1.4426950408889634f;
 constexpr unsigned long long kWaitBudgetNs = 2000000000ull;  // every device-side wait gives up after 2 s
 
 // ---- shared memory map --------------------------------------------------------------------
-constexpr int kRingBytes = kStages * kStageBytes;                        // 163840
+constexpr int kRingBytes = kStages * kStageBytes;                        // 131072
 constexpr int kRedBytes = NW * GT * 128 * 4;                             // 32768
 constexpr int kKvTileBytes = kKeyTile * (128 + 8) * 2;                   // 17408 (D = 128)
-constexpr int kUnionBytes = (2 * kKvTileBytes > kRedBytes) ? 2 * kKvTileBytes : kRedBytes;
 constexpr int kQTileBytes = kMaxRowsAttn * (128 + 8) * 2;                // 17408
+constexpr int kAttnBytes = 2 * kKvTileBytes + kQTileBytes;               // K, V and Q tiles of the attention phase
 constexpr int kMiscBytes = 2048;
-constexpr int kSmemBytes = kRingBytes + kUnionBytes + kQTileBytes + kMiscBytes;
+// The operand of a GEMM phase (<= 8 rows x one chunk, bf16) and its norm gain land in a staging buffer by
+// bulk copy before they go to registers.  The attention tiles share that buffer: the two are never alive
+// at the same time.  The reduction buffer has bytes of its own (partial sums stay parked there while the
+// next chunk of a long contraction is staged).
+constexpr int kXRowBytes = kChunk * 2;                                   // 8192
+constexpr int kXBytes = 8 * kXRowBytes;                                  // 65536
+constexpr int kGainBytes = kChunk * 2;                                   // 8192
+constexpr int kStageBufBytes = (kXBytes + kGainBytes > kAttnBytes) ? kXBytes + kGainBytes : kAttnBytes;
+constexpr int kSmemBytes = kRingBytes + kRedBytes + kStageBufBytes + kMiscBytes;
 static_assert(kSmemBytes <= 227 * 1024, "shared memory budget of one SM");
 
 // misc region (floats): [0,128) per-warp row sums, [128,136) running arg-max values, [136,144) its
 // indices, [144,152) 1/scale of the operand rows, [152,184) per-tile sums of squares, [200] abort flag, [256,512) candidates / per-warp
 // row maxima, byte 1536.. the mbarriers.
-constexpr int kMiscRowSum = 0, kMiscRunV = 128, kMiscRunI = 136, kMiscInvScale = 144, kMiscPart = 152, kMiscAbort = 200,
-              kMiscCand = 256, kMiscBarBytes = 1536;
+constexpr int kMiscRowSum = 0, kMiscRunV = 128, kMiscRunI = 136, kMiscInvScale = 144, kMiscPart = 152, kMiscFlag = 190, kMiscAbort = 200,
+              kMiscCand = 256, kMiscBarBytes = 1536;   // 2 kStages + 1 barriers of 8 bytes
 
 __device__ __forceinline__ void mma16816_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                               uint32_t b0, uint32_t b1) {
@@ -127,6 +137,19 @@ __device__ __forceinline__ float warp_sum(float v) {
   return v;
 }
 
+// Loads that must be ISSUED where they are written (the compiler may not sink them to their first use):
+// the epilogue's step sizes and residual are requested before the stage loop and arrive during it.
+__device__ __forceinline__ float ld_early_f32(const float* p) {
+  float v;
+  asm volatile("ld.global.nc.f32 %0, [%1];\n" : "=f"(v) : "l"(p));
+  return v;
+}
+__device__ __forceinline__ float ld_early_bf16_cg(const __nv_bfloat16* p) {
+  unsigned short v;
+  asm volatile("ld.global.cg.u16 %0, [%1];\n" : "=h"(v) : "l"(p));
+  return __uint_as_float((unsigned)v << 16);
+}
+
 // barrier among the consumer warps only (the producer warp never joins it)
 __device__ __forceinline__ void cbar() { asm volatile("bar.sync 1, %0;\n" ::"n"(kCT) : "memory"); }
 
@@ -136,6 +159,17 @@ __device__ __forceinline__ unsigned long long now_ns() {
   return t;
 }
 
+#ifdef QUASAR_TIMELINE
+__device__ long long g_timeline[160][256];
+__device__ long long g_timeline2[160][16][40];
+#define TL_DECL __shared__ long long s_tl[256]; int tl_n = 0;
+#define TL_MARK() do { if (threadIdx.x == 0 && tl_on && tl_n < 256) s_tl[tl_n++] = clock64(); } while (0)
+#define TL_FLUSH() do { if (threadIdx.x == 0 && tl_on) { for (int i__ = 0; i__ < tl_n; ++i__) g_timeline[blockIdx.x][i__] = s_tl[i__]; g_timeline[blockIdx.x][255] = tl_n; } } while (0)
+#else
+#define TL_DECL
+#define TL_MARK() do { } while (0)
+#define TL_FLUSH() do { } while (0)
+#endif
 #ifdef QUASAR_PHASE_TIMER
 // Diagnostic build only: thread 0 of every CTA stamps the SM clock at each phase boundary.
 constexpr int kMaxMarks = 640;
@@ -143,7 +177,13 @@ __device__ long long g_phase_clk[160][kMaxMarks];
 __device__ int g_phase_n[160];
 __device__ long long g_gemm_clk[160][8];
 __device__ int g_clk_on_dummy;
-#define g_clk_on (job == p.n_jobs - 1)   // warp 0 of every CTA: cycles waiting for stages, in stats, in epilogues, in GEMM phases
+#ifndef QUASAR_TIMER_KIND
+#define QUASAR_TIMER_KIND 4
+#endif
+#define g_clk_on (jb.kind == QUASAR_TIMER_KIND)
+__device__ long long g_attn_clk[160][8];
+__device__ long long g_attn_tmp_unused;
+#define ATTN_T(i) do { if (threadIdx.x == 0) { const long long c__ = clock64(); s_attn_clk[i] += c__ - at0; at0 = c__; } } while (0)
 #define PHASE_MARK()                                                                         \
   do {                                                                                       \
     if (threadIdx.x == 0 && mark_n < kMaxMarks) g_phase_clk[blockIdx.x][mark_n++] = clock64(); \
@@ -153,12 +193,13 @@ __device__ int g_clk_on_dummy;
   do {                                                              \
     const long long c0__ = clock64();                               \
     expr;                                                           \
-    if (threadIdx.x == 0 && g_clk_on) g_gemm_clk[blockIdx.x][i] += clock64() - c0__; \
+    tacc[i] += (unsigned)(clock64() - c0__);                          \
   } while (0)
 #else
 #define GEMM_CLK(i, expr) do { expr; } while (0)
 #endif
 #else
+#define ATTN_T(i) do { } while (0)
 #define PHASE_MARK() do { } while (0)
 #define GEMM_CLK(i, expr) do { expr; } while (0)
 #endif
@@ -360,90 +401,128 @@ struct GridSync {
 };
 
 // ---- operand load: the <= 8 activation rows of this warp's share of a contraction chunk ----------
-// A stage holds a 1024-byte piece of every weight row of a tile; warp w reads bytes [64 w, 64 w + 64)
-// of the piece and lane (g, t) the 16 bytes at 16 t.  int8 weights: stage s of the chunk covers k = base + 1024 s + 64 w +
-// 16 t + (0..15), held in xr[2s], xr[2s+1] (fp16).  bf16 weights: k = base + 512 s + 32 w + 8 t + (0..7),
-// held in xr[s] (bf16).
+// A stage holds a 1024-byte piece of every weight row of a tile; warp w reads bytes [kWarpBytes w,
+// kWarpBytes (w + 1)) of the piece as kSub sub-slices of 64 bytes, lane (g, t) the 16 bytes at 16 t of each.
+// int8 weights: stage s, sub-slice u covers k = base + 1024 s + kWarpBytes w + 64 u + 16 t + (0..15), held
+// in xr[2 (s kSub + u)], xr[.. + 1] (fp16).  bf16 weights: half as many elements per byte range, held in
+// xr[s kSub + u] (bf16).
 template <bool W_INT8>
 __device__ __forceinline__ int x_index(int i, int kbase, int warp, int t) {
-  return W_INT8 ? (kbase + (i >> 1) * 1024 + warp * 64 + t * 16 + (i & 1) * 8) : (kbase + i * 512 + warp * 32 + t * 8);
+  if (W_INT8) {
+    const int su = i >> 1, s = su / kSub, u = su % kSub;
+    return kbase + s * 1024 + warp * kWarpBytes + u * 64 + t * 16 + (i & 1) * 8;
+  }
+  const int s = i / kSub, u = i % kSub;
+  return kbase + s * 512 + (warp * kWarpBytes + u * 64 + t * 16) / 2;
 }
 
-// The <= 8 operand rows of this warp's share of chunk `kbase`, ready for the MMA.  Normed GEMMs
-// (gain != null): h = bf16(x * r * gain), the RMSNorm output rounded where the decoder layer rounds
-// it.  int8 weights: the value is then multiplied by the row's power-of-two scale and converted to
-// fp16 (exact unless the scaled value falls below the fp16 normal range).
-template <bool W_INT8>
-__device__ __forceinline__ void load_operand(uint4 (&xr)[kXr], const __nv_bfloat16* src, int ld, int M, int K, int kbase,
-                                             const __nv_bfloat16* gain, float rnorm, float xscale, int warp, int g,
-                                             int t) {
-  uint4 gv[kXr];
-#pragma unroll
-  for (int i = 0; i < kXr; ++i) {   // all loads first: one round trip to L2
-    const int k = x_index<W_INT8>(i, kbase, warp, t);
-    xr[i] = make_uint4(0, 0, 0, 0);
-    gv[i] = make_uint4(0, 0, 0, 0);
-    if (k < K) {
-      if (g < M) xr[i] = __ldcg(reinterpret_cast<const uint4*>(src + (size_t)g * ld + k));
-      if (gain != nullptr) gv[i] = __ldg(reinterpret_cast<const uint4*>(gain + k));
-    }
+// Plain bulk copy global -> shared (both addresses and the size multiples of 16 bytes), counted on `bar`.
+__device__ __forceinline__ void bulk_copy_plain(void* smem_dst, const void* gmem_src, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n" ::"r"(
+                   (uint32_t)__cvta_generic_to_shared(smem_dst)),
+               "l"(gmem_src), "r"(bytes), "r"((uint32_t)__cvta_generic_to_shared(bar))
+               : "memory");
+}
+
+// One thread asks for the operand chunk: the M rows (one copy when the chunk is the whole contraction,
+// else one per row) and the norm gain, into the staging buffer.  A bulk copy keeps the whole request in
+// flight at once, which 16-byte loads from 256 threads do not.
+__device__ __forceinline__ void request_operand(unsigned char* x_s, const __nv_bfloat16* src, int ld, int M, int K,
+                                                int kbase, const __nv_bfloat16* gain, uint64_t* xbar) {
+  const uint32_t cbytes = (uint32_t)min(kChunk, K - kbase) * 2;
+  const bool whole = K <= kChunk;
+  asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");   // earlier reads / writes of the buffer come first
+  mbar_arrive_expect_tx(xbar, (uint32_t)M * cbytes + (gain != nullptr ? cbytes : 0u));
+  if (whole) {
+    bulk_copy_plain(x_s, src, (uint32_t)M * cbytes, xbar);
+  } else {
+    for (int m = 0; m < M; ++m) bulk_copy_plain(x_s + m * kXRowBytes, src + (size_t)m * ld + kbase, cbytes, xbar);
   }
-  if (!W_INT8 && gain == nullptr) return;   // bf16 operand as stored
+  if (gain != nullptr) bulk_copy_plain(x_s + kXBytes, gain + kbase, cbytes, xbar);
+}
+
+// The <= 8 operand rows of this warp's share of the chunk, from the staging buffer to registers, one
+// 16-byte piece at a time.  Normed GEMMs: h = bf16(x * r * gain), the RMSNorm output rounded where the
+// decoder layer rounds it.  int8 weights: h times the row's power-of-two scale, as fp16 (exact unless
+// the scaled value falls below the fp16 normal range); the scale is folded into `rs` = r * scale, which
+// commutes with the rounding.  Without a norm rs is the scale alone and the gain is one.
+template <bool W_INT8>
+__device__ __forceinline__ void read_operand(uint4 (&xr)[kXr], const unsigned char* x_s, int M, int K, int kbase,
+                                             bool has_gain, float rs, int warp, int g, int t) {
+  const int pitch = K <= kChunk ? K * 2 : kXRowBytes;
+  const bool convert = W_INT8 || has_gain;
 #pragma unroll
   for (int i = 0; i < kXr; ++i) {
-    uint32_t* w = reinterpret_cast<uint32_t*>(&xr[i]);
-    const __nv_bfloat162* gp = reinterpret_cast<const __nv_bfloat162*>(&gv[i]);
+    const int k = x_index<W_INT8>(i, kbase, warp, t);
+    uint4 xv = make_uint4(0, 0, 0, 0);
+    uint4 gv = make_uint4(0x3f803f80u, 0x3f803f80u, 0x3f803f80u, 0x3f803f80u);   // bf16 ones
+    if (k < K) {
+      if (g < M) xv = *reinterpret_cast<const uint4*>(x_s + g * pitch + (k - kbase) * 2);
+      if (has_gain) gv = *reinterpret_cast<const uint4*>(x_s + kXBytes + (k - kbase) * 2);
+    }
+    if (convert) {
+      uint32_t* w = reinterpret_cast<uint32_t*>(&xv);
+      const __nv_bfloat162* gp = reinterpret_cast<const __nv_bfloat162*>(&gv);
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w[e]));
-      if (gain != nullptr) {
+      for (int e = 0; e < 4; ++e) {
+        const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w[e]));
         const float2 gf = __bfloat1622float2(gp[e]);
-        f.x = bf16_round_f(f.x * rnorm * gf.x);
-        f.y = bf16_round_f(f.y * rnorm * gf.y);
-      }
-      if (W_INT8) {
-        const __half2 h = __floats2half2_rn(f.x * xscale, f.y * xscale);
-        w[e] = *reinterpret_cast<const uint32_t*>(&h);
-      } else {
-        w[e] = pack_bf16(f.x, f.y);
+        const __nv_bfloat162 h = __floats2bfloat162_rn(f.x * rs * gf.x, f.y * rs * gf.y);
+        if (W_INT8) {
+          const float2 hf = __bfloat1622float2(h);
+          const __half2 q = __floats2half2_rn(hf.x, hf.y);
+          w[e] = *reinterpret_cast<const uint32_t*>(&q);
+        } else {
+          w[e] = *reinterpret_cast<const uint32_t*>(&h);
+        }
       }
     }
+    xr[i] = xv;
   }
 }
 
 // One stage = one block [rows][pb bytes].  MMA row g of the tile is block row ra, MMA row g + 8
 // block row rb; the 16-byte pieces of a row are XOR-swizzled by its parity when pb is a multiple
-// of 128 (off_a / off_b are this lane's byte offsets, computed once per tile and piece size).
-// The MMAs of a stage go to separate accumulators so that no MMA waits for the one before it.
+// of 128.  off_a[u] / off_b[u] are this lane's byte offsets for sub-slice u (computed once per tile
+// and piece size).  The four MMAs of a sub-slice go to separate accumulators so that no MMA waits
+// for the one before it.
 template <bool W_INT8>
-__device__ __forceinline__ void consume_stage(const unsigned char* stage, int s, int off_a, int off_b, bool lane_valid,
-                                              const uint4 (&xr)[kXr], float (&acc)[4][4]) {
-  uint4 wa = *reinterpret_cast<const uint4*>(stage + off_a);
-  uint4 wb = *reinterpret_cast<const uint4*>(stage + off_b);
-  if (W_INT8) {
-    // bytes no copy has written convert to finite numbers: they meet zero activations (k beyond K)
-    // or land in accumulator rows that are never stored (rows beyond the tile)
-    const uint4 x0 = xr[2 * s], x1 = xr[2 * s + 1];
-    uint32_t a0, a1, a2, a3;
-    u8x4_to_f16x4(wa.x, a0, a2); u8x4_to_f16x4(wb.x, a1, a3);
-    mma16816_f16(acc[0], a0, a1, a2, a3, x0.x, x0.y);
-    u8x4_to_f16x4(wa.y, a0, a2); u8x4_to_f16x4(wb.y, a1, a3);
-    mma16816_f16(acc[1], a0, a1, a2, a3, x0.z, x0.w);
-    u8x4_to_f16x4(wa.z, a0, a2); u8x4_to_f16x4(wb.z, a1, a3);
-    mma16816_f16(acc[2], a0, a1, a2, a3, x1.x, x1.y);
-    u8x4_to_f16x4(wa.w, a0, a2); u8x4_to_f16x4(wb.w, a1, a3);
-    mma16816_f16(acc[3], a0, a1, a2, a3, x1.z, x1.w);
-  } else {
-    if (!lane_valid) { wa = make_uint4(0, 0, 0, 0); wb = make_uint4(0, 0, 0, 0); }  // stale bytes may be NaN patterns
-    const uint4 x0 = xr[s];
-    mma16816_bf16(acc[0], wa.x, wb.x, wa.y, wb.y, x0.x, x0.y);
-    mma16816_bf16(acc[1], wa.z, wb.z, wa.w, wb.w, x0.z, x0.w);
+__device__ __forceinline__ void consume_stage(const unsigned char* stage, int s, const int (&off_a)[kSub],
+                                              const int (&off_b)[kSub], unsigned valid_mask, const uint4 (&xr)[kXr],
+                                              float (&acc)[4][4]) {
+  uint4 wa[kSub], wb[kSub];
+#pragma unroll
+  for (int u = 0; u < kSub; ++u) {
+    wa[u] = *reinterpret_cast<const uint4*>(stage + off_a[u]);
+    wb[u] = *reinterpret_cast<const uint4*>(stage + off_b[u]);
+  }
+#pragma unroll
+  for (int u = 0; u < kSub; ++u) {
+    if (W_INT8) {
+      // bytes no copy has written convert to finite numbers: they meet zero activations (k beyond K)
+      // or land in accumulator rows that are never stored (rows beyond the tile)
+      const uint4 x0 = xr[2 * (s * kSub + u)], x1 = xr[2 * (s * kSub + u) + 1];
+      uint32_t a0, a1, a2, a3;
+      u8x4_to_f16x4(wa[u].x, a0, a2); u8x4_to_f16x4(wb[u].x, a1, a3);
+      mma16816_f16(acc[0], a0, a1, a2, a3, x0.x, x0.y);
+      u8x4_to_f16x4(wa[u].y, a0, a2); u8x4_to_f16x4(wb[u].y, a1, a3);
+      mma16816_f16(acc[1], a0, a1, a2, a3, x0.z, x0.w);
+      u8x4_to_f16x4(wa[u].z, a0, a2); u8x4_to_f16x4(wb[u].z, a1, a3);
+      mma16816_f16(acc[2], a0, a1, a2, a3, x1.x, x1.y);
+      u8x4_to_f16x4(wa[u].w, a0, a2); u8x4_to_f16x4(wb[u].w, a1, a3);
+      mma16816_f16(acc[3], a0, a1, a2, a3, x1.z, x1.w);
+    } else {
+      if (!((valid_mask >> u) & 1u)) { wa[u] = make_uint4(0, 0, 0, 0); wb[u] = make_uint4(0, 0, 0, 0); }  // stale bytes may be NaN patterns
+      const uint4 x0 = xr[s * kSub + u];
+      mma16816_bf16(acc[2 * (u & 1)], wa[u].x, wb[u].x, wa[u].y, wb[u].y, x0.x, x0.y);
+      mma16816_bf16(acc[2 * (u & 1) + 1], wa[u].z, wb[u].z, wa[u].w, wb[u].w, x0.z, x0.w);
+    }
   }
 }
 
-// byte offset, inside a block of pitch pb, of the 16 bytes lane (warp, t) reads from block row r
-__device__ __forceinline__ int block_offset(int r, int pb, int warp, int t) {
-  int chunk = warp * 4 + t;
+// byte offset, inside a block of pitch pb, of the 16 bytes lane (warp, t) reads from block row r in sub-slice u
+__device__ __forceinline__ int block_offset(int r, int pb, int warp, int u, int t) {
+  int chunk = (warp * kWarpBytes + u * 64) / 16 + t;
   if ((pb & 127) == 0) chunk ^= (r & 1) << 2;
   return r * pb + chunk * 16;
 }
@@ -454,12 +533,17 @@ struct GemmPhase {
   static constexpr int kElemBytes = W_INT8 ? 1 : 2;
   static constexpr int kStageElems = kRowBytes / kElemBytes;
   static constexpr int SPC = kChunk / kStageElems;   // stages per chunk: 4 (int8) or 8 (bf16)
-  static_assert(kCT == GT * 128, "one epilogue element per consumer thread and tile group");
+  static constexpr int kItems = GT * 128 / kCT;   // epilogue elements per consumer thread and tile group
+  static_assert(kItems * kCT == GT * 128 && kCT % 128 == 0, "epilogue elements divide evenly; a thread keeps its operand row");
 
   __device__ __forceinline__ static bool run(const MegaParams& p, int job, const Pipe& pipe, int& slot_io,
-                                             uint32_t& phase_io, float* red, float* misc, int cta, int ncta) {
+                                             uint32_t& phase_io, float* red, float* misc, unsigned char* x_s, uint64_t* xbar,
+                                             uint32_t& xphase, int cta, int ncta) {
     int slot = slot_io;
     uint32_t phase = phase_io;
+#ifdef QUASAR_GEMM_TIMER
+    unsigned tacc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+#endif
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
     const JobView v = job_view<W_INT8>(p.jobs, job, cta, ncta);
     const MegaJob jb = p.jobs[job];
@@ -469,69 +553,108 @@ struct GemmPhase {
     const __nv_bfloat16* xsrc = jb.kind == kJobO ? p.attn : (jb.kind == kJobDown ? p.act : p.x);
     const int ld = jb.K;
 
-    // Per-row factors of the operand, computed by every warp for itself (no CTA barrier, one round
-    // trip to L2).  Normed GEMMs: the RMSNorm factor from the per-CTA sums of squares that the phase
-    // which wrote x left behind, added in a fixed order; the fp16 scale is the job's static one
-    // (|h| <= sqrt(K) * max|gain|).  Other GEMMs with int8 weights: a power-of-two scale from the
-    // row maximum gathered while the operand was written.
-#ifdef QUASAR_GEMM_TIMER
-    const long long c_f0 = clock64();
+    // The operand of the first chunk and the per-row factors, all in ONE round trip to L2: the
+    // loads of the operand, of the gains and of the statistics are issued together.  Normed GEMMs:
+    // the RMSNorm factor comes from the per-CTA sums of squares that the phase which wrote x left
+    // behind (each warp adds its share of the CTAs, the shares meet in shared memory: a fixed order);
+    // the fp16 scale is the job's static one (|h| <= sqrt(K) * max|gain|).  Other GEMMs with int8
+    // weights: a power-of-two scale from the row maximum gathered while the operand was written.
+    TL_DECL
+#ifdef QUASAR_TIMELINE
+    __shared__ long long s_tl2[16][40];
+    __shared__ int tl2_n[16];
+    if (threadIdx.x < 16) tl2_n[threadIdx.x] = 0;
+    cbar();
 #endif
-    float rnorm = 1.f, xscale = 1.f, inv = 1.f;
-    if (normed) {
-      float ss = 0.f;
-#pragma unroll 8
-      for (int c = t; c < ncta; c += 4) ss += __ldcg(p.ss_part + c * 8 + g);
-      ss += __shfl_xor_sync(0xffffffffu, ss, 1);
-      ss += __shfl_xor_sync(0xffffffffu, ss, 2);
-      rnorm = 1.0f / sqrtf(ss / (float)jb.K + p.rms_eps);
-      if (W_INT8) { xscale = jb.xscale; inv = 1.0f / xscale; }
-    } else if (W_INT8) {
-      const float mx = __uint_as_float(__ldcg(p.amax_buf + job * 8 + g));
-      if (mx > 32768.f && mx < 3.0e38f) {
-        int e;
-        (void)frexpf(mx, &e);               // mx = f * 2^e, f in [0.5, 1)
-        xscale = ldexpf(1.f, 15 - e);       // scaled row maximum <= 2^15
-        inv = ldexpf(1.f, e - 15);
-      }
-    }
-    if (warp == 0 && t == 0) misc[kMiscInvScale + g] = inv;   // read in the epilogues, behind a CTA barrier
-
-#ifdef QUASAR_GEMM_TIMER
-    if (threadIdx.x == 0 && rnorm != 123.f && g_clk_on) g_gemm_clk[blockIdx.x][1] += clock64() - c_f0;
+#ifdef QUASAR_TIMELINE
+#ifndef QUASAR_TL_KIND
+#define QUASAR_TL_KIND 4
 #endif
+    const bool tl_on = jb.kind == QUASAR_TL_KIND && job >= p.n_jobs - 5;
+#endif
+    TL_MARK();
     uint4 xr[kXr];
-    bool have_x = false;
+    bool have_x = false, first = true;
+    float rs = 1.f;   // RMSNorm factor times the fp16 scale of the operand row
     float ss_run = 0.f;   // threads 0..7 (o / down): sum of squares of the row of x this CTA has written
+    float best = -INFINITY;   // LM head: this thread's running arg-max over the elements it finishes
+    int best_i = 0x7fffffff;
 
     for (int tg = 0; tg < v.ngroups; ++tg) {
       const int gt = min(GT, v.tiles - tg * GT);
-      // The element this thread finishes in the group's epilogue; its step sizes and residual are
-      // fetched now so that the epilogue does not wait for L2.
-      const int e_tile = jb.kind == kJobGateUp ? (int)threadIdx.x >> 6 : (int)threadIdx.x >> 7;
-      const int e_col = jb.kind == kJobGateUp ? ((int)threadIdx.x >> 3) & 7 : ((int)threadIdx.x >> 4) & 7;
-      const int e_row = jb.kind == kJobGateUp ? (int)threadIdx.x & 7 : (int)threadIdx.x & 15;
-      const int e_unit = v.u0 + (tg * GT + e_tile) * v.rows_per_tile + e_row;   // output channel, or gate/up pair
-      const bool e_ok = e_tile < gt && e_unit < v.u1 && e_col < M;
-      float d0 = 1.f, d1 = 1.f, resid = 0.f;
-      if (e_ok) {
-        if (jb.delta != nullptr) {
-          d0 = __ldg(jb.delta + e_unit);
-          if (jb.kind == kJobGateUp) d1 = __ldg(jb.delta + v.units + e_unit);
+      // The elements this thread finishes in the group's epilogue (element e = thread + it * kCT of the
+      // group's GT x 16 x 8); their step sizes and residuals are requested now so that the epilogue
+      // does not wait for them.
+      float d0[kItems], d1[kItems], resid[kItems];
+#pragma unroll
+      for (int it = 0; it < kItems; ++it) {
+        const EpiItem ei = epi_item(jb, v, tg, gt, M, it);
+        d0[it] = d1[it] = 1.f;
+        resid[it] = 0.f;
+        if (ei.ok) {
+          if (jb.delta != nullptr) {
+            d0[it] = ld_early_f32(jb.delta + ei.unit);
+            if (jb.kind == kJobGateUp) d1[it] = ld_early_f32(jb.delta + v.units + ei.unit);
+          }
+          if (residual) resid[it] = ld_early_bf16_cg(p.x + (size_t)ei.col * jb.N + ei.unit);
         }
-        if (residual) resid = __bfloat162float(__ldcg(p.x + (size_t)e_col * jb.N + e_unit));
       }
 
       // Accumulators live for one tile and one chunk; each warp then parks them in its own part of
-      // `red` (summing over the chunks of a long contraction), where the epilogue adds the 16 warps up.
+      // `red` (summing over the chunks of a long contraction), where the epilogue adds the warps up.
 #ifdef QUASAR_GEMM_TIMER
       const long long c_t0 = clock64();
 #endif
       for (int kc = 0; kc < v.nchunks; ++kc) {
         if (!have_x) {
-          GEMM_CLK(4, load_operand<W_INT8>(xr, xsrc, ld, M, jb.K, kc * kChunk, jb.gain, rnorm, xscale, warp, g, t); if (xr[0].x == 0x12345u) slot ^= 0);
-          have_x = (v.nchunks == 1);
+          TL_MARK();
+          // every warp is past its last use of the buffer's other tenants (epilogue / attention end in a CTA barrier)
+          if (threadIdx.x == 0) request_operand(x_s, xsrc, ld, M, jb.K, kc * kChunk, jb.gain, xbar);
+          TL_MARK();
+          if (first) {   // the row factors ride on the same round trip as the first chunk's loads
+            first = false;
+            float rnorm = 1.f, xscale = 1.f, inv = 1.f;
+            if (normed) {
+              const int per_warp = (ncta + NW - 1) / NW;
+              const int c_end = min(ncta, (warp + 1) * per_warp);
+              float ss = 0.f;
+              for (int c = warp * per_warp + t; c < c_end; c += 4) ss += __ldcg(p.ss_part + c * 8 + g);
+              ss += __shfl_xor_sync(0xffffffffu, ss, 1);
+              ss += __shfl_xor_sync(0xffffffffu, ss, 2);
+              if (t == 0) misc[kMiscRowSum + warp * 8 + g] = ss;
+              TL_MARK();
+              cbar();
+              TL_MARK();
+              float tot = 0.f;
+#pragma unroll
+              for (int w = 0; w < NW; ++w) tot += misc[kMiscRowSum + w * 8 + g];
+              rnorm = 1.0f / sqrtf(tot / (float)jb.K + p.rms_eps);
+              if (W_INT8) { xscale = jb.xscale; inv = 1.0f / xscale; }
+            } else if (W_INT8) {
+              const float mx = __uint_as_float(__ldcg(p.amax_buf + job * 8 + g));
+              if (mx > 32768.f && mx < 3.0e38f) {
+                int e;
+                (void)frexpf(mx, &e);               // mx = f * 2^e, f in [0.5, 1)
+                xscale = ldexpf(1.f, 15 - e);       // scaled row maximum <= 2^15
+                inv = ldexpf(1.f, e - 15);
+              }
+            }
+            rs = rnorm * xscale;
+            if (warp == 0 && t == 0) misc[kMiscInvScale + g] = inv;   // read in the epilogues, behind a CTA barrier
+          }
+          {
+            int got = 1;
+            if (lane == 0) got = mbar_wait(xbar, xphase, pipe.abort_flag, pipe.status) ? 1 : 0;
+            got = __shfl_sync(0xffffffffu, got, 0);
+            if (!got) return false;
+            xphase ^= 1u;
+          }
+          TL_MARK();
+          read_operand<W_INT8>(xr, x_s, M, jb.K, kc * kChunk, normed, rs, warp, g, t);
+          cbar();   // every warp has its share: the staging buffer may be refilled
+          TL_MARK();
         }
+        have_x = (v.nchunks == 1);   // a long contraction reloads its chunks for every tile group
         const int kbase = kc * kChunk;
         const int cb = min(kChunk, jb.K - kbase) * kElemBytes;        // bytes of a weight row in this chunk
         const int pb_last = cb - (cb - 1) / kRowBytes * kRowBytes;    // bytes of its last piece
@@ -541,8 +664,14 @@ struct GemmPhase {
           // accumulator rows that are never stored)
           const int ra = g;
           const int rb = v.kind == kJobGateUp ? tile_units(v, tg * GT + tile) + g : g + 8;
-          const int oa_full = block_offset(ra, kRowBytes, warp, t), ob_full = block_offset(rb, kRowBytes, warp, t);
-          const int oa_last = block_offset(ra, pb_last, warp, t), ob_last = block_offset(rb, pb_last, warp, t);
+          int oa_full[kSub], ob_full[kSub], oa_last[kSub], ob_last[kSub];
+#pragma unroll
+          for (int u = 0; u < kSub; ++u) {
+            oa_full[u] = block_offset(ra, kRowBytes, warp, u, t);
+            ob_full[u] = block_offset(rb, kRowBytes, warp, u, t);
+            oa_last[u] = block_offset(ra, pb_last, warp, u, t);
+            ob_last[u] = block_offset(rb, pb_last, warp, u, t);
+          }
           float ch[4][4];
 #pragma unroll
           for (int i = 0; i < 4; ++i) ch[i][0] = ch[i][1] = ch[i][2] = ch[i][3] = 0.f;
@@ -551,16 +680,25 @@ struct GemmPhase {
             const int b0 = s * kRowBytes;
             if (b0 < cb) {
               const bool last = b0 + kRowBytes >= cb;
-              const bool lane_valid = b0 + warp * 64 + t * 16 < cb;
-              bool got;
-              GEMM_CLK(0, got = mbar_wait(pipe.full + slot, phase, pipe.abort_flag, pipe.status));
+              // one lane polls the stage's barrier for the warp; the warp-level barrier then orders the
+              // other lanes' reads after the arrival it has seen
+              int got = 1;
+              if (lane == 0) got = mbar_wait(pipe.full + slot, phase, pipe.abort_flag, pipe.status) ? 1 : 0;
+              got = __shfl_sync(0xffffffffu, got, 0);
               if (!got) return false;
               // a lane past the end of a short piece reads inside the stage (offset < 16 KB) but not its own data
-              const int oa = last ? (lane_valid ? oa_last : 0) : oa_full;
-              const int ob = last ? (lane_valid ? ob_last : 0) : ob_full;
-              GEMM_CLK(3, consume_stage<W_INT8>(pipe.ring + slot * kStageBytes, s, oa, ob, lane_valid, xr, ch);
-                       __syncwarp();
-                       if (lane == 0) mbar_arrive(pipe.empty + slot));
+              int oa[kSub], ob[kSub];
+              unsigned valid_mask = 0;
+#pragma unroll
+              for (int u = 0; u < kSub; ++u) {
+                const bool lane_valid = b0 + warp * kWarpBytes + u * 64 + t * 16 < cb;
+                valid_mask |= (lane_valid ? 1u : 0u) << u;
+                oa[u] = last ? (lane_valid ? oa_last[u] : 0) : oa_full[u];
+                ob[u] = last ? (lane_valid ? ob_last[u] : 0) : ob_full[u];
+              }
+              consume_stage<W_INT8>(pipe.ring + slot * kStageBytes, s, oa, ob, valid_mask, xr, ch);
+              __syncwarp();
+              if (lane == 0) mbar_arrive(pipe.empty + slot);
               if (++slot == kStages) { slot = 0; phase ^= 1u; }
             }
           }
@@ -578,20 +716,53 @@ struct GemmPhase {
         }
       }
 #ifdef QUASAR_GEMM_TIMER
-      if (threadIdx.x == 0 && g_clk_on) g_gemm_clk[blockIdx.x][5] += clock64() - c_t0;
+      tacc[5] += (unsigned)(clock64() - c_t0);
 #endif
+      TL_MARK();
       // ---- cross-warp reduction in a fixed order, then the fused epilogue ----
-      GEMM_CLK(2, cbar();
-               epilogue(p, jb, v, job, e_ok, e_tile, e_row, e_col, e_unit, d0, d1, resid, red, misc);
-               cbar());
+      cbar();
+#pragma unroll
+      for (int it = 0; it < kItems; ++it) {
+        const EpiItem ei = epi_item(jb, v, tg, gt, M, it);
+        epilogue(p, jb, v, job, ei, d0[it], d1[it], resid[it], best, best_i, red, misc);
+      }
+      cbar();
+      TL_MARK();
       if (residual && threadIdx.x < 8) {   // fixed order: tiles of the group, groups of the phase
         for (int tile = 0; tile < gt; ++tile) ss_run += misc[kMiscPart + tile * 8 + threadIdx.x];
       }
     }
     if (residual && threadIdx.x < 8) p.ss_part[cta * 8 + threadIdx.x] = ss_run;
+    if (jb.kind == kJobLm) finish_argmax(best, best_i, misc);
+    TL_MARK();
+    TL_FLUSH();
+#ifdef QUASAR_TIMELINE
+    cbar();
+    if (tl_on && threadIdx.x < 16) for (int i = 0; i < 40; ++i) g_timeline2[blockIdx.x][threadIdx.x][i] = s_tl2[threadIdx.x][i];
+#endif
+#ifdef QUASAR_GEMM_TIMER
+    if (threadIdx.x == 0 && g_clk_on) {
+      for (int i = 0; i < 8; ++i) g_gemm_clk[blockIdx.x][i] += tacc[i];
+    }
+#endif
     slot_io = slot;
     phase_io = phase;
     return true;
+  }
+
+  struct EpiItem {
+    int tile, row, col, unit;   // tile in the group, MMA row, operand row, output channel (or gate/up pair)
+    bool ok;
+  };
+  __device__ __forceinline__ static EpiItem epi_item(const MegaJob& jb, const JobView& v, int tg, int gt, int M, int it) {
+    const int e = (int)threadIdx.x + it * kCT;
+    EpiItem ei;
+    ei.tile = jb.kind == kJobGateUp ? e >> 6 : e >> 7;
+    ei.col = jb.kind == kJobGateUp ? (e >> 3) & 7 : (e >> 4) & 7;
+    ei.row = jb.kind == kJobGateUp ? e & 7 : e & 15;
+    ei.unit = v.u0 + (tg * GT + ei.tile) * v.rows_per_tile + ei.row;
+    ei.ok = ei.tile < gt && ei.unit < v.u1 && ei.col < M;
+    return ei;
   }
 
   __device__ __forceinline__ static float reduce_at(const float* red, int tile, int row, int col) {
@@ -604,9 +775,11 @@ struct GemmPhase {
   // One output element per thread: sum the 16 warps' partials, apply the step size (and the operand's
   // scale), then what the step of the pass asks for.
   __device__ __forceinline__ static void epilogue(const MegaParams& p, const MegaJob& jb, const JobView& v, int job,
-                                                  bool ok, int tile, int row, int col, int unit_idx, float d0, float d1,
-                                                  float resid, const float* red, float* misc) {
+                                                  const EpiItem& ei, float d0, float d1, float resid, float& best,
+                                                  int& best_i, const float* red, float* misc) {
     const int lane = threadIdx.x & 31;
+    const bool ok = ei.ok;
+    const int tile = ei.tile, row = ei.row, col = ei.col, unit_idx = ei.unit;
     const float unit = W_INT8 ? misc[kMiscInvScale + col] : 1.f;
     if (jb.kind == kJobGateUp) {
       // SwiGLU: act = silu(gate) * up, gate and up rounded to bf16 first (they are tensors of the layer)
@@ -626,8 +799,6 @@ struct GemmPhase {
       }
       return;
     }
-    float best = -INFINITY;
-    int best_i = 0x7fffffff;
     float sq = 0.f;
     if (ok) {
       const float val = reduce_at(red, tile, row, col) * unit * d0;
@@ -636,8 +807,8 @@ struct GemmPhase {
         p.qkv[idx] = __float2bfloat16_rn(val);
       } else if (jb.kind == kJobLm) {
         if (p.logits) p.logits[idx] = val;
-        best = val;
-        best_i = unit_idx;
+        // a thread's channels only grow from group to group: on equal values the earlier, lower one stays
+        if (val > best) { best = val; best_i = unit_idx; }
       } else {  // o / down: residual add into the stream
         const __nv_bfloat16 xn = __float2bfloat16_rn(bf16_round_f(val) + resid);
         p.x[idx] = xn;
@@ -651,36 +822,34 @@ struct GemmPhase {
       for (int o = 8; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
       if ((lane & 15) == 0) misc[kMiscPart + tile * 8 + col] = sq;
     }
-    if (jb.kind == kJobLm) {
-      // combine the 16 lanes that share a col (lanes differ in row), then the 4 such groups per col in the CTA
+  }
+
+  // End of the LM head: the CTA's arg-max per operand row from its threads' running ones (lowest
+  // channel on ties).  16 consecutive lanes share a row, as do the threads 128 apart.
+  __device__ __forceinline__ static void finish_argmax(float best, int best_i, float* misc) {
 #pragma unroll
-      for (int o = 8; o > 0; o >>= 1) {
-        const float ob = __shfl_xor_sync(0xffffffffu, best, o);
-        const int oi = __shfl_xor_sync(0xffffffffu, best_i, o);
-        if (ob > best || (ob == best && oi < best_i)) { best = ob; best_i = oi; }
+    for (int o = 8; o > 0; o >>= 1) {
+      const float ob = __shfl_xor_sync(0xffffffffu, best, o);
+      const int oi = __shfl_xor_sync(0xffffffffu, best_i, o);
+      if (ob > best || (ob == best && oi < best_i)) { best = ob; best_i = oi; }
+    }
+    float* cand_v = misc + kMiscCand;
+    int* cand_i = reinterpret_cast<int*>(misc + kMiscCand + 64);
+    if ((threadIdx.x & 15) == 0) {
+      cand_v[threadIdx.x >> 4] = best;
+      cand_i[threadIdx.x >> 4] = best_i;
+    }
+    cbar();
+    if (threadIdx.x < 8) {
+      float bv = -INFINITY;
+      int bi = 0x7fffffff;
+      for (int q = threadIdx.x; q < kCT / 16; q += 8) {
+        const float ov = cand_v[q];
+        const int oi = cand_i[q];
+        if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
       }
-      float* cand_v = misc + kMiscCand;
-      int* cand_i = reinterpret_cast<int*>(misc + kMiscCand + 64);
-      if ((threadIdx.x & 15) == 0) {
-        cand_v[threadIdx.x >> 4] = best;
-        cand_i[threadIdx.x >> 4] = best_i;
-      }
-      cbar();
-      if (threadIdx.x < 8) {
-        float* run_v = misc + kMiscRunV;
-        int* run_i = reinterpret_cast<int*>(misc + kMiscRunI);
-        float bv = run_v[threadIdx.x];
-        int bi = run_i[threadIdx.x];
-        for (int q = 0; q < kCT / 16; ++q) {
-          if (((q & 7) == (int)threadIdx.x)) {
-            const float ov = cand_v[q];
-            const int oi = cand_i[q];
-            if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
-          }
-        }
-        run_v[threadIdx.x] = bv;
-        run_i[threadIdx.x] = bi;
-      }
+      misc[kMiscRunV + threadIdx.x] = bv;
+      reinterpret_cast<int*>(misc + kMiscRunI)[threadIdx.x] = bi;
     }
   }
 };
@@ -714,6 +883,7 @@ __device__ void prep_phase(const MegaParams& p, float* misc, int cta, int ncta) 
   }
   // row maxima of the un-normed GEMM operands start at zero (gathered with atomicMax during the pass)
   for (int i = cta * kCT + threadIdx.x; i < p.n_jobs * 8; i += ncta * kCT) p.amax_buf[i] = 0u;
+  for (int i = cta * kCT + threadIdx.x; i < p.L * p.B * p.Hkv; i += ncta * kCT) p.attn_count[i] = 0u;
   // Embedding rows: CTA m gathers row m and leaves its sum of squares for the first RMSNorm; every
   // CTA leaves a (possibly zero) entry per row, the layout the later phases use too.
   float* wsum = misc + kMiscRowSum;
@@ -779,9 +949,45 @@ __device__ void rope_vec(const __nv_bfloat16* src, const __nv_bfloat16* gain, co
   }
 }
 
+__device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"((uint32_t)__cvta_generic_to_shared(smem)), "l"(gmem)
+               : "memory");
+}
+
+// The attention work items: (sequence, kv head, chunk of kKeyTile keys), item = (b * Hkv + hk) * nchunk + c.
+// Called before the grid barrier that ends the qkv GEMM: starts copying the part of this CTA's first
+// K/V tile that is already in the cache (keys before seq_len), so that the copy's latency hides
+// behind the barrier.  The tiles alias the GEMM's reduction buffer, which is free by then.
 template <int D>
-__device__ __noinline__ void attention_phase(const MegaParams& p, int layer, __nv_bfloat16* k_s, __nv_bfloat16* v_s,
-                                __nv_bfloat16* q_s, int cta, int ncta) {
+__device__ __forceinline__ void attention_prefetch(const MegaParams& p, int layer, __nv_bfloat16* k_s,
+                                                   __nv_bfloat16* v_s, int cta) {
+  constexpr int kStride = D + 8;
+  const int n_items = p.B * p.Hkv * p.attn_nchunk;
+  if (cta < n_items) {
+    const int c = cta % p.attn_nchunk;
+    const int hk = (cta / p.attn_nchunk) % p.Hkv;
+    const int b = cta / (p.attn_nchunk * p.Hkv);
+    if (p.bi.valid[b]) {
+      const int P = p.seq_len[b];
+      const int key_begin = c * kKeyTile;
+      const int rows = min(kKeyTile, P - key_begin);
+      const size_t layer_stride = (size_t)p.kv_batch * p.Hkv * (size_t)p.s_max * D;
+      const size_t head_off = (size_t)layer * layer_stride + ((size_t)b * p.Hkv + hk) * (size_t)p.s_max * D;
+      const __nv_bfloat16* kbase = p.k_cache + head_off + (size_t)key_begin * D;
+      const __nv_bfloat16* vbase = p.v_cache + head_off + (size_t)key_begin * D;
+      for (int i = threadIdx.x; i < rows * (D / 8); i += kCT) {
+        const int key = i / (D / 8), ch = i % (D / 8);
+        cp_async16(k_s + key * kStride + ch * 8, kbase + (size_t)key * D + ch * 8);
+        cp_async16(v_s + key * kStride + ch * 8, vbase + (size_t)key * D + ch * 8);
+      }
+    }
+  }
+  asm volatile("cp.async.commit_group;\n" ::: "memory");
+}
+
+template <int D>
+__device__ __noinline__ void attention_phase(const MegaParams& p, int layer, bool want_amax, __nv_bfloat16* k_s,
+                                             __nv_bfloat16* v_s, __nv_bfloat16* q_s, float* misc, int cta, int ncta) {
   constexpr int kStride = D + 8;
   constexpr int kDSteps = D / 16;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
@@ -792,11 +998,28 @@ __device__ __noinline__ void attention_phase(const MegaParams& p, int layer, __n
   __nv_bfloat16* kc_l = p.k_cache + (size_t)layer * layer_stride;
   __nv_bfloat16* vc_l = p.v_cache + (size_t)layer * layer_stride;
   const int n_items = p.B * p.Hkv * p.attn_nchunk;
+  int* last_flag = reinterpret_cast<int*>(misc + kMiscFlag);
+#ifdef QUASAR_PHASE_TIMER
+  __shared__ long long s_attn_clk[8];
+  if (threadIdx.x < 8) s_attn_clk[threadIdx.x] = 0;
+  cbar();
+  long long at0 = clock64();
+#endif
+
+  // rows that take no part (beyond a block's length, or of a skipped sequence) give zero attention output
+  for (int m = cta; m < p.M; m += ncta) {
+    const int b = m / p.T_max, i = m % p.T_max;
+    if (!p.bi.valid[b] || i >= p.block_len[b]) {
+      uint4* dst = reinterpret_cast<uint4*>(p.attn + (size_t)m * p.Hq * D);
+      for (int j = threadIdx.x; j < p.Hq * D / 8; j += kCT) dst[j] = make_uint4(0, 0, 0, 0);
+    }
+  }
 
   for (int item = cta; item < n_items; item += ncta) {
     const int c = item % p.attn_nchunk;
     const int hk = (item / p.attn_nchunk) % p.Hkv;
     const int b = item / (p.attn_nchunk * p.Hkv);
+    const bool prefetched = item == cta;   // attention_prefetch has started the cached rows of this tile
     if (!p.bi.valid[b]) continue;
     const int T = p.block_len[b], P = p.seq_len[b];
     const int Lk = P + T;
@@ -829,9 +1052,12 @@ __device__ __noinline__ void attention_phase(const MegaParams& p, int layer, __n
       }
     }
     cbar();  // block-level visibility of the K/V rows just stored and of q_s
+    ATTN_T(0);
 
-    // (b) stage the K / V tile (zero beyond the end of the sequence)
-    for (int i = threadIdx.x; i < kKeyTile * (D / 8); i += kCT) {
+    // (b) stage the K / V tile (zero beyond the end of the sequence); cached rows of a prefetched
+    //     tile are already on their way
+    const int first_row = prefetched ? max(0, min(kKeyTile, P - key_begin)) : 0;
+    for (int i = first_row * (D / 8) + threadIdx.x; i < kKeyTile * (D / 8); i += kCT) {
       const int key = i / (D / 8), ch = i % (D / 8);
       uint4 kv4 = make_uint4(0, 0, 0, 0), vv4 = make_uint4(0, 0, 0, 0);
       if (key_begin + key < key_end) {
@@ -841,7 +1067,9 @@ __device__ __noinline__ void attention_phase(const MegaParams& p, int layer, __n
       *reinterpret_cast<uint4*>(k_s + key * kStride + ch * 8) = kv4;
       *reinterpret_cast<uint4*>(v_s + key * kStride + ch * 8) = vv4;
     }
+    asm volatile("cp.async.wait_all;\n" ::: "memory");
     cbar();
+    ATTN_T(1);
 
     // (c) one warp per 16 query rows
     const int row_tiles = (R + 15) / 16;
@@ -909,7 +1137,7 @@ __device__ __noinline__ void attention_phase(const MegaParams& p, int layer, __n
       }
       const size_t slot = (((size_t)b * p.Hkv + hk) * p.attn_nchunk + c) * p.attn_rpad;
       // O = P V in two halves of the head dimension (keeps the accumulators within the register budget)
-#pragma unroll
+#pragma unroll 1
       for (int half = 0; half < 2; ++half) {
         float o[D / 16][4];
 #pragma unroll
@@ -953,65 +1181,95 @@ __device__ __noinline__ void attention_phase(const MegaParams& p, int layer, __n
         }
       }
     }
-  }
-}
 
-// merge the chunk partials of every (row, query head) in chunk order: one warp per item
-template <int D>
-__device__ __noinline__ void merge_phase(const MegaParams& p, int layer, bool want_amax, int cta, int ncta) {
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  constexpr int kPer = D / 32;
-  const int G = p.Hq / p.Hkv;
-  const int n_items = p.M * p.Hq;
-  for (int item = cta * NW + warp; item < n_items; item += ncta * NW) {
-    const int hq = item % p.Hq, m = item / p.Hq;
-    const int b = m / p.T_max, i = m % p.T_max;
-    __nv_bfloat16* dst = p.attn + (size_t)m * p.Hq * D + (size_t)hq * D;
-    if (!p.bi.valid[b] || i >= p.block_len[b]) {
-#pragma unroll
-      for (int e = 0; e < kPer; ++e) dst[lane * kPer + e] = __float2bfloat16_rn(0.f);
-      continue;
-    }
-    const int hk = hq / G, r = i * G + (hq % G);
-    const int Lk = p.seq_len[b] + p.block_len[b];
+    // (d) The CTA that finishes the last chunk of this (sequence, kv head) merges all of its chunks, in
+    //     chunk order, so the result does not depend on which CTA that is.
     const int nch = (Lk + kKeyTile - 1) / kKeyTile;
-    const size_t slot0 = ((size_t)b * p.Hkv + hk) * p.attn_nchunk * p.attn_rpad;
-    float mx = -INFINITY;
-    for (int c = lane; c < nch; c += 32) mx = fmaxf(mx, __ldcg(p.ml_part + (slot0 + (size_t)c * p.attn_rpad + r) * 2));
+    ATTN_T(2);
+    __threadfence();   // this CTA's partials are visible before its arrival is
+    cbar();
+    if (threadIdx.x == 0) {
+      const unsigned old = atomicAdd(p.attn_count + (size_t)layer * p.B * p.Hkv + b * p.Hkv + hk, 1u);
+      *last_flag = (old == (unsigned)(nch - 1));
+    }
+    cbar();
+    ATTN_T(3);
+    if (*last_flag) {
+      __threadfence();
+      ATTN_T(5);
+      const size_t slot0 = ((size_t)b * p.Hkv + hk) * p.attn_nchunk * p.attn_rpad;
+      // half a warp per query row: lane l16 owns D/16 consecutive output dimensions
+      constexpr int kV4 = D / 64;              // float4 loads per lane and chunk
+      constexpr int kBlk = 8;                  // chunks fetched together
+      const int hsel = lane >> 4, l16 = lane & 15;
+#pragma unroll 1
+      for (int r0 = warp * 2; r0 < R; r0 += NW * 2) {
+        const int r = r0 + hsel;
+        const bool rv = r < R;
+        const int rr = rv ? r : R - 1;
+        float mx = -INFINITY;
+        for (int cc = l16; cc < nch; cc += 16)
+          mx = fmaxf(mx, __ldcg(p.ml_part + (slot0 + (size_t)cc * p.attn_rpad + rr) * 2));
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-    float acc[kPer];
+        for (int o = 8; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        float acc[4 * kV4];
 #pragma unroll
-    for (int e = 0; e < kPer; ++e) acc[e] = 0.f;
-    float den = 0.f;
-    for (int c = 0; c < nch; ++c) {
-      const size_t s = slot0 + (size_t)c * p.attn_rpad + r;
-      const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.ml_part + s * 2));
-      if (ml.x == -INFINITY) continue;
-      const float w = exp2f(ml.x - mx);
-      den += w * ml.y;
-      if constexpr (kPer == 4) {
-        const float4 ov = __ldcg(reinterpret_cast<const float4*>(p.o_part + s * D) + lane);
-        acc[0] += w * ov.x; acc[1] += w * ov.y; acc[2] += w * ov.z; acc[kPer - 1] += w * ov.w;
-      } else {
-        const float2 ov = __ldcg(reinterpret_cast<const float2*>(p.o_part + s * D) + lane);
-        acc[0] += w * ov.x; acc[kPer - 1] += w * ov.y;
+        for (int e = 0; e < 4 * kV4; ++e) acc[e] = 0.f;
+        float den = 0.f;
+#pragma unroll 1
+        for (int c0 = 0; c0 < nch; c0 += kBlk) {
+          float4 ov[kBlk][kV4];
+#pragma unroll
+          for (int j = 0; j < kBlk; ++j) {
+            const size_t sidx = slot0 + (size_t)min(c0 + j, nch - 1) * p.attn_rpad + rr;
+#pragma unroll
+            for (int q = 0; q < kV4; ++q) ov[j][q] = __ldcg(reinterpret_cast<const float4*>(p.o_part + sidx * D) + l16 * kV4 + q);
+          }
+          float2 ml = make_float2(-INFINITY, 0.f);
+          if (l16 < kBlk && c0 + l16 < nch)
+            ml = __ldcg(reinterpret_cast<const float2*>(p.ml_part + (slot0 + (size_t)(c0 + l16) * p.attn_rpad + rr) * 2));
+          const float w_lane = ml.x == -INFINITY ? 0.f : exp2f(ml.x - mx);
+#pragma unroll
+          for (int j = 0; j < kBlk; ++j) {   // chunk order; lane j of this half holds chunk c0 + j's weight
+            const float w = __shfl_sync(0xffffffffu, w_lane, (lane & 16) | j);
+            den += w * __shfl_sync(0xffffffffu, ml.y, (lane & 16) | j);
+#pragma unroll
+            for (int q = 0; q < kV4; ++q) {
+              acc[4 * q + 0] += w * ov[j][q].x; acc[4 * q + 1] += w * ov[j][q].y;
+              acc[4 * q + 2] += w * ov[j][q].z; acc[4 * q + 3] += w * ov[j][q].w;
+            }
+          }
+        }
+        const float inv = 1.0f / den;
+        const int i = rr / G, hq = hk * G + (rr % G);
+        const int m = b * p.T_max + i;
+        float amax = 0.f;
+        uint32_t packed[2 * kV4];
+#pragma unroll
+        for (int e = 0; e < 2 * kV4; ++e) {
+          const __nv_bfloat162 pr = __floats2bfloat162_rn(acc[2 * e] * inv, acc[2 * e + 1] * inv);
+          packed[e] = *reinterpret_cast<const uint32_t*>(&pr);
+          const float2 back = __bfloat1622float2(pr);
+          amax = fmaxf(amax, fmaxf(fabsf(back.x), fabsf(back.y)));
+        }
+        if (rv) {
+          __nv_bfloat16* dst = p.attn + (size_t)m * p.Hq * D + (size_t)hq * D + l16 * (D / 16);
+          if constexpr (kV4 == 2) *reinterpret_cast<uint4*>(dst) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+          else *reinterpret_cast<uint2*>(dst) = make_uint2(packed[0], packed[1]);
+        }
+        if (want_amax) {   // row maximum of the o projection's operand
+#pragma unroll
+          for (int o = 8; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+          if (l16 == 0 && rv && amax > 0.f) atomicMax(p.amax_buf + (4 * layer + 1) * 8 + m, __float_as_uint(amax));
+        }
       }
     }
-    const float inv = 1.0f / den;
-    float amax = 0.f;
-#pragma unroll
-    for (int e = 0; e < kPer; ++e) {
-      const __nv_bfloat16 ov = __float2bfloat16_rn(acc[e] * inv);
-      dst[lane * kPer + e] = ov;
-      amax = fmaxf(amax, fabsf(__bfloat162float(ov)));
-    }
-    if (want_amax) {   // row maximum of the o projection's operand
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
-      if (lane == 0 && amax > 0.f) atomicMax(p.amax_buf + (4 * layer + 1) * 8 + m, __float_as_uint(amax));
-    }
   }
+  ATTN_T(4);
+#ifdef QUASAR_PHASE_TIMER
+  if (threadIdx.x == 0) for (int i = 0; i < 8; ++i) g_attn_clk[blockIdx.x][i] += s_attn_clk[i];
+#endif
+  asm volatile("cp.async.wait_all;\n" ::: "memory");   // a prefetch whose item was skipped has landed before the tiles are reused
 }
 
 // final phase on CTA 0: arg-max over the per-CTA candidates, then greedy acceptance
@@ -1068,15 +1326,16 @@ __global__ void __launch_bounds__(kThreads, 1) verify_megakernel(const MegaParam
   extern __shared__ __align__(128) unsigned char smem[];
   const int cta = blockIdx.x, ncta = gridDim.x;
   const int warp = threadIdx.x >> 5;
-  unsigned char* uni = smem + kRingBytes;
-  float* red = reinterpret_cast<float*>(uni);
-  __nv_bfloat16* k_s = reinterpret_cast<__nv_bfloat16*>(uni);
-  __nv_bfloat16* v_s = reinterpret_cast<__nv_bfloat16*>(uni + kKvTileBytes);
-  __nv_bfloat16* q_s = reinterpret_cast<__nv_bfloat16*>(uni + kUnionBytes);
-  float* misc = reinterpret_cast<float*>(uni + kUnionBytes + kQTileBytes);
+  float* red = reinterpret_cast<float*>(smem + kRingBytes);
+  unsigned char* x_s = smem + kRingBytes + kRedBytes;   // operand staging; the attention tiles live in the same bytes
+  __nv_bfloat16* k_s = reinterpret_cast<__nv_bfloat16*>(x_s);
+  __nv_bfloat16* v_s = reinterpret_cast<__nv_bfloat16*>(x_s + kKvTileBytes);
+  __nv_bfloat16* q_s = reinterpret_cast<__nv_bfloat16*>(x_s + 2 * kKvTileBytes);
+  float* misc = reinterpret_cast<float*>(x_s + kStageBufBytes);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + kMiscAbort);
   uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<unsigned char*>(misc) + kMiscBarBytes);
   Pipe pipe{smem, bars, bars + kStages, abort_flag, p.status};
+  uint64_t* xbar = bars + 2 * kStages;   // the operand's bulk copies have landed
 
   if (threadIdx.x == 0) {
     *abort_flag = 0;
@@ -1084,6 +1343,7 @@ __global__ void __launch_bounds__(kThreads, 1) verify_megakernel(const MegaParam
       mbar_init(pipe.full + s, 1);     // the producer's arrive.expect_tx; the bytes complete the phase
       mbar_init(pipe.empty + s, NW);   // one arrival per consumer warp
     }
+    mbar_init(xbar, 1);
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
   }
   if (threadIdx.x < 8) {  // running arg-max of this CTA
@@ -1098,7 +1358,7 @@ __global__ void __launch_bounds__(kThreads, 1) verify_megakernel(const MegaParam
   }
 
   int slot = 0;
-  uint32_t phase = 0;
+  uint32_t phase = 0, xphase = 0;
   GridSync gs{p.barrier, p.status, (unsigned)ncta, 0u, abort_flag};
   bool ok = true;
 #ifdef QUASAR_PHASE_TIMER
@@ -1112,17 +1372,14 @@ __global__ void __launch_bounds__(kThreads, 1) verify_megakernel(const MegaParam
   PHASE_MARK();
   // the GEMMs of the pass in order (qkv, o, gate+up, down per layer, then the LM head); attention follows every qkv
   for (int job = 0; job < p.n_jobs && ok; ++job) {
-    if (!(ok = GemmPhase<W_INT8>::run(p, job, pipe, slot, phase, red, misc, cta, ncta))) break;
+    if (!(ok = GemmPhase<W_INT8>::run(p, job, pipe, slot, phase, red, misc, x_s, xbar, xphase, cta, ncta))) break;
+    if ((job & 3) == 0 && job != p.n_jobs - 1) attention_prefetch<D>(p, job >> 2, k_s, v_s, cta);
     PHASE_MARK();
     if (job == p.n_jobs - 1) break;   // the LM head is followed by the candidate exchange below
     if (!(ok = gs.sync())) break;
     PHASE_MARK();
     if ((job & 3) == 0) {
-      attention_phase<D>(p, job >> 2, k_s, v_s, q_s, cta, ncta);
-      PHASE_MARK();
-      if (!(ok = gs.sync())) break;
-      PHASE_MARK();
-      merge_phase<D>(p, job >> 2, W_INT8, cta, ncta);
+      attention_phase<D>(p, job >> 2, W_INT8, k_s, v_s, q_s, misc, cta, ncta);
       PHASE_MARK();
       if (!(ok = gs.sync())) break;
       PHASE_MARK();
@@ -1208,6 +1465,20 @@ extern "C" int quasar_debug_phase_marks(long long* clk_host, int* n_host) {
   if (cudaMemcpyFromSymbol(clk_host, g_phase_clk, sizeof(long long) * 160 * kMaxMarks) != cudaSuccess) return -1;
   if (cudaMemcpyFromSymbol(n_host, g_phase_n, sizeof(int) * 160) != cudaSuccess) return -1;
   return kMaxMarks;
+}
+#ifdef QUASAR_TIMELINE
+extern "C" int quasar_debug_timeline2(long long* host) {
+  if (cudaMemcpyFromSymbol(host, g_timeline2, sizeof(long long) * 160 * 16 * 40) != cudaSuccess) return -1;
+  return 0;
+}
+extern "C" int quasar_debug_timeline(long long* host) {
+  if (cudaMemcpyFromSymbol(host, g_timeline, sizeof(long long) * 160 * 256) != cudaSuccess) return -1;
+  return 0;
+}
+#endif
+extern "C" int quasar_debug_attn_clocks(long long* host) {
+  if (cudaMemcpyFromSymbol(host, g_attn_clk, sizeof(long long) * 160 * 8) != cudaSuccess) return -1;
+  return 0;
 }
 extern "C" int quasar_debug_gemm_clocks(long long* host, int reset) {
   if (cudaMemcpyFromSymbol(host, g_gemm_clk, sizeof(long long) * 160 * 8) != cudaSuccess) return -1;

@@ -5,7 +5,7 @@
 
 namespace quasar {
 
-constexpr int kMegaWarps = 16;
+constexpr int kMegaWarps = 8;
 
 enum MegaJobKind { kJobQkv = 0, kJobO = 1, kJobGateUp = 2, kJobDown = 3, kJobLm = 4 };
 
@@ -43,6 +43,7 @@ struct MegaParams {
   float* cand_val;          // [grid][8] per-CTA arg-max candidates
   int* cand_idx;
   float* ss_part;           // [grid][8] per-CTA sums of squares of the rows of x, left by the phase that wrote x
+  unsigned* attn_count;     // [L][B*Hkv] chunks of a (sequence, kv head) whose attention partial is complete
   unsigned* amax_buf;       // [n_jobs][8] row maxima (float bits) of the un-normed GEMM operands
   unsigned* barrier;        // zeroed before every launch
   int32_t *accept_len, *bonus, *accept_path, *status;
