@@ -54,7 +54,7 @@ constexpr int kSub = kWarpBytes / 64;        // 64-byte sub-slices of it: four l
 constexpr int kXr = 8 * kSub;                // 16-byte registers holding this thread's share of the operand chunk
 constexpr int GT = 4;                      // 16-row tiles accumulated together before a reduction
 constexpr int kKeyTile = 64;
-constexpr int kMaxRowsAttn = 64;           // query rows (heads-in-group x block rows) per kv head
+constexpr int kMaxRowsAttn = 32;           // query rows (heads-in-group x block rows) per kv head
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr unsigned long long kWaitBudgetNs = 2000000000ull;  // every device-side wait gives up after 2 s
 
@@ -63,7 +63,9 @@ constexpr int kRingBytes = kStages * kStageBytes;                        // 1310
 constexpr int kRedBytes = NW * GT * 128 * 4;                             // 32768
 constexpr int kKvTileBytes = kKeyTile * (128 + 8) * 2;                   // 17408 (D = 128)
 constexpr int kQTileBytes = kMaxRowsAttn * (128 + 8) * 2;                // 17408
-constexpr int kAttnBytes = 2 * kKvTileBytes + kQTileBytes;               // K, V and Q tiles of the attention phase
+constexpr int kOTileBytes = kMaxRowsAttn * 128 * 4;                      // 16384: a CTA's partial output before it is stored
+constexpr int kMlTileBytes = kMaxRowsAttn * 8;                           // its row maxima and sums
+constexpr int kAttnBytes = 2 * kKvTileBytes + kQTileBytes + kOTileBytes + kMlTileBytes;   // tiles of the attention phase
 constexpr int kMiscBytes = 2048;
 // The operand of a GEMM phase (<= 8 rows x one chunk, bf16) and its norm gain land in a staging buffer by
 // bulk copy before they go to registers.  The attention tiles share that buffer: the two are never alive
@@ -79,7 +81,7 @@ static_assert(kSmemBytes <= 227 * 1024, "shared memory budget of one SM");
 // misc region (floats): [0,128) per-warp row sums, [128,136) running arg-max values, [136,144) its
 // indices, [144,152) 1/scale of the operand rows, [152,184) per-tile sums of squares, [200] abort flag, [256,512) candidates / per-warp
 // row maxima, byte 1536.. the mbarriers.
-constexpr int kMiscRowSum = 0, kMiscRunV = 128, kMiscRunI = 136, kMiscInvScale = 144, kMiscPart = 152, kMiscFlag = 190, kMiscAbort = 200,
+constexpr int kMiscRowSum = 0, kMiscRunV = 128, kMiscRunI = 136, kMiscInvScale = 144, kMiscPart = 152, kMiscFlag = 190, kMiscRs = 192, kMiscAbort = 200,
               kMiscCand = 256, kMiscBarBytes = 1536;   // 2 kStages + 1 barriers of 8 bytes
 
 __device__ __forceinline__ void mma16816_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
@@ -424,6 +426,14 @@ __device__ __forceinline__ void bulk_copy_plain(void* smem_dst, const void* gmem
                : "memory");
 }
 
+// Bulk store shared -> global (both addresses and the size multiples of 16 bytes); completion through the
+// issuing thread's bulk group.
+__device__ __forceinline__ void bulk_store(void* gmem_dst, const void* smem_src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;\n" ::"l"(gmem_dst),
+               "r"((uint32_t)__cvta_generic_to_shared(smem_src)), "r"(bytes)
+               : "memory");
+}
+
 // One thread asks for the operand chunk: the M rows (one copy when the chunk is the whole contraction,
 // else one per row) and the norm gain, into the staging buffer.  A bulk copy keeps the whole request in
 // flight at once, which 16-byte loads from 256 threads do not.
@@ -441,43 +451,53 @@ __device__ __forceinline__ void request_operand(unsigned char* x_s, const __nv_b
   if (gain != nullptr) bulk_copy_plain(x_s + kXBytes, gain + kbase, cbytes, xbar);
 }
 
-// The <= 8 operand rows of this warp's share of the chunk, from the staging buffer to registers, one
-// 16-byte piece at a time.  Normed GEMMs: h = bf16(x * r * gain), the RMSNorm output rounded where the
+// The staged operand chunk is converted where it lies, every thread taking 16-byte pieces in turn (a
+// rolled loop: little code).  Normed GEMMs: h = bf16(x * r * gain), the RMSNorm output rounded where the
 // decoder layer rounds it.  int8 weights: h times the row's power-of-two scale, as fp16 (exact unless
-// the scaled value falls below the fp16 normal range); the scale is folded into `rs` = r * scale, which
-// commutes with the rounding.  Without a norm rs is the scale alone and the gain is one.
+// the scaled value falls below the fp16 normal range); the scale is folded into rs[row] = r * scale,
+// which commutes with the rounding.  Without a norm rs is the scale alone and the gain is one.
+template <bool W_INT8>
+__device__ __forceinline__ void convert_staged(unsigned char* x_s, int M, int K, int kbase, bool has_gain,
+                                               const float* rs_row) {
+  const int per_row = min(kChunk, K - kbase) / 8;          // 16-byte pieces of a row
+  const int pitch = K <= kChunk ? K * 2 : kXRowBytes;
+#pragma unroll 2
+  for (int idx = threadIdx.x; idx < M * per_row; idx += kCT) {
+    const int row = idx / per_row, c = idx - row * per_row;
+    uint4* px = reinterpret_cast<uint4*>(x_s + row * pitch + c * 16);
+    uint4 xv = *px;
+    uint4 gv = make_uint4(0x3f803f80u, 0x3f803f80u, 0x3f803f80u, 0x3f803f80u);   // bf16 ones
+    if (has_gain) gv = *reinterpret_cast<const uint4*>(x_s + kXBytes + c * 16);
+    const float rs = rs_row[row];
+    uint32_t* w = reinterpret_cast<uint32_t*>(&xv);
+    const __nv_bfloat162* gp = reinterpret_cast<const __nv_bfloat162*>(&gv);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w[e]));
+      const float2 gf = __bfloat1622float2(gp[e]);
+      const __nv_bfloat162 h = __floats2bfloat162_rn(f.x * rs * gf.x, f.y * rs * gf.y);
+      if (W_INT8) {
+        const float2 hf = __bfloat1622float2(h);
+        const __half2 q = __floats2half2_rn(hf.x, hf.y);
+        w[e] = *reinterpret_cast<const uint32_t*>(&q);
+      } else {
+        w[e] = *reinterpret_cast<const uint32_t*>(&h);
+      }
+    }
+    *px = xv;
+  }
+}
+
+// this warp's share of the (converted) chunk, from the staging buffer to registers
 template <bool W_INT8>
 __device__ __forceinline__ void read_operand(uint4 (&xr)[kXr], const unsigned char* x_s, int M, int K, int kbase,
-                                             bool has_gain, float rs, int warp, int g, int t) {
+                                             int warp, int g, int t) {
   const int pitch = K <= kChunk ? K * 2 : kXRowBytes;
-  const bool convert = W_INT8 || has_gain;
 #pragma unroll
   for (int i = 0; i < kXr; ++i) {
     const int k = x_index<W_INT8>(i, kbase, warp, t);
-    uint4 xv = make_uint4(0, 0, 0, 0);
-    uint4 gv = make_uint4(0x3f803f80u, 0x3f803f80u, 0x3f803f80u, 0x3f803f80u);   // bf16 ones
-    if (k < K) {
-      if (g < M) xv = *reinterpret_cast<const uint4*>(x_s + g * pitch + (k - kbase) * 2);
-      if (has_gain) gv = *reinterpret_cast<const uint4*>(x_s + kXBytes + (k - kbase) * 2);
-    }
-    if (convert) {
-      uint32_t* w = reinterpret_cast<uint32_t*>(&xv);
-      const __nv_bfloat162* gp = reinterpret_cast<const __nv_bfloat162*>(&gv);
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w[e]));
-        const float2 gf = __bfloat1622float2(gp[e]);
-        const __nv_bfloat162 h = __floats2bfloat162_rn(f.x * rs * gf.x, f.y * rs * gf.y);
-        if (W_INT8) {
-          const float2 hf = __bfloat1622float2(h);
-          const __half2 q = __floats2half2_rn(hf.x, hf.y);
-          w[e] = *reinterpret_cast<const uint32_t*>(&q);
-        } else {
-          w[e] = *reinterpret_cast<const uint32_t*>(&h);
-        }
-      }
-    }
-    xr[i] = xv;
+    xr[i] = make_uint4(0, 0, 0, 0);
+    if (k < K && g < M) xr[i] = *reinterpret_cast<const uint4*>(x_s + g * pitch + (k - kbase) * 2);
   }
 }
 
@@ -575,7 +595,6 @@ struct GemmPhase {
     TL_MARK();
     uint4 xr[kXr];
     bool have_x = false, first = true;
-    float rs = 1.f;   // RMSNorm factor times the fp16 scale of the operand row
     float ss_run = 0.f;   // threads 0..7 (o / down): sum of squares of the row of x this CTA has written
     float best = -INFINITY;   // LM head: this thread's running arg-max over the elements it finishes
     int best_i = 0x7fffffff;
@@ -639,8 +658,10 @@ struct GemmPhase {
                 inv = ldexpf(1.f, e - 15);
               }
             }
-            rs = rnorm * xscale;
-            if (warp == 0 && t == 0) misc[kMiscInvScale + g] = inv;   // read in the epilogues, behind a CTA barrier
+            if (warp == 0 && t == 0) {
+              misc[kMiscRs + g] = rnorm * xscale;   // conversion factor of operand row g
+              misc[kMiscInvScale + g] = inv;
+            }   // read in the epilogues, behind a CTA barrier
           }
           {
             int got = 1;
@@ -650,7 +671,12 @@ struct GemmPhase {
             xphase ^= 1u;
           }
           TL_MARK();
-          read_operand<W_INT8>(xr, x_s, M, jb.K, kc * kChunk, normed, rs, warp, g, t);
+          if (W_INT8 || normed) {
+            cbar();   // the rows' factors are published
+            convert_staged<W_INT8>(x_s, M, jb.K, kc * kChunk, normed, misc + kMiscRs);
+            cbar();
+          }
+          read_operand<W_INT8>(xr, x_s, M, jb.K, kc * kChunk, warp, g, t);
           cbar();   // every warp has its share: the staging buffer may be refilled
           TL_MARK();
         }
@@ -917,36 +943,30 @@ __device__ void prep_phase(const MegaParams& p, float* misc, int cta, int ncta) 
 }
 
 // ---- attention phase: QK-RMSNorm + RoPE + KV append + split-KV partials -------------------------
-template <int D>
-__device__ void rope_vec(const __nv_bfloat16* src, const __nv_bfloat16* gain, const float2* rope_row, float eps,
-                         __nv_bfloat16* dst, int lane) {
-  constexpr int kPairs = D / 64;
-  float lo[kPairs], hi[kPairs];
-  float ss = 0.f;
-#pragma unroll
-  for (int q = 0; q < kPairs; ++q) {
-    const int d = lane + 32 * q;
-    lo[q] = __bfloat162float(__ldcg(src + d));
-    hi[q] = __bfloat162float(__ldcg(src + d + D / 2));
-    ss += lo[q] * lo[q] + hi[q] * hi[q];
-  }
-  if (gain != nullptr) {
-    ss = warp_sum(ss);
-    const float r = 1.0f / sqrtf(ss / (float)D + eps);
-#pragma unroll
-    for (int q = 0; q < kPairs; ++q) {
-      const int d = lane + 32 * q;
-      lo[q] = lo[q] * r * __bfloat162float(gain[d]);
-      hi[q] = hi[q] * r * __bfloat162float(gain[d + D / 2]);
-    }
+// kP consecutive bf16 (kP = 4 or 8) from / to 8- or 16-byte aligned memory, as floats
+template <int kP>
+__device__ __forceinline__ void load_bf16_vec(float (&f)[kP], const __nv_bfloat16* src, bool through_l2) {
+  uint32_t w[kP / 2];
+  if constexpr (kP == 8) {
+    const uint4 v = through_l2 ? __ldcg(reinterpret_cast<const uint4*>(src)) : __ldg(reinterpret_cast<const uint4*>(src));
+    w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
+  } else {
+    const uint2 v = through_l2 ? __ldcg(reinterpret_cast<const uint2*>(src)) : __ldg(reinterpret_cast<const uint2*>(src));
+    w[0] = v.x; w[1] = v.y;
   }
 #pragma unroll
-  for (int q = 0; q < kPairs; ++q) {
-    const int d = lane + 32 * q;
-    const float2 cs = rope_row[d];
-    dst[d] = __float2bfloat16_rn(lo[q] * cs.x - hi[q] * cs.y);
-    dst[d + D / 2] = __float2bfloat16_rn(hi[q] * cs.x + lo[q] * cs.y);
+  for (int i = 0; i < kP / 2; ++i) {
+    f[2 * i] = __uint_as_float(w[i] << 16);
+    f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
   }
+}
+template <int kP>
+__device__ __forceinline__ void store_bf16_vec(__nv_bfloat16* dst, const float (&f)[kP]) {
+  uint32_t w[kP / 2];
+#pragma unroll
+  for (int i = 0; i < kP / 2; ++i) w[i] = pack_bf16(f[2 * i], f[2 * i + 1]);
+  if constexpr (kP == 8) *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
+  else *reinterpret_cast<uint2*>(dst) = make_uint2(w[0], w[1]);
 }
 
 __device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
@@ -987,7 +1007,11 @@ __device__ __forceinline__ void attention_prefetch(const MegaParams& p, int laye
 
 template <int D>
 __device__ __noinline__ void attention_phase(const MegaParams& p, int layer, bool want_amax, __nv_bfloat16* k_s,
-                                             __nv_bfloat16* v_s, __nv_bfloat16* q_s, float* misc, int cta, int ncta) {
+                                             __nv_bfloat16* v_s, __nv_bfloat16* q_s, float* misc, uint64_t* xbar,
+                                             uint32_t& xphase, uint32_t& xphase2, int cta, int ncta) {
+  float* o_s = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(k_s) + 2 * kKvTileBytes + kQTileBytes);
+  float* ml_s = o_s + kMaxRowsAttn * 128;
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + kMiscAbort);
   constexpr int kStride = D + 8;
   constexpr int kDSteps = D / 16;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
@@ -1032,22 +1056,78 @@ __device__ __noinline__ void attention_phase(const MegaParams& p, int layer, boo
 
     // (a) rotate this kv head's query rows into shared memory; the item that owns a block row's
     //     cache slot also rotates its K row and stores K and V there
-    for (int u = warp; u < R + T; u += NW) {
-      if (u < R) {
-        const int node = u / G, hq = hk * G + (u % G);
-        const int m = b * p.T_max + node;
-        rope_vec<D>(p.qkv + (size_t)m * qkv_w + (size_t)hq * D, ly.q_norm,
-                    p.rope_table + (size_t)(P + p.bi.depth[m]) * (D / 2), p.rms_eps, q_s + u * kStride, lane);
-      } else {
-        const int node = u - R;
-        const int slot = P + node;
-        if (slot >= key_begin && slot < key_end) {
-          const int m = b * p.T_max + node;
-          rope_vec<D>(p.qkv + (size_t)m * qkv_w + (size_t)(p.Hq + hk) * D, ly.k_norm,
-                      p.rope_table + (size_t)(P + p.bi.depth[m]) * (D / 2), p.rms_eps, kbase + (size_t)slot * D, lane);
-          const __nv_bfloat16* vsrc = p.qkv + (size_t)m * qkv_w + (size_t)(p.Hq + p.Hkv + hk) * D;
-          if (lane < D / 8)
-            reinterpret_cast<uint4*>(vbase + (size_t)slot * D)[lane] = __ldcg(reinterpret_cast<const uint4*>(vsrc) + lane);
+    // A quarter of a warp per head vector (four vectors per warp at a time, one code path): lane q8 owns
+    // the rotation pairs (d, d + D/2) for d = kP q8 .. kP q8 + kP - 1.
+    {
+      constexpr int kP = D / 16;
+      const int q8 = lane & 7, d0 = q8 * kP;
+#pragma unroll 1
+      for (int ub = warp * 4; ub < R + T; ub += NW * 4) {
+        const int u = ub + (lane >> 3);
+        int kind = 0;   // 0 nothing, 1 query vector, 2 key vector (with its value row)
+        int m = 0, slot = 0;
+        const __nv_bfloat16* src = p.qkv;
+        if (u < R) {
+          kind = 1;
+          m = b * p.T_max + u / G;
+          src = p.qkv + (size_t)m * qkv_w + (size_t)(hk * G + (u % G)) * D;
+        } else if (u < R + T) {
+          slot = P + (u - R);
+          if (slot >= key_begin && slot < key_end) {
+            kind = 2;
+            m = b * p.T_max + (u - R);
+            src = p.qkv + (size_t)m * qkv_w + (size_t)(p.Hq + hk) * D;
+          }
+        }
+        const __nv_bfloat16* gain = kind == 2 ? ly.k_norm : ly.q_norm;
+        float lo[kP], hi[kP], glo[kP], ghi[kP];
+        float4 cs[kP / 2];
+        uint4 vrow[kP / 4];
+#pragma unroll
+        for (int i = 0; i < kP; ++i) { lo[i] = hi[i] = 0.f; glo[i] = ghi[i] = 1.f; }
+        if (kind != 0) {   // every load of the vector before any use
+          load_bf16_vec<kP>(lo, src + d0, true);
+          load_bf16_vec<kP>(hi, src + D / 2 + d0, true);
+          const float4* cp = reinterpret_cast<const float4*>(p.rope_table + (size_t)(P + p.bi.depth[m]) * (D / 2) + d0);
+#pragma unroll
+          for (int i = 0; i < kP / 2; ++i) cs[i] = __ldg(cp + i);
+          if (gain != nullptr) {
+            load_bf16_vec<kP>(glo, gain + d0, false);
+            load_bf16_vec<kP>(ghi, gain + D / 2 + d0, false);
+          }
+          if (kind == 2) {
+            const uint4* vsrc = reinterpret_cast<const uint4*>(p.qkv + (size_t)m * qkv_w + (size_t)(p.Hq + p.Hkv + hk) * D) + q8 * (kP / 4);
+#pragma unroll
+            for (int i = 0; i < kP / 4; ++i) vrow[i] = __ldcg(vsrc + i);
+          }
+        }
+        if (ly.q_norm != nullptr) {   // QK-RMSNorm (a model either has both gains or none)
+          float ss = 0.f;
+#pragma unroll
+          for (int i = 0; i < kP; ++i) ss += lo[i] * lo[i] + hi[i] * hi[i];
+          ss += __shfl_xor_sync(0xffffffffu, ss, 1);
+          ss += __shfl_xor_sync(0xffffffffu, ss, 2);
+          ss += __shfl_xor_sync(0xffffffffu, ss, 4);
+          const float rn = 1.0f / sqrtf(ss / (float)D + p.rms_eps);
+#pragma unroll
+          for (int i = 0; i < kP; ++i) { lo[i] = lo[i] * rn * glo[i]; hi[i] = hi[i] * rn * ghi[i]; }
+        }
+        if (kind != 0) {
+          float olo[kP], ohi[kP];
+#pragma unroll
+          for (int i = 0; i < kP; ++i) {
+            const float c = (i & 1) ? cs[i / 2].z : cs[i / 2].x, sn = (i & 1) ? cs[i / 2].w : cs[i / 2].y;
+            olo[i] = lo[i] * c - hi[i] * sn;
+            ohi[i] = hi[i] * c + lo[i] * sn;
+          }
+          __nv_bfloat16* dst = kind == 1 ? q_s + u * kStride : kbase + (size_t)slot * D;
+          store_bf16_vec<kP>(dst + d0, olo);
+          store_bf16_vec<kP>(dst + D / 2 + d0, ohi);
+          if (kind == 2) {
+            uint4* vdst = reinterpret_cast<uint4*>(vbase + (size_t)slot * D) + q8 * (kP / 4);
+#pragma unroll
+            for (int i = 0; i < kP / 4; ++i) vdst[i] = vrow[i];
+          }
         }
       }
     }
@@ -1135,7 +1215,6 @@ __device__ __noinline__ void attention_phase(const MegaParams& p, int layer, boo
         row_sum[h] += __shfl_xor_sync(0xffffffffu, row_sum[h], 1);
         row_sum[h] += __shfl_xor_sync(0xffffffffu, row_sum[h], 2);
       }
-      const size_t slot = (((size_t)b * p.Hkv + hk) * p.attn_nchunk + c) * p.attn_rpad;
       // O = P V in two halves of the head dimension (keeps the accumulators within the register budget)
 #pragma unroll 1
       for (int half = 0; half < 2; ++half) {
@@ -1165,7 +1244,7 @@ __device__ __noinline__ void attention_phase(const MegaParams& p, int layer, boo
         for (int h = 0; h < 2; ++h) {
           const int r = warp * 16 + g + 8 * h;
           if (r >= p.attn_rpad) continue;
-          float* op = p.o_part + (slot + r) * D + half * (D / 2);
+          float* op = o_s + r * D + half * (D / 2);
 #pragma unroll
           for (int i = 0; i < D / 16; ++i)
             *reinterpret_cast<float2*>(op + 8 * i + 2 * t) = make_float2(o[i][2 * h], o[i][2 * h + 1]);
@@ -1176,91 +1255,106 @@ __device__ __noinline__ void attention_phase(const MegaParams& p, int layer, boo
         for (int h = 0; h < 2; ++h) {
           const int r = warp * 16 + g + 8 * h;
           if (r >= p.attn_rpad) continue;
-          p.ml_part[(slot + r) * 2] = row_max[h];
-          p.ml_part[(slot + r) * 2 + 1] = row_sum[h];
+          ml_s[r * 2] = row_max[h];
+          ml_s[r * 2 + 1] = row_sum[h];
         }
       }
     }
 
-    // (d) The CTA that finishes the last chunk of this (sequence, kv head) merges all of its chunks, in
-    //     chunk order, so the result does not depend on which CTA that is.
+    // (d) The partial (un-normalised output, row maxima and sums) leaves as two bulk stores.  Then the
+    //     CTAs of this (sequence, kv head) wait for one another (a bounded wait on the head's arrival
+    //     count: all of them are resident) and share the merge: the CTA of chunk c takes the query rows
+    //     c, c + nch, ...  A row's chunks are added in a fixed order whoever does it.
     const int nch = (Lk + kKeyTile - 1) / kKeyTile;
+    const size_t slot0 = ((size_t)b * p.Hkv + hk) * p.attn_nchunk * p.attn_rpad;
+    unsigned* arrivals = p.attn_count + (size_t)layer * p.B * p.Hkv + b * p.Hkv + hk;
     ATTN_T(2);
-    __threadfence();   // this CTA's partials are visible before its arrival is
-    cbar();
+    cbar();   // o_s and ml_s are complete
     if (threadIdx.x == 0) {
-      const unsigned old = atomicAdd(p.attn_count + (size_t)layer * p.B * p.Hkv + b * p.Hkv + hk, 1u);
-      *last_flag = (old == (unsigned)(nch - 1));
+      const size_t slot = slot0 + (size_t)c * p.attn_rpad;
+      asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+      bulk_store(p.o_part + slot * D, o_s, (uint32_t)p.attn_rpad * D * 4);
+      bulk_store(p.ml_part + slot * 2, ml_s, (uint32_t)p.attn_rpad * 8);
+      asm volatile("cp.async.bulk.commit_group;\ncp.async.bulk.wait_group 0;\n" ::: "memory");
+      __threadfence();   // this CTA's partial is visible before its arrival is
+      atomicAdd(arrivals, 1u);
+      int ok_flag = 1;
+      if (c < R) {   // this CTA has rows to merge: wait for the other chunks
+        const unsigned long long t0 = now_ns();
+        unsigned polls = 0;
+        while (true) {
+          unsigned v;
+          asm volatile("ld.acquire.gpu.global.u32 %0, [%1];\n" : "=r"(v) : "l"(arrivals) : "memory");
+          if (v >= (unsigned)nch) break;
+          if ((++polls & 63u) == 0 && (*abort_flag || now_ns() - t0 > kWaitBudgetNs)) {
+            atomicMin(p.status, QUASAR_ERR_TIMEOUT);
+            *abort_flag = 1;
+            ok_flag = 0;
+            break;
+          }
+        }
+      }
+      *last_flag = ok_flag;
     }
     cbar();
     ATTN_T(3);
     if (*last_flag) {
-      __threadfence();
-      ATTN_T(5);
-      const size_t slot0 = ((size_t)b * p.Hkv + hk) * p.attn_nchunk * p.attn_rpad;
-      // half a warp per query row: lane l16 owns D/16 consecutive output dimensions
-      constexpr int kV4 = D / 64;              // float4 loads per lane and chunk
-      constexpr int kBlk = 8;                  // chunks fetched together
-      const int hsel = lane >> 4, l16 = lane & 15;
+      // warp w adds the chunks w, w + NW, ... of a row (lane l: four output dimensions), then the
+      // warps' sums meet in shared memory in warp order
+      float* part = o_s;                                   // [NW][D + 4] floats; the partial has left
+      constexpr int kPS = 128 + 4;
 #pragma unroll 1
-      for (int r0 = warp * 2; r0 < R; r0 += NW * 2) {
-        const int r = r0 + hsel;
-        const bool rv = r < R;
-        const int rr = rv ? r : R - 1;
+      for (int r = c; r < R; r += nch) {
         float mx = -INFINITY;
-        for (int cc = l16; cc < nch; cc += 16)
-          mx = fmaxf(mx, __ldcg(p.ml_part + (slot0 + (size_t)cc * p.attn_rpad + rr) * 2));
+        for (int cc = lane; cc < nch; cc += 32) mx = fmaxf(mx, __ldcg(p.ml_part + (slot0 + (size_t)cc * p.attn_rpad + r) * 2));
 #pragma unroll
-        for (int o = 8; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-        float acc[4 * kV4];
-#pragma unroll
-        for (int e = 0; e < 4 * kV4; ++e) acc[e] = 0.f;
+        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
         float den = 0.f;
 #pragma unroll 1
-        for (int c0 = 0; c0 < nch; c0 += kBlk) {
-          float4 ov[kBlk][kV4];
-#pragma unroll
-          for (int j = 0; j < kBlk; ++j) {
-            const size_t sidx = slot0 + (size_t)min(c0 + j, nch - 1) * p.attn_rpad + rr;
-#pragma unroll
-            for (int q = 0; q < kV4; ++q) ov[j][q] = __ldcg(reinterpret_cast<const float4*>(p.o_part + sidx * D) + l16 * kV4 + q);
-          }
-          float2 ml = make_float2(-INFINITY, 0.f);
-          if (l16 < kBlk && c0 + l16 < nch)
-            ml = __ldcg(reinterpret_cast<const float2*>(p.ml_part + (slot0 + (size_t)(c0 + l16) * p.attn_rpad + rr) * 2));
-          const float w_lane = ml.x == -INFINITY ? 0.f : exp2f(ml.x - mx);
-#pragma unroll
-          for (int j = 0; j < kBlk; ++j) {   // chunk order; lane j of this half holds chunk c0 + j's weight
-            const float w = __shfl_sync(0xffffffffu, w_lane, (lane & 16) | j);
-            den += w * __shfl_sync(0xffffffffu, ml.y, (lane & 16) | j);
-#pragma unroll
-            for (int q = 0; q < kV4; ++q) {
-              acc[4 * q + 0] += w * ov[j][q].x; acc[4 * q + 1] += w * ov[j][q].y;
-              acc[4 * q + 2] += w * ov[j][q].z; acc[4 * q + 3] += w * ov[j][q].w;
-            }
+        for (int cc = warp; cc < nch; cc += NW) {
+          const size_t sidx = slot0 + (size_t)cc * p.attn_rpad + r;
+          const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.ml_part + sidx * 2));
+          const float w = ml.x == -INFINITY ? 0.f : exp2f(ml.x - mx);
+          den += w * ml.y;
+          if constexpr (D == 128) {
+            const float4 ov = __ldcg(reinterpret_cast<const float4*>(p.o_part + sidx * D) + lane);
+            acc[0] += w * ov.x; acc[1] += w * ov.y; acc[2] += w * ov.z; acc[3] += w * ov.w;
+          } else {
+            const float2 ov = __ldcg(reinterpret_cast<const float2*>(p.o_part + sidx * D) + lane);
+            acc[0] += w * ov.x; acc[1] += w * ov.y;
           }
         }
-        const float inv = 1.0f / den;
-        const int i = rr / G, hq = hk * G + (rr % G);
-        const int m = b * p.T_max + i;
-        float amax = 0.f;
-        uint32_t packed[2 * kV4];
+        cbar();   // the previous row's sums have been read
+        *reinterpret_cast<float4*>(part + warp * kPS + lane * 4) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+        if (lane == 0) part[warp * kPS + 128] = den;
+        cbar();
+        if (warp == 0) {
+          float tot[4] = {0.f, 0.f, 0.f, 0.f};
+          float dsum = 0.f;
 #pragma unroll
-        for (int e = 0; e < 2 * kV4; ++e) {
-          const __nv_bfloat162 pr = __floats2bfloat162_rn(acc[2 * e] * inv, acc[2 * e + 1] * inv);
-          packed[e] = *reinterpret_cast<const uint32_t*>(&pr);
-          const float2 back = __bfloat1622float2(pr);
-          amax = fmaxf(amax, fmaxf(fabsf(back.x), fabsf(back.y)));
-        }
-        if (rv) {
-          __nv_bfloat16* dst = p.attn + (size_t)m * p.Hq * D + (size_t)hq * D + l16 * (D / 16);
-          if constexpr (kV4 == 2) *reinterpret_cast<uint4*>(dst) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
-          else *reinterpret_cast<uint2*>(dst) = make_uint2(packed[0], packed[1]);
-        }
-        if (want_amax) {   // row maximum of the o projection's operand
+          for (int w = 0; w < NW; ++w) {
+            const float4 v = *reinterpret_cast<const float4*>(part + w * kPS + lane * 4);
+            tot[0] += v.x; tot[1] += v.y; tot[2] += v.z; tot[3] += v.w;
+            dsum += part[w * kPS + 128];
+          }
+          const float inv = 1.0f / dsum;
+          const int i = r / G, hq = hk * G + (r % G);
+          const int m = b * p.T_max + i;
+          __nv_bfloat16* dst = p.attn + (size_t)m * p.Hq * D + (size_t)hq * D + lane * (D / 32);
+          float amax = 0.f;
 #pragma unroll
-          for (int o = 8; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
-          if (l16 == 0 && rv && amax > 0.f) atomicMax(p.amax_buf + (4 * layer + 1) * 8 + m, __float_as_uint(amax));
+          for (int e = 0; e < D / 64; ++e) {
+            const __nv_bfloat162 pr = __floats2bfloat162_rn(tot[2 * e] * inv, tot[2 * e + 1] * inv);
+            reinterpret_cast<__nv_bfloat162*>(dst)[e] = pr;
+            const float2 back = __bfloat1622float2(pr);
+            amax = fmaxf(amax, fmaxf(fabsf(back.x), fabsf(back.y)));
+          }
+          if (want_amax) {   // row maximum of the o projection's operand
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+            if (lane == 0 && amax > 0.f) atomicMax(p.amax_buf + (4 * layer + 1) * 8 + m, __float_as_uint(amax));
+          }
         }
       }
     }
@@ -1335,7 +1429,7 @@ __global__ void __launch_bounds__(kThreads, 1) verify_megakernel(const MegaParam
   volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + kMiscAbort);
   uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<unsigned char*>(misc) + kMiscBarBytes);
   Pipe pipe{smem, bars, bars + kStages, abort_flag, p.status};
-  uint64_t* xbar = bars + 2 * kStages;   // the operand's bulk copies have landed
+  uint64_t* xbar = bars + 2 * kStages;   // the operand's bulk copies have landed (xbar[1]: second buffer of the attention merge)
 
   if (threadIdx.x == 0) {
     *abort_flag = 0;
@@ -1344,6 +1438,7 @@ __global__ void __launch_bounds__(kThreads, 1) verify_megakernel(const MegaParam
       mbar_init(pipe.empty + s, NW);   // one arrival per consumer warp
     }
     mbar_init(xbar, 1);
+    mbar_init(xbar + 1, 1);
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
   }
   if (threadIdx.x < 8) {  // running arg-max of this CTA
@@ -1358,7 +1453,7 @@ __global__ void __launch_bounds__(kThreads, 1) verify_megakernel(const MegaParam
   }
 
   int slot = 0;
-  uint32_t phase = 0, xphase = 0;
+  uint32_t phase = 0, xphase = 0, xphase2 = 0;
   GridSync gs{p.barrier, p.status, (unsigned)ncta, 0u, abort_flag};
   bool ok = true;
 #ifdef QUASAR_PHASE_TIMER
@@ -1379,7 +1474,7 @@ __global__ void __launch_bounds__(kThreads, 1) verify_megakernel(const MegaParam
     if (!(ok = gs.sync())) break;
     PHASE_MARK();
     if ((job & 3) == 0) {
-      attention_phase<D>(p, job >> 2, W_INT8, k_s, v_s, q_s, misc, cta, ncta);
+      attention_phase<D>(p, job >> 2, W_INT8, k_s, v_s, q_s, misc, xbar, xphase, xphase2, cta, ncta);
       PHASE_MARK();
       if (!(ok = gs.sync())) break;
       PHASE_MARK();
