@@ -747,10 +747,15 @@ struct GemmPhase {
       TL_MARK();
       // ---- cross-warp reduction in a fixed order, then the fused epilogue ----
       cbar();
-#pragma unroll
-      for (int it = 0; it < kItems; ++it) {
+#pragma unroll 1
+      for (int it = 0; it < kItems; ++it) {   // rolled: the epilogue's code exists once
         const EpiItem ei = epi_item(jb, v, tg, gt, M, it);
-        epilogue(p, jb, v, job, ei, d0[it], d1[it], resid[it], best, best_i, red, misc);
+        float e0 = d0[0], e1 = d1[0], er = resid[0];
+#pragma unroll
+        for (int j = 1; j < kItems; ++j) {
+          if (it == j) { e0 = d0[j]; e1 = d1[j]; er = resid[j]; }
+        }
+        epilogue(p, jb, v, job, ei, e0, e1, er, best, best_i, red, misc);
       }
       cbar();
       TL_MARK();
@@ -1154,13 +1159,13 @@ __device__ __noinline__ void attention_phase(const MegaParams& p, int layer, boo
     // (c) one warp per 16 query rows
     const int row_tiles = (R + 15) / 16;
     if (warp < row_tiles) {
-      uint64_t anc[2];
+      uint32_t anc[2];   // the block has at most 8 rows here: the ancestor mask fits 32 bits
       uint32_t qf[kDSteps][4];
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
         const int r = warp * 16 + g + 8 * h;
         const bool ok = r < R;
-        anc[h] = ok ? p.bi.anc[b * p.T_max + r / G] : 0ull;
+        anc[h] = ok ? (uint32_t)p.bi.anc[b * p.T_max + r / G] : 0u;
         const __nv_bfloat16* qrow = q_s + (ok ? r : 0) * kStride;
 #pragma unroll
         for (int kd = 0; kd < kDSteps; ++kd) {
@@ -1188,7 +1193,7 @@ __device__ __noinline__ void attention_phase(const MegaParams& p, int layer, boo
           const int h = e >> 1;
           const int key = key_begin + 8 * j + 2 * t + (e & 1);
           bool ok = key < key_end;
-          if (ok && key >= P) ok = (anc[h] >> (key - P)) & 1ull;
+          if (ok && key >= P) ok = (anc[h] >> (key - P)) & 1u;
           const float v = ok ? s[j][e] * scale_log2 : -INFINITY;
           s[j][e] = v;
           row_max[h] = fmaxf(row_max[h], v);
