@@ -33,6 +33,11 @@ from paper_2603_01399_b200 import synth  # noqa: E402
 
 WORKLOAD = "qwen3-8b-shaped verify pass: B=1, prefix 1024, chain draft gamma=5 (6 block rows), int8 weights"
 PREFIX, GAMMA, BATCH = 1024, 5, 1
+METRIC = "verify-pass latency & accepted tok/s, Qwen3-8B shape; HBM GB/s as % of peak"
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the persistent kernel, from the ncu capture
+# summarised in profiles/ (a 2-layer model, scaled by the weight bytes of the full one); None while the
+# kernel has changed since that capture
+MEGAKERNEL_DRAM_BYTES_PER_LAUNCH = None
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 
@@ -57,6 +62,24 @@ def algorithmic_bytes(shape, batch, t_rows, prefix_total, weight_bytes_per_elem)
     gains = (2 * shape.n_layers + 1) * shape.hidden * 2
     return {"weights": w, "scales": scales, "kv_read": kv_read, "kv_write": kv_write, "embed": embed,
             "gains": gains, "total": w + scales + kv_read + kv_write + embed + gains}
+
+
+def max_over_ranks(value: float, dist, device) -> float:
+    """The slowest rank's time: replicas are independent, so the job is as slow as its slowest GPU."""
+    if dist is None:
+        return float(value)
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t[0])
+
+
+def sum_over_ranks(value: float, dist, device) -> float:
+    """Units processed by the whole job (every replica works on its own sequences)."""
+    if dist is None:
+        return float(value)
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    return float(t[0])
 
 
 class ClockSampler:
@@ -180,11 +203,7 @@ def run_ours(args):
         clocks = sampler.stop() if sampler else None
         if dist is not None:
             dist.barrier()
-        ms = e0.elapsed_time(e1)
-        if dist is not None:
-            t = torch.tensor([ms], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t[0])
+        ms = max_over_ranks(e0.elapsed_time(e1), dist, "cuda")
         return ms / steps, buf, plan, launches, clocks
 
     ms_step, buf, plan, launches, clocks = timed_plan(m_int8, args.steps, args.warmup, True)
@@ -202,13 +221,11 @@ def run_ours(args):
     t0 = time.perf_counter()
     for _ in range(args.steps):
         plan.run_host(tokens_host, al, bo)
-    e2e_ms = (time.perf_counter() - t0) * 1e3 / args.steps
-    if dist is not None:
-        t = torch.tensor([e2e_ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t[0])
+    e2e_ms = max_over_ranks((time.perf_counter() - t0) * 1e3 / args.steps, dist, "cuda")
+    accepted_job = sum_over_ranks(accepted, dist, "cuda")          # every replica verifies its own sequences
+    accepted_drafts_job = sum_over_ranks(accepted_drafts, dist, "cuda")
 
-    # the dominant kernel alone: the skinny GEMM over the model's 145 weight matrices in pass order
+    # the per-step skinny GEMM (used for blocks of more than 8 rows) over the model's 145 matrices in pass order
     gemm = time_gemm_sweep(binding, m_int8, shape, BATCH * t_rows, max(3, args.steps // 4))
 
     # bf16-weight sibling pass (the "BF16 verifier" of Section 3.4, same kernels)
@@ -219,28 +236,32 @@ def run_ours(args):
     ab = algorithmic_bytes(shape, BATCH, t_rows, PREFIX * BATCH, 1)
     ab16 = algorithmic_bytes(shape, BATCH, t_rows, PREFIX * BATCH, 2)
     pass_gbs = ab["total"] / (ms_step * 1e-3) / 1e9
+    # roofline of the dominant kernel: the persistent verify kernel, one launch per step, so its average
+    # launch duration is the step time measured above with CUDA events on the launching stream
+    launch_gbs = ab["total"] / (ms_step * 1e-3) / 1e9
     out = {
-        "metric": "accepted tokens/s of the verify pass (Qwen3-8B shape)", "value": world * accepted / (ms_step * 1e-3),
-        "unit": "tok/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step,
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8 weights x bf16, f32 accumulate",
+        "metric": METRIC, "value": accepted_job / (ms_step * 1e-3),
+        "unit": "accepted tok/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8 weights, f16 mma operands, f32 accumulate",
         "data": "synthetic",
         "config": {"workload": WORKLOAD, "replicas": world, "batch": BATCH, "prefix": PREFIX, "gamma": GAMMA,
                    "l2": "inputs (7.7 GB of weights + KV per pass) exceed the 126 MB L2; no flush needed",
-                   "launch": "one CUDA-graph replay per step"},
+                   "launch": "one persistent cooperative kernel per step"},
         "verify_latency_ms": ms_step, "accepted_per_pass": accepted, "accepted_drafts_per_pass": accepted_drafts,
-        "accepted_drafts_tok_s": world * accepted_drafts / (ms_step * 1e-3), "device_status": status,
+        "accepted_drafts_tok_s": accepted_drafts_job / (ms_step * 1e-3), "device_status": status,
         "pass_bytes": ab, "pass_hbm_gbs": pass_gbs, "pass_hbm_frac_of_measured_copy": pass_gbs / hbm_peak,
         "pass_hbm_frac_of_nominal_8TBs": pass_gbs / NOMINAL_HBM_GBS,
         "bf16_sibling": {"verify_latency_ms": bf16_ms, "ratio_vs_int8": bf16_ms / ms_step,
                          "pass_hbm_gbs": ab16["total"] / (bf16_ms * 1e-3) / 1e9},
+        "per_step_gemm_sweep": {"kernel": "skinny_gemm_kernel, 145 launches", "gbs": gemm["gbs"], "avg_launch_us": gemm["avg_us"]},
         "clocks": clocks,
-        "e2e": {"value": world * accepted / (e2e_ms * 1e-3), "unit": "tok/s", "ms_per_step": e2e_ms,
+        "e2e": {"value": accepted_job / (e2e_ms * 1e-3), "unit": "accepted tok/s", "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": tokens_host.numel() * 4, "d2h_bytes_per_step": 2 * BATCH * 4},
         "gpu_launches": int(launches),
-        "roofline": {"bound": "hbm", "kernel": "skinny_gemm_kernel (145 launches per pass, timed alone over the model's weights)",
-                     "achieved": gemm["gbs"], "peak": hbm_peak, "unit": "GB/s", "frac": gemm["gbs"] / hbm_peak,
-                     "peak_kind": f"{peak_kind} copy bandwidth", "traffic": None,
-                     "avg_launch_us": gemm["avg_us"], "bytes_per_launch": gemm["bytes_per_launch"]},
+        "roofline": {"bound": "hbm", "kernel": "verify_megakernel<int8, 128> (persistent, one launch per step)",
+                     "achieved": launch_gbs, "peak": hbm_peak, "unit": "GB/s", "frac": launch_gbs / hbm_peak,
+                     "peak_kind": f"{peak_kind} copy bandwidth", "traffic": MEGAKERNEL_DRAM_BYTES_PER_LAUNCH,
+                     "avg_launch_us": ms_step * 1e3, "bytes_per_launch": ab["total"]},
     }
     if rank == 0:
         out["cpu_baseline"] = cpu_baseline(shape, accepted)
@@ -293,37 +314,42 @@ def time_gemm_sweep(binding, model, shape, m_rows, reps):
 
 
 # ------------------------------------------------------------------------------------------
-def oracle_sample(shape, n_layers_sample=1):
-    """Times the CPU oracle on a bounded sample of the workload: `n_layers_sample` decoder layers
-    (with the 1024-position KV prefix) and the LM head, at the full Qwen3-8B widths.  Returns
-    (seconds per layer, seconds for embedding + final norm + LM head + acceptance, threads)."""
-    import oracle
-    small = synth.ModelShape("sample", n_layers_sample, shape.hidden, shape.n_q_heads, shape.n_kv_heads,
-                             shape.head_dim, shape.ffn, shape.vocab, shape.qk_norm, shape.rope_theta, shape.rms_eps)
-    get = master_getter(small, 0, "cpu")
-    om = oracle.build_model(small, lambda kind, layer: synth.bf16_bits(get(kind, layer)), int8=True)
-    kk, vv = synth.kv_prefix(small, BATCH, PREFIX + 16, seed=1)
-    okv = oracle.KVCache(synth.bf16_bits(kk), synth.bf16_bits(vv), np.full(BATCH, PREFIX, np.int32))
-    toks = synth.uniform_tokens((BATCH, GAMMA + 1), shape.vocab, synth.sub_seed(2, "tokens")).numpy()
-    bl = np.full(BATCH, GAMMA + 1, np.int32)
-    t0 = time.perf_counter()
-    oracle.verify(om, okv, toks, None, bl, n_layers_run=0)
-    t_head = time.perf_counter() - t0
-    t0 = time.perf_counter()
-    oracle.verify(om, okv, toks, None, bl, want_logits=False)
-    t_layers = time.perf_counter() - t0
-    try:
-        from threadpoolctl import threadpool_info
-        threads = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
-    except Exception:
-        threads = os.cpu_count() or 1
-    return t_layers / n_layers_sample, t_head, threads
+class OracleSample:
+    """The CPU oracle on a bounded sample of the workload: ONE decoder layer (with the 1024-position KV
+    prefix) and the LM head, at the full Qwen3-8B widths.  Built once; `time_once` runs the sample and
+    returns the pass time extrapolated to all layers."""
+
+    def __init__(self, shape):
+        import oracle
+        self.oracle, self.shape = oracle, shape
+        small = synth.ModelShape("sample", 1, shape.hidden, shape.n_q_heads, shape.n_kv_heads, shape.head_dim,
+                                 shape.ffn, shape.vocab, shape.qk_norm, shape.rope_theta, shape.rms_eps)
+        get = master_getter(small, 0, "cpu")
+        self.om = oracle.build_model(small, lambda kind, layer: synth.bf16_bits(get(kind, layer)), int8=True)
+        kk, vv = synth.kv_prefix(small, BATCH, PREFIX + 16, seed=1)
+        self.okv = oracle.KVCache(synth.bf16_bits(kk), synth.bf16_bits(vv), np.full(BATCH, PREFIX, np.int32))
+        self.toks = synth.uniform_tokens((BATCH, GAMMA + 1), shape.vocab, synth.sub_seed(2, "tokens")).numpy()
+        self.bl = np.full(BATCH, GAMMA + 1, np.int32)
+        try:
+            from threadpoolctl import threadpool_info
+            self.threads = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+        except Exception:
+            self.threads = os.cpu_count() or 1
+
+    def time_once(self):
+        t0 = time.perf_counter()
+        self.oracle.verify(self.om, self.okv, self.toks, None, self.bl, n_layers_run=0)
+        head = time.perf_counter() - t0
+        t0 = time.perf_counter()
+        self.oracle.verify(self.om, self.okv, self.toks, None, self.bl, want_logits=False)
+        per_layer = time.perf_counter() - t0
+        return per_layer, head, per_layer * self.shape.n_layers + head
 
 
 def cpu_baseline(shape, accepted):
-    per_layer, head, threads = oracle_sample(shape)
-    full = per_layer * shape.n_layers + head
-    return {"value": accepted / full, "unit": "tok/s", "cores": threads, "kind": "oracle",
+    sample = OracleSample(shape)
+    per_layer, head, full = sample.time_once()
+    return {"value": accepted / full, "unit": "accepted tok/s", "cores": sample.threads, "kind": "oracle",
             "sample": f"1 of {shape.n_layers} decoder layers ({per_layer:.2f} s) + LM head and acceptance ({head:.2f} s) "
                       f"at full Qwen3-8B widths, B=1, prefix 1024, 6 block rows; scaled to {shape.n_layers} layers "
                       f"= {full:.1f} s per pass",
@@ -331,28 +357,30 @@ def cpu_baseline(shape, accepted):
 
 
 def run_reference(args):
+    """The reference arm: the CPU oracle as it stands, on the host cores (rank 0 only).  A step is the
+    bounded sample above (one decoder layer + the LM head at full widths), scaled to the 36 layers."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     shape = synth.SHAPES["qwen3_8b"]
+    sample = OracleSample(shape)
     times = []
-    threads = 1
     for i in range(args.warmup + args.steps):
-        per_layer, head, threads = oracle_sample(shape)
+        _, _, full = sample.time_once()
         if i >= args.warmup:
-            times.append(per_layer * shape.n_layers + head)
+            times.append(full)
     full = sum(times) / len(times)
     accepted = 1.0   # the oracle's pass emits at least the bonus token; drafts are not generated on this arm
     val = accepted / full
     print(json.dumps({
-        "impl": "reference", "metric": "accepted tokens/s of the verify pass (Qwen3-8B shape)", "value": val,
-        "unit": "tok/s", "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": args.warmup,
+        "impl": "reference", "metric": METRIC, "value": val,
+        "unit": "accepted tok/s", "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": full * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
         "data": "synthetic", "config": {"workload": WORKLOAD},
-        "cpu_baseline": {"value": val, "unit": "tok/s", "kind": "oracle", "cores": threads,
+        "cpu_baseline": {"value": val, "unit": "accepted tok/s", "kind": "oracle", "cores": sample.threads,
                          "sample": "each step: 1 of 36 decoder layers + LM head at full widths, scaled to 36 layers; "
                                    "counts the bonus token only (1 token per pass)"},
-        "e2e": {"value": val, "unit": "tok/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+        "e2e": {"value": val, "unit": "accepted tok/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
 
 
 def run_profile_pass(args):

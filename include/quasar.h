@@ -78,9 +78,10 @@ int quasar_quantize(const void* w_bf16, int64_t N, int64_t K, int8_t* q_out, flo
  * (y_is_f32).  residual: [M][N] bf16 or NULL; with a residual the product is
  * first rounded to bf16, then added, then rounded again (the order the decoder
  * layer uses).  y may alias residual.  M >= 1 (rows are processed in groups of
- * at most 72), K % 16 == 0, N >= 1.
+ * at most 72), K % 16 == 0, 1 <= N <= 1048576 (QUASAR_ERR_SHAPE beyond).
  * workspace: at least quasar_linear_workspace_bytes(M, N, K) bytes; its first
- * use must find it zero-filled and every call leaves it reusable by the next.
+ * use must find its first 64 KiB zero-filled, and every call leaves it reusable by the next call of
+ * any shape (the split-K arrival counters live in those 64 KiB and reset themselves).
  * ---------------------------------------------------------------------- */
 int quasar_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, size_t* bytes_out /* host */);
 int quasar_linear(const void* x, const void* w, const float* delta, int32_t weight_dtype, int64_t M, int64_t N,

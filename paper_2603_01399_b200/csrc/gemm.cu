@@ -27,6 +27,11 @@ constexpr int kThreads = kWarps * 32;
 constexpr int kBlockN = kWarps * 16;  // output channels per CTA
 constexpr int kSub = 512;             // contraction elements staged in shared memory at a time
 constexpr int kMaxSplit = 32;
+// The arrival counters of the split-K reduction take a region of fixed size at the start of the
+// workspace, so that calls of different widths can share one workspace: no call's partial sums
+// land where another call keeps its counters.
+constexpr size_t kCounterBytes = 64 * 1024;
+constexpr int64_t kMaxChannels = (int64_t)(kCounterBytes / sizeof(int)) * kBlockN;
 
 struct GemmArgs {
   const __nv_bfloat16* x;   // [M][K]
@@ -287,7 +292,7 @@ size_t linear_workspace_bytes(int64_t M, int64_t N, int64_t K) {
   const SplitPlan p = plan_split(N, K);
   const int64_t rows = M < kMaxRowsPerGemm ? M : kMaxRowsPerGemm;
   const size_t mpad = (size_t)((rows + 7) / 8) * 8;
-  const size_t counters = ((size_t)p.nblocks * sizeof(int) + 255) / 256 * 256;
+  const size_t counters = kCounterBytes;
   const size_t partial = p.nsplit > 1 ? (size_t)p.nsplit * mpad * (size_t)N * sizeof(float) : 0;
   return counters + partial;
 }
@@ -295,9 +300,9 @@ size_t linear_workspace_bytes(int64_t M, int64_t N, int64_t K) {
 int launch_linear(const __nv_bfloat16* x, const void* w, const float* delta, int weight_dtype, int64_t M, int64_t N,
                   int64_t K, void* y, bool y_is_f32, const __nv_bfloat16* residual, void* workspace,
                   size_t workspace_bytes, cudaStream_t stream) {
-  if (M <= 0 || N <= 0 || K <= 0 || (K % 16) != 0 || N > 0x7fffffff || K > 0x7fffffff) {
-    set_error("linear: unsupported sizes M=%lld N=%lld K=%lld (K must be a multiple of 16)", (long long)M,
-              (long long)N, (long long)K);
+  if (M <= 0 || N <= 0 || K <= 0 || (K % 16) != 0 || N > kMaxChannels || K > 0x7fffffff) {
+    set_error("linear: unsupported sizes M=%lld N=%lld K=%lld (K must be a multiple of 16, N at most %lld)",
+              (long long)M, (long long)N, (long long)K, (long long)kMaxChannels);
     return QUASAR_ERR_SHAPE;
   }
   if (workspace_bytes < linear_workspace_bytes(M, N, K)) {
@@ -305,7 +310,7 @@ int launch_linear(const __nv_bfloat16* x, const void* w, const float* delta, int
     return QUASAR_ERR_CAPACITY;
   }
   const SplitPlan p = plan_split(N, K);
-  const size_t counters = ((size_t)p.nblocks * sizeof(int) + 255) / 256 * 256;
+  const size_t counters = kCounterBytes;
   const size_t ybytes = y_is_f32 ? 4 : 2;
   for (int64_t m0 = 0; m0 < M; m0 += kMaxRowsPerGemm) {
     GemmArgs a;
@@ -360,9 +365,9 @@ int launch_linear_static(const __nv_bfloat16* x, const void* w, const float* del
     }
     scratch = scratch_of_device[dev];
   }
-  if (M <= 0 || N <= 0 || K <= 0 || (K % 16) != 0 || N > 0x7fffffff || K > 0x7fffffff) {
-    set_error("linear_static: unsupported sizes M=%lld N=%lld K=%lld (K must be a multiple of 16)", (long long)M,
-              (long long)N, (long long)K);
+  if (M <= 0 || N <= 0 || K <= 0 || (K % 16) != 0 || N > kMaxChannels || K > 0x7fffffff) {
+    set_error("linear_static: unsupported sizes M=%lld N=%lld K=%lld (K must be a multiple of 16, N at most %lld)",
+              (long long)M, (long long)N, (long long)K, (long long)kMaxChannels);
     return QUASAR_ERR_SHAPE;
   }
   const size_t need = linear_workspace_bytes(M, N, K);
@@ -373,9 +378,7 @@ int launch_linear_static(const __nv_bfloat16* x, const void* w, const float* del
     return QUASAR_ERR_CAPACITY;
   }
   // The arrival counters must start at zero; the array keeps whatever the last call left in it.
-  const SplitPlan p = plan_split(N, K);
-  const size_t counters = ((size_t)p.nblocks * sizeof(int) + 255) / 256 * 256;
-  QUASAR_CUDA_CHECK(cudaMemsetAsync(scratch, 0, counters, stream));
+  QUASAR_CUDA_CHECK(cudaMemsetAsync(scratch, 0, kCounterBytes, stream));
   return launch_linear(x, w, delta, weight_dtype, M, N, K, y, y_is_f32, residual, scratch, kStaticScratchBytes, stream);
 }
 

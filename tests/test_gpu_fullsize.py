@@ -1,0 +1,282 @@
+"""Parity at the benchmark's full widths, in the launch configuration bench.py times (needs a GPU).
+
+The CPU oracle cannot run 36 full-width layers inside a test, so the full sizes are covered three ways.
+
+  * Step by step at full WIDTH ("teacher forced"): the kernel-per-step path records every tensor of a
+    layer; each recorded tensor is recomputed by the oracle's operation from the tensor the GPU recorded
+    just before it, so one step's rounding cannot leak into the next comparison.  Every step must agree
+    within about one bf16 rounding; the 151,936-row LM head within 5e-4.
+  * End to end at full width and one or two layers' depth, both GPU paths against the oracle.  Here the
+    activations are rounded to bf16 after every step: a sum that differs in its last fp32 bits (fp32
+    against the oracle's fp64, or another summation order) now and then rounds the other way, and each
+    such flip of one element of the 4096-wide residual stream moves all 24,576 gate/up sums a little, a
+    good part of which flip in turn.  Measured at two layers, both independent GPU implementations sit
+    at the same distance from the oracle (mean |dlogit| 6e-3 at a logit spread of 1.3, 1 % of the
+    elements beyond max(2e-2, 1e-2 |o|), worst 4e-2).  The benchmark's tolerance is therefore asserted
+    on the share of elements it must hold for, with bounds on the mean and the worst element; top-1 and
+    acceptance are compared exactly on the rows whose top-2 margin is clear of that noise.
+  * At full DEPTH, properties that hold at any size: the two GPU implementations agree with each other
+    to the same statistical standard, the pass is idempotent bit for bit, acceptance stays in bounds.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from oracle import quasar_oracle as qo
+from paper_2603_01399_b200 import binding, synth
+from tests.common import logits_close, margins, master_getter
+
+pytestmark = pytest.mark.gpu
+
+
+def _cut(shape, n_layers, name):
+    return synth.ModelShape(name, n_layers, shape.hidden, shape.n_q_heads, shape.n_kv_heads, shape.head_dim,
+                            shape.ffn, shape.vocab, shape.qk_norm, shape.rope_theta, shape.rms_eps)
+
+
+def _models(shape, s_max):
+    get = master_getter(shape, 0, "cpu")
+    om = oracle.build_model(shape, lambda kind, layer: synth.bf16_bits(get(kind, layer)), int8=True)
+    gm = binding.Model.from_master(shape, get, s_max, int8=True)
+    return om, gm
+
+
+def _caches(shape, batch, s_max, prefix_lens):
+    kk, vv = synth.kv_prefix(shape, batch, s_max, seed=1)
+    okv = oracle.KVCache(synth.bf16_bits(kk).copy(), synth.bf16_bits(vv).copy(), np.array(prefix_lens, np.int32))
+    kv = binding.KVCache(shape, batch, s_max, k=kk.cuda(), v=vv.cuda(),
+                         seq_len=torch.tensor(prefix_lens, dtype=torch.int32, device="cuda"))
+    return okv, kv
+
+
+def _run(gm, kv, tokens, parents, block_len, path, trace=False):
+    B, T = tokens.shape
+    buf = binding.VerifyBuffers(gm, B, T, tree=parents is not None)
+    buf.tokens.copy_(torch.from_numpy(tokens))
+    buf.block_len.copy_(torch.from_numpy(block_len))
+    if parents is not None:
+        buf.parents.copy_(torch.from_numpy(parents))
+    tr = torch.zeros(gm.trace_bytes(B, T), dtype=torch.uint8, device="cuda") if trace else None
+    gm.set_path(path)
+    gm.set_trace(tr)
+    try:
+        binding.quasar_verify(gm, kv, buf)
+        torch.cuda.synchronize()
+    finally:
+        gm.set_trace(None)
+        gm.set_path(0)
+    assert int(buf.status[0]) == 0
+    return buf, (binding.split_trace(gm, tr, B, T) if trace else None)
+
+
+# What end-to-end agreement means at these widths (see the module docstring): the benchmark's element
+# test on at least 97 % of the logits, mean |d| <= 1.2e-2, worst |d| <= 1e-1.
+def _assert_statistically_close(got, want, what, share=0.97, mean_tol=1.2e-2, worst_tol=1e-1):
+    got = np.asarray(got, np.float64)
+    want = np.asarray(want, np.float64)
+    d = np.abs(got - want)
+    inside = float(np.mean(d <= np.maximum(2e-2, 1e-2 * np.abs(want))))
+    assert inside >= share and d.mean() <= mean_tol and d.max() <= worst_tol, \
+        f"{what}: {inside:.4f} of the logits inside max(2e-2, 1e-2|o|), mean |d| {d.mean():.3e}, worst {d.max():.3e}"
+
+
+CLEAR_MARGIN = 0.25      # top-2 margin beyond which the rounding noise above cannot change the arg-max
+
+
+def _compare_end_to_end(r, buf, block_len, what):
+    lg = buf.logits.cpu().numpy()
+    for b in range(len(block_len)):
+        T = int(block_len[b])
+        _assert_statistically_close(lg[b, :T], r.logits[b, :T], f"{what}, sequence {b}")
+        safe = margins(r.logits[b, :T]) > CLEAR_MARGIN
+        assert np.array_equal(lg[b, :T].argmax(-1)[safe], r.top1[b, :T][safe])
+        path = [int(q) for q in r.accept_path[b] if q >= 0]
+        if all(safe[q] for q in path):
+            assert int(buf.accept_len[b]) == int(r.accept_len[b])
+            assert int(buf.bonus[b]) == int(r.bonus[b])
+            got_path = [int(q) for q in buf.accept_path[b].cpu().numpy() if q >= 0]
+            assert got_path == path
+
+
+def _np(t):
+    return t.float().cpu().numpy().astype(np.float64)
+
+
+def _near(name, got, want, ulps=2.5, prev=None):
+    """|got - want| within `ulps` * 2^-8 of the magnitudes involved (2^-8 relative is half a bf16 step at
+    worst, a whole one at best); for x = prev + term the rounding of the term bounds the error."""
+    mag = np.abs(want) if prev is None else np.abs(want) + np.abs(prev) + np.abs(want - prev)
+    tol = ulps * 2.0 ** -8 * np.maximum(mag, np.sqrt(np.mean(mag ** 2))) + 1e-6
+    bad = np.abs(got - want) > tol
+    assert not bad.any(), f"{name}: {bad.sum()} of {bad.size} differ, worst {np.abs(got - want).max():.3e}"
+    return float(np.mean(got != want))
+
+
+def _teacher_forced_layer0(shape, om, kv, tr, b, tokens, par, P, logits_gpu, n_layers):
+    """Every step of layer 0 (and the final norm + LM head) recomputed by the oracle from the tensor the
+    GPU recorded before it."""
+    T = len(par)
+    Hq, Hkv, D = shape.n_q_heads, shape.n_kv_heads, shape.head_dim
+    G = Hq // Hkv
+    ly = om.layers[0]
+    R = qo.bf16_round
+    x0 = _np(tr["embed"][b, :T])
+    assert np.array_equal(x0, qo.bf16_bits_to_f64(om.embed_bits[tokens[:T]]))
+    h1 = _np(tr["l0.h1"][b, :T])
+    _near("h1", h1, R(qo.rmsnorm(x0, ly.attn_norm, shape.rms_eps)))
+    qkv = _np(tr["l0.qkv"][b, :T])
+    flips = _near("qkv", qkv, R(ly.qkv(h1)))
+    assert flips < 0.01, f"qkv: {flips:.4f} of the elements rounded the other way"
+    # QK-norm + RoPE of the recorded qkv rows
+    dep = np.array(qo.block_depths(par))
+    pos = (P + dep)[:, None]
+    q = qkv[:, : Hq * D].reshape(T, Hq, D)
+    k = qkv[:, Hq * D: (Hq + Hkv) * D].reshape(T, Hkv, D)
+    if shape.qk_norm:
+        q = qo.rmsnorm(q, ly.q_norm, shape.rms_eps)
+        k = qo.rmsnorm(k, ly.k_norm, shape.rms_eps)
+    q = R(qo.rope(q, pos, shape.rope_theta))
+    k = R(qo.rope(k, pos, shape.rope_theta))
+    roped = _np(tr["l0.qkv_rope"][b, :T])
+    _near("q after RoPE", roped[:, : Hq * D], q.reshape(T, Hq * D))
+    # the rows appended to the cache: K normed and rotated, V as the GEMM produced it
+    k_new = _np(kv.k[0, b, :, P:P + T]).transpose(1, 0, 2).reshape(T, Hkv * D)
+    v_new = _np(kv.v[0, b, :, P:P + T]).transpose(1, 0, 2).reshape(T, Hkv * D)
+    _near("k after RoPE", k_new, k.reshape(T, Hkv * D))
+    assert np.array_equal(v_new, qkv[:, (Hq + Hkv) * D:])
+    # attention of the recorded queries over the GPU's own cache
+    qg = roped[:, : Hq * D].reshape(T, Hq, D)
+    mask = qo.ancestor_mask(par)
+    att = np.zeros((T, Hq, D))
+    for hk in range(Hkv):
+        kc = _np(kv.k[0, b, hk, :P + T])
+        vc = _np(kv.v[0, b, hk, :P + T])
+        att[:, hk * G:(hk + 1) * G] = qo.attention(qg[:, hk * G:(hk + 1) * G], kc, vc, P, mask)
+    attn = _np(tr["l0.attn"][b, :T])
+    _near("attention", attn, R(att).reshape(T, Hq * D))
+    x1 = _np(tr["l0.x_attn"][b, :T])
+    _near("x after attention", x1, R(x0 + R(ly.o(attn))), prev=x0)
+    act = _np(tr["l0.act"][b, :T])
+    gu = R(ly.gateup(R(qo.rmsnorm(x1, ly.mlp_norm, shape.rms_eps))))
+    _near("act", act, R(qo.silu(gu[:, : shape.ffn]) * gu[:, shape.ffn:]), ulps=8.0)
+    x2 = _np(tr["l0.x_mlp"][b, :T])
+    _near("x after MLP", x2, R(x1 + R(ly.down(act))), prev=x1)
+    # final norm and LM head from the last recorded stream
+    xl = _np(tr[f"l{n_layers - 1}.x_mlp"][b, :T])
+    hf = _np(tr["hf"][b, :T])
+    _near("final norm", hf, R(qo.rmsnorm(xl, om.final_norm, shape.rms_eps)))
+    lg = om.lm_head(hf)
+    got = logits_gpu[b, :T].astype(np.float64)
+    assert np.abs(got - lg).max() <= 5e-4, f"LM head: worst {np.abs(got - lg).max():.3e}"
+    clear = margins(lg) > 2e-3
+    assert np.array_equal(got.argmax(-1)[clear], lg.argmax(-1)[clear])
+
+
+def test_qwen3_8b_width_chain_block():
+    """B=1, 1024 cached positions, chain of 5 drafts (6 rows): the bench workload at two layers' depth,
+    through the persistent kernel (as bench.py launches it) and through the kernel-per-step path."""
+    shape = _cut(synth.SHAPES["qwen3_8b"], 2, "qwen3_8b_2l")
+    s_max = 1040
+    om, gm = _models(shape, s_max)
+    okv, kv = _caches(shape, 1, s_max, [1024])
+    tokens = synth.uniform_tokens((1, 6), shape.vocab, synth.sub_seed(2, "tokens")).numpy()
+    bl = np.array([6], np.int32)
+    # plant the oracle's own choices as the first two drafts: acceptance has something to accept
+    r = oracle.verify(om, okv, tokens, None, bl)
+    tokens[0, 1] = r.top1[0, 0]
+    r = oracle.verify(om, okv, tokens, None, bl)
+    tokens[0, 2] = r.top1[0, 1]
+    r = oracle.verify(om, okv, tokens, None, bl)
+    assert int(r.accept_len[0]) >= 2
+
+    buf2, _ = _run(gm, kv, tokens, None, bl, path=2)
+    _compare_end_to_end(r, buf2, bl, "persistent kernel")
+    assert 0 <= int(buf2.accept_len[0]) <= 5
+
+    buf1, tr = _run(gm, kv, tokens, None, bl, path=1, trace=True)
+    _compare_end_to_end(r, buf1, bl, "kernel per step")
+    _teacher_forced_layer0(shape, om, kv, tr, 0, tokens[0], list(range(-1, 5)), 1024, buf1.logits.cpu().numpy(), 2)
+    _assert_statistically_close(buf2.logits.cpu().numpy(), buf1.logits.cpu().numpy(), "the two GPU paths")
+
+
+def test_qwen3_8b_width_ragged_batch_of_eight():
+    """Eight sequences, prefixes drawn from 512..4096, chains of 8 drafts (72 rows), one layer deep."""
+    shape = _cut(synth.SHAPES["qwen3_8b"], 1, "qwen3_8b_1l")
+    s_max = 4096 + 16
+    rng = np.random.default_rng(4)
+    prefix = [int(x) for x in rng.integers(512, 4097, 8)]
+    prefix[0], prefix[1] = 4096, 512                  # both ends of the range
+    om, gm = _models(shape, s_max)
+    okv, kv = _caches(shape, 8, s_max, prefix)
+    tokens = synth.uniform_tokens((8, 9), shape.vocab, synth.sub_seed(2, "tokens")).numpy()
+    bl = np.full(8, 9, np.int32)
+    bl[3] = 4                                          # a ragged block
+    r = oracle.verify(om, okv, tokens, None, bl)
+    buf, tr = _run(gm, kv, tokens, None, bl, path=0, trace=True)
+    _compare_end_to_end(r, buf, bl, "batch of eight")
+    lg = buf.logits.cpu().numpy()
+    for b in (0, 3):
+        T = int(bl[b])
+        _teacher_forced_layer0(shape, om, kv, tr, b, tokens[b], list(range(-1, T - 1)), prefix[b], lg, 1)
+
+
+def test_qwen3_14b_width_tree_of_sixteen_nodes():
+    """Four sequences, 2048 cached positions, the 16-node draft tree (17 rows each), one layer deep."""
+    shape = _cut(synth.SHAPES["qwen3_14b"], 1, "qwen3_14b_1l")
+    s_max = 2048 + 32
+    om, gm = _models(shape, s_max)
+    okv, kv = _caches(shape, 4, s_max, [2048] * 4)
+    par1 = synth.tree_parents_16()
+    par = np.array([par1] * 4, np.int32)
+    tokens = synth.uniform_tokens((4, 17), shape.vocab, synth.sub_seed(2, "tokens")).numpy()
+    bl = np.full(4, 17, np.int32)
+    # one branch follows the verifier's own choices two levels deep
+    r = oracle.verify(om, okv, tokens, par, bl)
+    first = [i for i, q in enumerate(par1) if q == 0][1]
+    tokens[:, first] = r.top1[:, 0]
+    r = oracle.verify(om, okv, tokens, par, bl)
+    kids = [i for i, q in enumerate(par1) if q == first]
+    if kids:
+        tokens[:, kids[0]] = r.top1[:, first]
+        r = oracle.verify(om, okv, tokens, par, bl)
+    assert np.all(r.accept_len >= 1)
+    buf, tr = _run(gm, kv, tokens, par, bl, path=0, trace=True)
+    _compare_end_to_end(r, buf, bl, "tree block")
+    assert np.all(buf.accept_len.cpu().numpy() <= max(qo.block_depths(par1)))
+    _teacher_forced_layer0(shape, om, kv, tr, 1, tokens[1], par1, 2048, buf.logits.cpu().numpy(), 1)
+
+
+def test_full_depth_qwen3_8b_two_gpu_paths_agree_and_pass_is_idempotent():
+    """All 36 layers.  The persistent kernel and the kernel-per-step path are separate implementations of
+    the same pass (different summation orders, different attention splits).  After 36 layers of the flip
+    amplification described above they are apart by mean |dlogit| ~4e-2 at a logit spread of 1.3 (worst
+    ~0.25, measured); the bounds below leave a factor of two.  Each path must repeat itself bit for bit,
+    and acceptance must stay inside [0, gamma]."""
+    shape = synth.SHAPES["qwen3_8b"]
+    s_max = 1040
+    gm = binding.Model.from_master(shape, master_getter(shape, 0, "cuda"), s_max, int8=True)
+    kk, vv = synth.kv_prefix(shape, 1, s_max, seed=1, device="cuda")
+    kv = binding.KVCache(shape, 1, s_max, k=kk, v=vv, seq_len=torch.full((1,), 1024, dtype=torch.int32, device="cuda"))
+    tokens = synth.uniform_tokens((1, 6), shape.vocab, synth.sub_seed(2, "tokens")).numpy()
+    bl = np.array([6], np.int32)
+    out = {}
+    for path in (2, 1):
+        first, _ = _run(gm, kv, tokens, None, bl, path)
+        again, _ = _run(gm, kv, tokens, None, bl, path)
+        assert torch.equal(first.logits, again.logits), "the pass is not idempotent"
+        assert torch.equal(first.accept_len, again.accept_len) and torch.equal(first.bonus, again.bonus)
+        assert 0 <= int(first.accept_len[0]) <= 5 and 0 <= int(first.bonus[0]) < shape.vocab
+        lg = first.logits.cpu().numpy()[0]
+        assert np.isfinite(lg).all()
+        # the bonus token is the arg-max of the row acceptance stopped at
+        assert int(first.bonus[0]) == int(lg[int(first.accept_len[0])].argmax())
+        out[path] = (lg, int(first.accept_len[0]), int(first.bonus[0]))
+    a, b = out[2][0].astype(np.float64), out[1][0].astype(np.float64)
+    d = np.abs(a - b)
+    assert abs(a.std() - b.std()) <= 1e-2 * b.std()
+    assert d.mean() <= 8e-2 and d.max() <= 0.6, f"mean {d.mean():.3e}, worst {d.max():.3e}"
+    if margins(out[1][0]).min() > 0.6:
+        assert out[2][1:] == out[1][1:]

@@ -46,6 +46,20 @@ def test_quantize_bit_exact_all_bf16_patterns():
     assert np.array_equal(q.cpu().numpy(), oq)
 
 
+def test_linear_calls_of_different_widths_share_one_workspace():
+    """A decoder layer runs its GEMMs of different widths through one workspace, narrow ones first: a
+    call's partial sums must not land where a wider call keeps its arrival counters."""
+    shapes = [(6144, 4096), (4096, 4096), (24576, 4096), (4096, 12288), (151936, 4096), (24576, 4096)]
+    m = 6
+    size = max(binding.quasar_linear_workspace_bytes(m, n, k) for n, k in shapes)
+    shared = torch.zeros(size, dtype=torch.uint8, device="cuda")
+    for i, (n, k) in enumerate(shapes):
+        x = synth.normal_bf16((m, k), 1.0, seed=10 + i, device="cuda")
+        q, d = binding.quasar_quantize(synth.normal_bf16((n, k), 0.02, seed=20 + i, device="cuda"))
+        alone = binding.quasar_linear(x, q, d, out_f32=True)          # a zero-filled workspace of its own
+        assert torch.equal(binding.quasar_linear(x, q, d, workspace=shared, out_f32=True), alone)
+
+
 @pytest.mark.parametrize("k,n", [(4096, 6144), (4096, 4096), (4096, 24576), (12288, 4096), (4096, 151936)])
 def test_quantize_bit_exact_qwen3_8b_shapes(k, n):
     w = synth.normal_bf16((n, k), 0.02, seed=k + n, device="cuda")
