@@ -34,10 +34,12 @@ from paper_2603_01399_b200 import synth  # noqa: E402
 WORKLOAD = "qwen3-8b-shaped verify pass: B=1, prefix 1024, chain draft gamma=5 (6 block rows), int8 weights"
 PREFIX, GAMMA, BATCH = 1024, 5, 1
 METRIC = "verify-pass latency & accepted tok/s, Qwen3-8B shape; HBM GB/s as % of peak"
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the persistent kernel, from the ncu capture
-# summarised in profiles/ (a 2-layer model, scaled by the weight bytes of the full one); None while the
-# kernel has changed since that capture
-MEGAKERNEL_DRAM_BYTES_PER_LAUNCH = None
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the persistent kernel on the 2-layer case
+# of `--profile-pass --profile-layers 2` (the ncu capture summarised in profiles/), and that case's
+# algorithmic bytes.  Traffic follows the weight bytes, so a full launch is taken as the same ratio times
+# its own algorithmic bytes.  Both None while the kernel has changed since that capture.
+NCU_CASE_DRAM_BYTES = 1_018_779_000 + 7_184_896
+NCU_CASE_ALGORITHMIC_BYTES = 1_017_652_736
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 
@@ -225,6 +227,16 @@ def run_ours(args):
     accepted_job = sum_over_ranks(accepted, dist, "cuda")          # every replica verifies its own sequences
     accepted_drafts_job = sum_over_ranks(accepted_drafts, dist, "cuda")
 
+    # Random-initialised int8 and bf16 weights do not share their arg-max, so the bf16 model's draft is
+    # rarely accepted.  Beside it: the same pass on a draft that is the int8 model's own greedy continuation
+    # with the same replacement probability (the pass costs the same whatever the tokens are).
+    own = synth.corrupt_draft(greedy_continuation(binding, m_int8, kv, root, GAMMA), 0.3, shape.vocab, seed=2)
+    sbuf = binding.VerifyBuffers(m_int8, BATCH, t_rows, want_logits=False)
+    sbuf.tokens.copy_(torch.cat([root.cpu().view(-1, 1), own], dim=1).to(torch.int32))
+    binding.quasar_verify(m_int8, kv, sbuf)
+    torch.cuda.synchronize()
+    own_accepted = sum_over_ranks(int((sbuf.accept_len + 1).sum()), dist, "cuda")
+
     # the per-step skinny GEMM (used for blocks of more than 8 rows) over the model's 145 matrices in pass order
     gemm = time_gemm_sweep(binding, m_int8, shape, BATCH * t_rows, max(3, args.steps // 4))
 
@@ -249,6 +261,8 @@ def run_ours(args):
                    "launch": "one persistent cooperative kernel per step"},
         "verify_latency_ms": ms_step, "accepted_per_pass": accepted, "accepted_drafts_per_pass": accepted_drafts,
         "accepted_drafts_tok_s": accepted_drafts_job / (ms_step * 1e-3), "device_status": status,
+        "own_draft": {"what": "draft = the int8 model's own greedy continuation, each token replaced w.p. 0.3",
+                      "accepted_per_pass": own_accepted / world, "accepted_tok_s": own_accepted / (ms_step * 1e-3)},
         "pass_bytes": ab, "pass_hbm_gbs": pass_gbs, "pass_hbm_frac_of_measured_copy": pass_gbs / hbm_peak,
         "pass_hbm_frac_of_nominal_8TBs": pass_gbs / NOMINAL_HBM_GBS,
         "bf16_sibling": {"verify_latency_ms": bf16_ms, "ratio_vs_int8": bf16_ms / ms_step,
@@ -260,7 +274,9 @@ def run_ours(args):
         "gpu_launches": int(launches),
         "roofline": {"bound": "hbm", "kernel": "verify_megakernel<int8, 128> (persistent, one launch per step)",
                      "achieved": launch_gbs, "peak": hbm_peak, "unit": "GB/s", "frac": launch_gbs / hbm_peak,
-                     "peak_kind": f"{peak_kind} copy bandwidth", "traffic": MEGAKERNEL_DRAM_BYTES_PER_LAUNCH,
+                     "peak_kind": f"{peak_kind} copy bandwidth", "traffic": (round(ab["total"] * NCU_CASE_DRAM_BYTES / NCU_CASE_ALGORITHMIC_BYTES)
+                                 if NCU_CASE_DRAM_BYTES else None),
+                     "traffic_source": "ncu dram bytes of a 2-of-36-layer launch x (algorithmic bytes of this launch / of that one)",
                      "avg_launch_us": ms_step * 1e3, "bytes_per_launch": ab["total"]},
     }
     if rank == 0:
