@@ -48,10 +48,10 @@ constexpr int kThreads = kCT + 32;         // + the producer warp (9 warps: at m
 constexpr int kRowBytes = 1024;            // bytes of one weight row per stage
 constexpr int kStageBytes = 16 * kRowBytes;  // 16 weight rows
 constexpr int kStages = 8;                 // ring depth (128 KB of weights in flight per CTA)
-constexpr int kChunk = 4096;               // contraction elements whose activations a warp keeps in registers
+constexpr int kChunk = 4096;               // longest contraction whose operand rows stay in shared memory whole
+constexpr int kChunkLong = 2048;           // chunk of a longer contraction: two operand buffers, one in use while the next lands
 constexpr int kWarpBytes = kRowBytes / NW;   // bytes of a row piece one warp covers (128)
 constexpr int kSub = kWarpBytes / 64;        // 64-byte sub-slices of it: four lanes x 16 bytes each
-constexpr int kXr = 8 * kSub;                // 16-byte registers holding this thread's share of the operand chunk
 constexpr int GT = 4;                      // 16-row tiles accumulated together before a reduction
 constexpr int kKeyTile = 64;
 constexpr int kMaxRowsAttn = 32;           // query rows (heads-in-group x block rows) per kv head
@@ -67,14 +67,17 @@ constexpr int kOTileBytes = kMaxRowsAttn * 128 * 4;                      // 1638
 constexpr int kMlTileBytes = kMaxRowsAttn * 8;                           // its row maxima and sums
 constexpr int kAttnBytes = 2 * kKvTileBytes + kQTileBytes + kOTileBytes + kMlTileBytes;   // tiles of the attention phase
 constexpr int kMiscBytes = 2048;
-// The operand of a GEMM phase (<= 8 rows x one chunk, bf16) and its norm gain land in a staging buffer by
-// bulk copy before they go to registers.  The attention tiles share that buffer: the two are never alive
-// at the same time.  The reduction buffer has bytes of its own (partial sums stay parked there while the
-// next chunk of a long contraction is staged).
-constexpr int kXRowBytes = kChunk * 2;                                   // 8192
-constexpr int kXBytes = 8 * kXRowBytes;                                  // 65536
-constexpr int kGainBytes = kChunk * 2;                                   // 8192
-constexpr int kStageBufBytes = (kXBytes + kGainBytes > kAttnBytes) ? kXBytes + kGainBytes : kAttnBytes;
+// The operand of a GEMM phase (<= 8 rows x one chunk) and its norm gain land in a staging buffer by bulk
+// copy, are converted there and stay there while the phase multiplies: every stage reads its slice of
+// the rows from it.  Rows sit at a pitch of the chunk's bytes plus a pad that spreads the rows over the
+// banks.  A contraction longer than kChunk goes through two half-size buffers in turn.  The attention
+// tiles share the bytes: the two are never alive at the same time.  The reduction buffer has bytes of
+// its own.
+constexpr int kXPadInt8 = 16, kXPadBf16 = 64;
+constexpr int kXBufWhole = 8 * (kChunk * 2 + kXPadBf16) + kChunk * 2;            // rows + gain: 74240
+constexpr int kXBufLong = 8 * (kChunkLong * 2 + kXPadBf16) + kChunkLong * 2;     // 37376, twice
+constexpr int kXBufBytes = kXBufWhole > 2 * kXBufLong ? kXBufWhole : 2 * kXBufLong;
+constexpr int kStageBufBytes = kXBufBytes > kAttnBytes ? kXBufBytes : kAttnBytes;
 constexpr int kSmemBytes = kRingBytes + kRedBytes + kStageBufBytes + kMiscBytes;
 static_assert(kSmemBytes <= 227 * 1024, "shared memory budget of one SM");
 
@@ -164,11 +167,13 @@ __device__ __forceinline__ unsigned long long now_ns() {
 #ifdef QUASAR_TIMELINE
 __device__ long long g_timeline[160][256];
 __device__ long long g_timeline2[160][16][40];
+#define TL2_MARK() do { if (tl_on && lane == 0 && tl2_n[warp] < 40) s_tl2[warp][tl2_n[warp]++] = clock64(); } while (0)
 #define TL_DECL __shared__ long long s_tl[256]; int tl_n = 0;
 #define TL_MARK() do { if (threadIdx.x == 0 && tl_on && tl_n < 256) s_tl[tl_n++] = clock64(); } while (0)
 #define TL_FLUSH() do { if (threadIdx.x == 0 && tl_on) { for (int i__ = 0; i__ < tl_n; ++i__) g_timeline[blockIdx.x][i__] = s_tl[i__]; g_timeline[blockIdx.x][255] = tl_n; } } while (0)
 #else
 #define TL_DECL
+#define TL2_MARK() do { } while (0)
 #define TL_MARK() do { } while (0)
 #define TL_FLUSH() do { } while (0)
 #endif
@@ -269,7 +274,7 @@ __device__ __forceinline__ void bulk_copy(void* smem_dst, const void* gmem_src, 
 // piece, rows at a pitch of the piece's bytes.
 struct JobView {
   const unsigned char* wp;   // this CTA's repacked row range
-  int K, units, u0, u1, rows_per_tile, tiles, ngroups, nchunks, kind, n_rows;
+  int K, units, u0, u1, rows_per_tile, tiles, ngroups, nchunks, chunk, kind, n_rows;
 };
 
 __device__ __forceinline__ void job_split(int kind, int N, int K, int cta, int ncta, JobView& v) {
@@ -282,7 +287,8 @@ __device__ __forceinline__ void job_split(int kind, int N, int K, int cta, int n
   v.rows_per_tile = (kind == kJobGateUp) ? 8 : 16;
   v.tiles = (v.u1 - v.u0 + v.rows_per_tile - 1) / v.rows_per_tile;
   v.ngroups = (v.tiles + GT - 1) / GT;
-  v.nchunks = (K + kChunk - 1) / kChunk;
+  v.chunk = K <= kChunk ? K : kChunkLong;   // contraction elements per chunk
+  v.nchunks = (K + v.chunk - 1) / v.chunk;
 }
 
 template <bool W_INT8>
@@ -325,7 +331,6 @@ struct Pipe {
 template <bool W_INT8>
 __device__ void producer_loop(const MegaParams& p, const Pipe& pipe, int cta, int ncta) {
   constexpr int kElemBytes = W_INT8 ? 1 : 2;
-  constexpr int kChunkBytes = kChunk * kElemBytes;
   if ((threadIdx.x & 31) != 0) return;   // one thread issues every copy
   uint64_t policy;
   asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;\n" : "=l"(policy));
@@ -337,6 +342,7 @@ __device__ void producer_loop(const MegaParams& p, const Pipe& pipe, int cta, in
     const JobView v = job_view<W_INT8>(p.jobs, job, cta, ncta);
     const unsigned char* src = v.wp;
     const int kbytes = v.K * kElemBytes;
+    const int kChunkBytes = v.chunk * kElemBytes;
     for (int tg = 0; tg < v.ngroups && ok; ++tg) {
       const int gt = min(GT, v.tiles - tg * GT);
       for (int kc = 0; kc < v.nchunks && ok; ++kc) {
@@ -402,22 +408,7 @@ struct GridSync {
   }
 };
 
-// ---- operand load: the <= 8 activation rows of this warp's share of a contraction chunk ----------
-// A stage holds a 1024-byte piece of every weight row of a tile; warp w reads bytes [kWarpBytes w,
-// kWarpBytes (w + 1)) of the piece as kSub sub-slices of 64 bytes, lane (g, t) the 16 bytes at 16 t of each.
-// int8 weights: stage s, sub-slice u covers k = base + 1024 s + kWarpBytes w + 64 u + 16 t + (0..15), held
-// in xr[2 (s kSub + u)], xr[.. + 1] (fp16).  bf16 weights: half as many elements per byte range, held in
-// xr[s kSub + u] (bf16).
-template <bool W_INT8>
-__device__ __forceinline__ int x_index(int i, int kbase, int warp, int t) {
-  if (W_INT8) {
-    const int su = i >> 1, s = su / kSub, u = su % kSub;
-    return kbase + s * 1024 + warp * kWarpBytes + u * 64 + t * 16 + (i & 1) * 8;
-  }
-  const int s = i / kSub, u = i % kSub;
-  return kbase + s * 512 + (warp * kWarpBytes + u * 64 + t * 16) / 2;
-}
-
+// ---- operand staging: the <= 8 activation rows of a contraction chunk, in shared memory -------------
 // Plain bulk copy global -> shared (both addresses and the size multiples of 16 bytes), counted on `bar`.
 __device__ __forceinline__ void bulk_copy_plain(void* smem_dst, const void* gmem_src, uint32_t bytes, uint64_t* bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n" ::"r"(
@@ -434,108 +425,108 @@ __device__ __forceinline__ void bulk_store(void* gmem_dst, const void* smem_src,
                : "memory");
 }
 
-// One thread asks for the operand chunk: the M rows (one copy when the chunk is the whole contraction,
-// else one per row) and the norm gain, into the staging buffer.  A bulk copy keeps the whole request in
-// flight at once, which 16-byte loads from 256 threads do not.
-__device__ __forceinline__ void request_operand(unsigned char* x_s, const __nv_bfloat16* src, int ld, int M, int K,
-                                                int kbase, const __nv_bfloat16* gain, uint64_t* xbar) {
-  const uint32_t cbytes = (uint32_t)min(kChunk, K - kbase) * 2;
-  const bool whole = K <= kChunk;
-  asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");   // earlier reads / writes of the buffer come first
-  mbar_arrive_expect_tx(xbar, (uint32_t)M * cbytes + (gain != nullptr ? cbytes : 0u));
-  if (whole) {
-    bulk_copy_plain(x_s, src, (uint32_t)M * cbytes, xbar);
-  } else {
-    for (int m = 0; m < M; ++m) bulk_copy_plain(x_s + m * kXRowBytes, src + (size_t)m * ld + kbase, cbytes, xbar);
+// Geometry of an operand buffer: M rows of `len` elements (2 bytes each) at a padded pitch, the chunk of
+// the norm gain behind the eighth row.
+template <bool W_INT8>
+__device__ __forceinline__ int x_pitch(int chunk) { return chunk * 2 + (W_INT8 ? kXPadInt8 : kXPadBf16); }
+template <bool W_INT8>
+__device__ __forceinline__ int x_buf_bytes(int chunk) { return 8 * x_pitch<W_INT8>(chunk) + chunk * 2; }
+
+// Warp 0 asks for an operand chunk: lane m < M copies row m, lane 8 the norm gain.  A bulk copy keeps the
+// whole request in flight at once, which 16-byte loads do not.
+template <bool W_INT8>
+__device__ __forceinline__ void request_operand(unsigned char* buf, const __nv_bfloat16* src, int ld, int M, int chunk,
+                                                int kbase, int len, const __nv_bfloat16* gain, uint64_t* xbar, int lane) {
+  const uint32_t cbytes = (uint32_t)len * 2;
+  const int pitch = x_pitch<W_INT8>(chunk);
+  if (lane == 0) {
+    asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");   // earlier reads / writes of the buffer come first
+    mbar_arrive_expect_tx(xbar, (uint32_t)M * cbytes + (gain != nullptr ? cbytes : 0u));
   }
-  if (gain != nullptr) bulk_copy_plain(x_s + kXBytes, gain + kbase, cbytes, xbar);
+  __syncwarp();
+  if (lane < M) bulk_copy_plain(buf + lane * pitch, src + (size_t)lane * ld + kbase, cbytes, xbar);
+  if (lane == 8 && gain != nullptr) bulk_copy_plain(buf + 8 * pitch, gain + kbase, cbytes, xbar);
 }
 
-// The staged operand chunk is converted where it lies, every thread taking 16-byte pieces in turn (a
-// rolled loop: little code).  Normed GEMMs: h = bf16(x * r * gain), the RMSNorm output rounded where the
-// decoder layer rounds it.  int8 weights: h times the row's power-of-two scale, as fp16 (exact unless
-// the scaled value falls below the fp16 normal range); the scale is folded into rs[row] = r * scale,
-// which commutes with the rounding.  Without a norm rs is the scale alone and the gain is one.
+// The staged chunk is converted where it lies (a rolled loop: little code, hot after its first turn);
+// 32 threads per row, each taking every 32nd 16-byte piece.  Normed GEMMs: h = bf16(x * r * gain), the
+// RMSNorm output rounded where the decoder layer rounds it.  int8 weights: h times the row's
+// power-of-two scale, as fp16 (exact unless the scaled value falls below the fp16 normal range); the
+// scale is folded into rs[row] = r * scale, which commutes with the rounding.  Without a norm rs is the
+// scale alone and the gain is one.
 template <bool W_INT8>
-__device__ __forceinline__ void convert_staged(unsigned char* x_s, int M, int K, int kbase, bool has_gain,
+__device__ __forceinline__ void convert_staged(unsigned char* buf, int M, int chunk, int len, bool has_gain,
                                                const float* rs_row) {
-  const int per_row = min(kChunk, K - kbase) / 8;          // 16-byte pieces of a row
-  const int pitch = K <= kChunk ? K * 2 : kXRowBytes;
+  const int row = threadIdx.x >> 5;
+  if (row >= M) return;
+  const int pitch = x_pitch<W_INT8>(chunk);
+  const float rs = rs_row[row];
+  unsigned char* xrow = buf + row * pitch;
+  const unsigned char* gain = buf + 8 * pitch;
 #pragma unroll 2
-  for (int idx = threadIdx.x; idx < M * per_row; idx += kCT) {
-    const int row = idx / per_row, c = idx - row * per_row;
-    uint4* px = reinterpret_cast<uint4*>(x_s + row * pitch + c * 16);
-    uint4 xv = *px;
+  for (int c = (threadIdx.x & 31) * 16; c < len * 2; c += 512) {
+    uint4 xv = *reinterpret_cast<const uint4*>(xrow + c);
     uint4 gv = make_uint4(0x3f803f80u, 0x3f803f80u, 0x3f803f80u, 0x3f803f80u);   // bf16 ones
-    if (has_gain) gv = *reinterpret_cast<const uint4*>(x_s + kXBytes + c * 16);
-    const float rs = rs_row[row];
+    if (has_gain) gv = *reinterpret_cast<const uint4*>(gain + c);
     uint32_t* w = reinterpret_cast<uint32_t*>(&xv);
-    const __nv_bfloat162* gp = reinterpret_cast<const __nv_bfloat162*>(&gv);
+    const uint32_t* gw = reinterpret_cast<const uint32_t*>(&gv);
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
-      const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w[e]));
-      const float2 gf = __bfloat1622float2(gp[e]);
-      const __nv_bfloat162 h = __floats2bfloat162_rn(f.x * rs * gf.x, f.y * rs * gf.y);
+      // a bf16 is the upper half of an fp32
+      const float x0 = __uint_as_float(w[e] << 16), x1 = __uint_as_float(w[e] & 0xffff0000u);
+      const float g0 = __uint_as_float(gw[e] << 16), g1 = __uint_as_float(gw[e] & 0xffff0000u);
+      const __nv_bfloat162 h = __floats2bfloat162_rn(x0 * rs * g0, x1 * rs * g1);
       if (W_INT8) {
-        const float2 hf = __bfloat1622float2(h);
-        const __half2 q = __floats2half2_rn(hf.x, hf.y);
+        const uint32_t hb = *reinterpret_cast<const uint32_t*>(&h);
+        const __half2 q = __floats2half2_rn(__uint_as_float(hb << 16), __uint_as_float(hb & 0xffff0000u));
         w[e] = *reinterpret_cast<const uint32_t*>(&q);
       } else {
         w[e] = *reinterpret_cast<const uint32_t*>(&h);
       }
     }
-    *px = xv;
-  }
-}
-
-// this warp's share of the (converted) chunk, from the staging buffer to registers
-template <bool W_INT8>
-__device__ __forceinline__ void read_operand(uint4 (&xr)[kXr], const unsigned char* x_s, int M, int K, int kbase,
-                                             int warp, int g, int t) {
-  const int pitch = K <= kChunk ? K * 2 : kXRowBytes;
-#pragma unroll
-  for (int i = 0; i < kXr; ++i) {
-    const int k = x_index<W_INT8>(i, kbase, warp, t);
-    xr[i] = make_uint4(0, 0, 0, 0);
-    if (k < K && g < M) xr[i] = *reinterpret_cast<const uint4*>(x_s + g * pitch + (k - kbase) * 2);
+    *reinterpret_cast<uint4*>(xrow + c) = xv;
   }
 }
 
 // One stage = one block [rows][pb bytes].  MMA row g of the tile is block row ra, MMA row g + 8
 // block row rb; the 16-byte pieces of a row are XOR-swizzled by its parity when pb is a multiple
-// of 128.  off_a[u] / off_b[u] are this lane's byte offsets for sub-slice u (computed once per tile
-// and piece size).  The four MMAs of a sub-slice go to separate accumulators so that no MMA waits
-// for the one before it.
+// of 128.  off_a[u] / off_b[u] are this lane's byte offsets for sub-slice u.  `xs` points at this
+// lane's share of operand row g for the stage: for sub-slice u the 16 weight bytes of the lane meet 16
+// (int8 weights) or 8 (bf16 weights) consecutive operand elements.  The four MMAs of a sub-slice go to
+// separate accumulators so that no MMA waits for the one before it.
 template <bool W_INT8>
-__device__ __forceinline__ void consume_stage(const unsigned char* stage, int s, const int (&off_a)[kSub],
-                                              const int (&off_b)[kSub], unsigned valid_mask, const uint4 (&xr)[kXr],
-                                              float (&acc)[4][4]) {
-  uint4 wa[kSub], wb[kSub];
+__device__ __forceinline__ void consume_stage(const unsigned char* stage, const unsigned char* xs, const int (&off_a)[kSub],
+                                              const int (&off_b)[kSub], unsigned valid_mask, float (&acc)[4][4]) {
+  uint4 wa[kSub], wb[kSub], x0[kSub], x1[kSub];
 #pragma unroll
   for (int u = 0; u < kSub; ++u) {
     wa[u] = *reinterpret_cast<const uint4*>(stage + off_a[u]);
     wb[u] = *reinterpret_cast<const uint4*>(stage + off_b[u]);
+    x0[u] = *reinterpret_cast<const uint4*>(xs + u * (W_INT8 ? 128 : 64));
+    if (W_INT8) x1[u] = *reinterpret_cast<const uint4*>(xs + u * 128 + 16);
   }
 #pragma unroll
   for (int u = 0; u < kSub; ++u) {
+    // Past the end of a short piece the lane reads bytes no copy of this stage has written and operand
+    // elements beyond the contraction: both are replaced by zeros (stale bytes may be NaN patterns).
+    if (!((valid_mask >> u) & 1u)) {
+      x0[u] = make_uint4(0, 0, 0, 0);
+      x1[u] = make_uint4(0, 0, 0, 0);
+      if (!W_INT8) { wa[u] = make_uint4(0, 0, 0, 0); wb[u] = make_uint4(0, 0, 0, 0); }
+    }
     if (W_INT8) {
-      // bytes no copy has written convert to finite numbers: they meet zero activations (k beyond K)
-      // or land in accumulator rows that are never stored (rows beyond the tile)
-      const uint4 x0 = xr[2 * (s * kSub + u)], x1 = xr[2 * (s * kSub + u) + 1];
       uint32_t a0, a1, a2, a3;
       u8x4_to_f16x4(wa[u].x, a0, a2); u8x4_to_f16x4(wb[u].x, a1, a3);
-      mma16816_f16(acc[0], a0, a1, a2, a3, x0.x, x0.y);
+      mma16816_f16(acc[0], a0, a1, a2, a3, x0[u].x, x0[u].y);
       u8x4_to_f16x4(wa[u].y, a0, a2); u8x4_to_f16x4(wb[u].y, a1, a3);
-      mma16816_f16(acc[1], a0, a1, a2, a3, x0.z, x0.w);
+      mma16816_f16(acc[1], a0, a1, a2, a3, x0[u].z, x0[u].w);
       u8x4_to_f16x4(wa[u].z, a0, a2); u8x4_to_f16x4(wb[u].z, a1, a3);
-      mma16816_f16(acc[2], a0, a1, a2, a3, x1.x, x1.y);
+      mma16816_f16(acc[2], a0, a1, a2, a3, x1[u].x, x1[u].y);
       u8x4_to_f16x4(wa[u].w, a0, a2); u8x4_to_f16x4(wb[u].w, a1, a3);
-      mma16816_f16(acc[3], a0, a1, a2, a3, x1.z, x1.w);
+      mma16816_f16(acc[3], a0, a1, a2, a3, x1[u].z, x1[u].w);
     } else {
-      if (!((valid_mask >> u) & 1u)) { wa[u] = make_uint4(0, 0, 0, 0); wb[u] = make_uint4(0, 0, 0, 0); }  // stale bytes may be NaN patterns
-      const uint4 x0 = xr[s * kSub + u];
-      mma16816_bf16(acc[2 * (u & 1)], wa[u].x, wb[u].x, wa[u].y, wb[u].y, x0.x, x0.y);
-      mma16816_bf16(acc[2 * (u & 1) + 1], wa[u].z, wb[u].z, wa[u].w, wb[u].w, x0.z, x0.w);
+      mma16816_bf16(acc[2 * (u & 1)], wa[u].x, wb[u].x, wa[u].y, wb[u].y, x0[u].x, x0[u].y);
+      mma16816_bf16(acc[2 * (u & 1) + 1], wa[u].z, wb[u].z, wa[u].w, wb[u].w, x0[u].z, x0[u].w);
     }
   }
 }
@@ -583,7 +574,7 @@ struct GemmPhase {
 #ifdef QUASAR_TIMELINE
     __shared__ long long s_tl2[16][40];
     __shared__ int tl2_n[16];
-    if (threadIdx.x < 16) tl2_n[threadIdx.x] = 0;
+    if (threadIdx.x < 16) { tl2_n[threadIdx.x] = 0; for (int i = 0; i < 40; ++i) s_tl2[threadIdx.x][i] = 0; }
     cbar();
 #endif
 #ifdef QUASAR_TIMELINE
@@ -593,8 +584,11 @@ struct GemmPhase {
     const bool tl_on = jb.kind == QUASAR_TL_KIND && job >= p.n_jobs - 5;
 #endif
     TL_MARK();
-    uint4 xr[kXr];
     bool have_x = false, first = true;
+    bool requested = false;   // the next chunk's copy is already in flight
+    int xb = 0;               // operand buffer in use (a long contraction alternates between two)
+    const int xpitch = x_pitch<W_INT8>(v.chunk);
+    const int xbuf_bytes = x_buf_bytes<W_INT8>(v.chunk);
     float ss_run = 0.f;   // threads 0..7 (o / down): sum of squares of the row of x this CTA has written
     float best = -INFINITY;   // LM head: this thread's running arg-max over the elements it finishes
     int best_i = 0x7fffffff;
@@ -628,7 +622,10 @@ struct GemmPhase {
         if (!have_x) {
           TL_MARK();
           // every warp is past its last use of the buffer's other tenants (epilogue / attention end in a CTA barrier)
-          if (threadIdx.x == 0) request_operand(x_s, xsrc, ld, M, jb.K, kc * kChunk, jb.gain, xbar);
+          if (warp == 0 && !requested)
+            request_operand<W_INT8>(x_s + xb * xbuf_bytes, xsrc, ld, M, v.chunk, kc * v.chunk, min(v.chunk, jb.K - kc * v.chunk),
+                                    jb.gain, xbar, lane);
+          requested = false;
           TL_MARK();
           if (first) {   // the row factors ride on the same round trip as the first chunk's loads
             first = false;
@@ -661,7 +658,7 @@ struct GemmPhase {
             if (warp == 0 && t == 0) {
               misc[kMiscRs + g] = rnorm * xscale;   // conversion factor of operand row g
               misc[kMiscInvScale + g] = inv;
-            }   // read in the epilogues, behind a CTA barrier
+            }   // read by the conversion and in the epilogues, behind a CTA barrier
           }
           {
             int got = 1;
@@ -673,60 +670,60 @@ struct GemmPhase {
           TL_MARK();
           if (W_INT8 || normed) {
             cbar();   // the rows' factors are published
-            convert_staged<W_INT8>(x_s, M, jb.K, kc * kChunk, normed, misc + kMiscRs);
-            cbar();
+            convert_staged<W_INT8>(x_s + xb * xbuf_bytes, M, v.chunk, min(v.chunk, jb.K - kc * v.chunk), normed, misc + kMiscRs);
           }
-          read_operand<W_INT8>(xr, x_s, M, jb.K, kc * kChunk, warp, g, t);
-          cbar();   // every warp has its share: the staging buffer may be refilled
+          cbar();   // the chunk is ready; every warp is past the tiles of the chunk before it
           TL_MARK();
+          if (v.nchunks > 1 && (kc + 1 < v.nchunks || tg + 1 < v.ngroups)) {
+            // a long contraction reloads its chunks for every tile group: the next one lands in the
+            // other buffer while this one is multiplied
+            const int nk = kc + 1 < v.nchunks ? kc + 1 : 0;
+            if (warp == 0)
+              request_operand<W_INT8>(x_s + (xb ^ 1) * xbuf_bytes, xsrc, ld, M, v.chunk, nk * v.chunk,
+                                      min(v.chunk, jb.K - nk * v.chunk), jb.gain, xbar, lane);
+            requested = true;
+          }
         }
-        have_x = (v.nchunks == 1);   // a long contraction reloads its chunks for every tile group
-        const int kbase = kc * kChunk;
-        const int cb = min(kChunk, jb.K - kbase) * kElemBytes;        // bytes of a weight row in this chunk
-        const int pb_last = cb - (cb - 1) / kRowBytes * kRowBytes;    // bytes of its last piece
+        const int cb = min(v.chunk, jb.K - kc * v.chunk) * kElemBytes;   // bytes of a weight row in this chunk
+        const int nst = (cb + kRowBytes - 1) / kRowBytes;                 // stages per tile
+        const int pb_last = cb - (nst - 1) * kRowBytes;                   // bytes of a row's last piece
+        // this lane's share of operand row g: the elements that meet the warp's weight bytes, stage by stage
+        const unsigned char* xlane = x_s + xb * xbuf_bytes + g * xpitch + (warp * kWarpBytes + t * 16) * (2 / kElemBytes);
 #pragma unroll 1
         for (int tile = 0; tile < gt; ++tile) {
           // block rows behind MMA rows g and g + 8 (rows past the tile stay inside the stage and feed
           // accumulator rows that are never stored)
           const int ra = g;
           const int rb = v.kind == kJobGateUp ? tile_units(v, tg * GT + tile) + g : g + 8;
-          int oa_full[kSub], ob_full[kSub], oa_last[kSub], ob_last[kSub];
-#pragma unroll
-          for (int u = 0; u < kSub; ++u) {
-            oa_full[u] = block_offset(ra, kRowBytes, warp, u, t);
-            ob_full[u] = block_offset(rb, kRowBytes, warp, u, t);
-            oa_last[u] = block_offset(ra, pb_last, warp, u, t);
-            ob_last[u] = block_offset(rb, pb_last, warp, u, t);
-          }
           float ch[4][4];
 #pragma unroll
           for (int i = 0; i < 4; ++i) ch[i][0] = ch[i][1] = ch[i][2] = ch[i][3] = 0.f;
+#pragma unroll 1
+          for (int st = 0; st < nst; ++st) {   // rolled: the stage's code stays in the instruction cache
+            const bool last = st == nst - 1;
+            const int pb = last ? pb_last : kRowBytes;
+            int oa[kSub], ob[kSub];
+            unsigned valid_mask = 0;
 #pragma unroll
-          for (int s = 0; s < SPC; ++s) {
-            const int b0 = s * kRowBytes;
-            if (b0 < cb) {
-              const bool last = b0 + kRowBytes >= cb;
-              // one lane polls the stage's barrier for the warp; the warp-level barrier then orders the
-              // other lanes' reads after the arrival it has seen
-              int got = 1;
-              if (lane == 0) got = mbar_wait(pipe.full + slot, phase, pipe.abort_flag, pipe.status) ? 1 : 0;
-              got = __shfl_sync(0xffffffffu, got, 0);
-              if (!got) return false;
+            for (int u = 0; u < kSub; ++u) {
               // a lane past the end of a short piece reads inside the stage (offset < 16 KB) but not its own data
-              int oa[kSub], ob[kSub];
-              unsigned valid_mask = 0;
-#pragma unroll
-              for (int u = 0; u < kSub; ++u) {
-                const bool lane_valid = b0 + warp * kWarpBytes + u * 64 + t * 16 < cb;
-                valid_mask |= (lane_valid ? 1u : 0u) << u;
-                oa[u] = last ? (lane_valid ? oa_last[u] : 0) : oa_full[u];
-                ob[u] = last ? (lane_valid ? ob_last[u] : 0) : ob_full[u];
-              }
-              consume_stage<W_INT8>(pipe.ring + slot * kStageBytes, s, oa, ob, valid_mask, xr, ch);
-              __syncwarp();
-              if (lane == 0) mbar_arrive(pipe.empty + slot);
-              if (++slot == kStages) { slot = 0; phase ^= 1u; }
+              const bool lane_valid = warp * kWarpBytes + u * 64 + t * 16 < pb;
+              valid_mask |= (lane_valid ? 1u : 0u) << u;
+              oa[u] = lane_valid ? block_offset(ra, pb, warp, u, t) : 0;
+              ob[u] = lane_valid ? block_offset(rb, pb, warp, u, t) : 0;
             }
+            // one lane polls the stage's barrier for the warp; the warp-level barrier then orders the
+            // other lanes' reads after the arrival it has seen
+            int got = 1;
+            if (lane == 0) got = mbar_wait(pipe.full + slot, phase, pipe.abort_flag, pipe.status) ? 1 : 0;
+            got = __shfl_sync(0xffffffffu, got, 0);
+            if (!got) return false;
+            TL2_MARK();
+            consume_stage<W_INT8>(pipe.ring + slot * kStageBytes, xlane + st * (kRowBytes * 2 / kElemBytes), oa, ob, valid_mask, ch);
+            __syncwarp();
+            TL2_MARK();
+            if (lane == 0) mbar_arrive(pipe.empty + slot);
+            if (++slot == kStages) { slot = 0; phase ^= 1u; }
           }
           float* r = red + ((warp * GT + tile) * 16) * 8;
           float2 lo = make_float2((ch[0][0] + ch[1][0]) + (ch[2][0] + ch[3][0]), (ch[0][1] + ch[1][1]) + (ch[2][1] + ch[3][1]));
@@ -740,6 +737,8 @@ struct GemmPhase {
           *plo = lo;
           *phi = hi;
         }
+        if (v.nchunks > 1) xb ^= 1;   // the next chunk is (or will be) in the other buffer
+        else have_x = true;           // a short contraction keeps its operand for every tile group
       }
 #ifdef QUASAR_GEMM_TIMER
       tacc[5] += (unsigned)(clock64() - c_t0);
@@ -1498,7 +1497,13 @@ __global__ void __launch_bounds__(kThreads, 1) verify_megakernel(const MegaParam
 #ifdef QUASAR_PHASE_TIMER
   if (threadIdx.x == 0) g_phase_n[blockIdx.x] = mark_n;
 #endif
-  if (!ok && threadIdx.x == 0) *abort_flag = 1;  // tells the producer to stop issuing
+  if (!ok && threadIdx.x == 0) {
+    *abort_flag = 1;  // tells the producer to stop issuing
+    // an operand chunk may have been requested and never waited for: let it land (it takes a few
+    // microseconds at most) before the CTA gives its shared memory back
+    const unsigned long long t0 = now_ns();
+    while (!mbar_try(xbar, xphase) && now_ns() - t0 < 100000ull) {}
+  }
 }
 
 // ---- model creation: permute every CTA's row range into its consumption order ------------------
@@ -1509,10 +1514,10 @@ template <bool W_INT8>
 __global__ void __launch_bounds__(256) repack_kernel(const unsigned char* __restrict__ w, unsigned char* __restrict__ wp,
                                                      int N, int K, int kind, int ncta) {
   constexpr int kElemBytes = W_INT8 ? 1 : 2;
-  constexpr int kChunkBytes = kChunk * kElemBytes;
   const int cta = blockIdx.y, tile_g = blockIdx.x;
   JobView v;
   job_split(kind, N, K, cta, ncta, v);
+  const int kChunkBytes = v.chunk * kElemBytes;
   if (tile_g >= v.tiles) return;
   const int mult = kind == kJobGateUp ? 2 : 1;
   const int tg = tile_g / GT, tile = tile_g % GT;
