@@ -166,7 +166,11 @@ __device__ __forceinline__ unsigned long long now_ns() {
 
 #ifdef QUASAR_TIMELINE
 __device__ long long g_timeline[160][256];
+#ifndef QUASAR_TL_KIND
+#define QUASAR_TL_KIND 4
+#endif
 __device__ long long g_timeline2[160][16][40];
+__device__ long long g_timeline3[160][64];   // producer: clock at the issue of each stage of the watched phase
 #define TL2_MARK() do { if (tl_on && lane == 0 && tl2_n[warp] < 40) s_tl2[warp][tl2_n[warp]++] = clock64(); } while (0)
 #define TL_DECL __shared__ long long s_tl[256]; int tl_n = 0;
 #define TL_MARK() do { if (threadIdx.x == 0 && tl_on && tl_n < 256) s_tl[tl_n++] = clock64(); } while (0)
@@ -196,6 +200,7 @@ __device__ long long g_attn_tmp_unused;
     if (threadIdx.x == 0 && mark_n < kMaxMarks) g_phase_clk[blockIdx.x][mark_n++] = clock64(); \
   } while (0)
 #ifdef QUASAR_GEMM_TIMER
+#define STAGE_CLK(i) do { const long long n__ = clock64(); tacc[i] += (unsigned)(n__ - stage_prev); stage_prev = n__; } while (0)
 #define GEMM_CLK(i, expr)                                           \
   do {                                                              \
     const long long c0__ = clock64();                               \
@@ -204,11 +209,13 @@ __device__ long long g_attn_tmp_unused;
   } while (0)
 #else
 #define GEMM_CLK(i, expr) do { expr; } while (0)
+#define STAGE_CLK(i) do { } while (0)
 #endif
 #else
 #define ATTN_T(i) do { } while (0)
 #define PHASE_MARK() do { } while (0)
 #define GEMM_CLK(i, expr) do { expr; } while (0)
+#define STAGE_CLK(i) do { } while (0)
 #endif
 
 // ---- mbarriers ----------------------------------------------------------------------------
@@ -338,6 +345,9 @@ __device__ void producer_loop(const MegaParams& p, const Pipe& pipe, int cta, in
   uint32_t phase = 0;
   long long issued = 0;
   bool ok = true;
+#ifdef QUASAR_TIMELINE
+  int tl3_n = 0;
+#endif
   for (int job = 0; job < p.n_jobs && ok; ++job) {
     const JobView v = job_view<W_INT8>(p.jobs, job, cta, ncta);
     const unsigned char* src = v.wp;
@@ -352,6 +362,9 @@ __device__ void producer_loop(const MegaParams& p, const Pipe& pipe, int cta, in
           for (int b0 = 0; b0 < cb; b0 += kRowBytes) {
             const uint32_t bytes = (uint32_t)(rows * min(kRowBytes, cb - b0));
             if (!mbar_wait(pipe.empty + slot, phase ^ 1u, pipe.abort_flag, pipe.status)) { ok = false; break; }
+#ifdef QUASAR_TIMELINE
+            if (p.jobs[job].kind == QUASAR_TL_KIND && job >= p.n_jobs - 5 && tl3_n < 64) g_timeline3[blockIdx.x][tl3_n++] = clock64();
+#endif
             mbar_arrive_expect_tx(pipe.full + slot, bytes);
             bulk_copy(pipe.ring + slot * kStageBytes, src, bytes, pipe.full + slot, policy);
             src += bytes;
@@ -554,6 +567,7 @@ struct GemmPhase {
     uint32_t phase = phase_io;
 #ifdef QUASAR_GEMM_TIMER
     unsigned tacc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    long long stage_prev = clock64();
 #endif
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
     const JobView v = job_view<W_INT8>(p.jobs, job, cta, ncta);
@@ -578,9 +592,6 @@ struct GemmPhase {
     cbar();
 #endif
 #ifdef QUASAR_TIMELINE
-#ifndef QUASAR_TL_KIND
-#define QUASAR_TL_KIND 4
-#endif
     const bool tl_on = jb.kind == QUASAR_TL_KIND && job >= p.n_jobs - 5;
 #endif
     TL_MARK();
@@ -698,32 +709,41 @@ struct GemmPhase {
           float ch[4][4];
 #pragma unroll
           for (int i = 0; i < 4; ++i) ch[i][0] = ch[i][1] = ch[i][2] = ch[i][3] = 0.f;
+          // this lane's byte offsets in a stage of full pieces and in the stage of the rows' last pieces
+          int oa_full[kSub], ob_full[kSub], oa_last[kSub], ob_last[kSub];
+          unsigned mask_last = 0;
+#pragma unroll
+          for (int u = 0; u < kSub; ++u) {
+            // a lane past the end of a short piece reads inside the stage (offset < 16 KB) but not its own data
+            const bool lane_valid = warp * kWarpBytes + u * 64 + t * 16 < pb_last;
+            mask_last |= (lane_valid ? 1u : 0u) << u;
+            oa_full[u] = block_offset(ra, kRowBytes, warp, u, t);
+            ob_full[u] = block_offset(rb, kRowBytes, warp, u, t);
+            oa_last[u] = lane_valid ? block_offset(ra, pb_last, warp, u, t) : 0;
+            ob_last[u] = lane_valid ? block_offset(rb, pb_last, warp, u, t) : 0;
+          }
 #pragma unroll 1
           for (int st = 0; st < nst; ++st) {   // rolled: the stage's code stays in the instruction cache
             const bool last = st == nst - 1;
-            const int pb = last ? pb_last : kRowBytes;
             int oa[kSub], ob[kSub];
-            unsigned valid_mask = 0;
 #pragma unroll
             for (int u = 0; u < kSub; ++u) {
-              // a lane past the end of a short piece reads inside the stage (offset < 16 KB) but not its own data
-              const bool lane_valid = warp * kWarpBytes + u * 64 + t * 16 < pb;
-              valid_mask |= (lane_valid ? 1u : 0u) << u;
-              oa[u] = lane_valid ? block_offset(ra, pb, warp, u, t) : 0;
-              ob[u] = lane_valid ? block_offset(rb, pb, warp, u, t) : 0;
+              oa[u] = last ? oa_last[u] : oa_full[u];
+              ob[u] = last ? ob_last[u] : ob_full[u];
             }
-            // one lane polls the stage's barrier for the warp; the warp-level barrier then orders the
-            // other lanes' reads after the arrival it has seen
-            int got = 1;
-            if (lane == 0) got = mbar_wait(pipe.full + slot, phase, pipe.abort_flag, pipe.status) ? 1 : 0;
-            got = __shfl_sync(0xffffffffu, got, 0);
-            if (!got) return false;
+            const unsigned valid_mask = last ? mask_last : (1u << kSub) - 1u;
+            // every lane tests the stage's barrier itself (one instruction per warp, no broadcast afterwards)
+            STAGE_CLK(0);
+            if (!__all_sync(0xffffffffu, mbar_wait(pipe.full + slot, phase, pipe.abort_flag, pipe.status))) return false;   // the warp leaves together
+            STAGE_CLK(1);
             TL2_MARK();
             consume_stage<W_INT8>(pipe.ring + slot * kStageBytes, xlane + st * (kRowBytes * 2 / kElemBytes), oa, ob, valid_mask, ch);
             __syncwarp();
+            STAGE_CLK(2);
             TL2_MARK();
             if (lane == 0) mbar_arrive(pipe.empty + slot);
             if (++slot == kStages) { slot = 0; phase ^= 1u; }
+            STAGE_CLK(3);
           }
           float* r = red + ((warp * GT + tile) * 16) * 8;
           float2 lo = make_float2((ch[0][0] + ch[1][0]) + (ch[2][0] + ch[3][0]), (ch[0][1] + ch[1][1]) + (ch[2][1] + ch[3][1]));
@@ -1572,6 +1592,10 @@ extern "C" int quasar_debug_phase_marks(long long* clk_host, int* n_host) {
   return kMaxMarks;
 }
 #ifdef QUASAR_TIMELINE
+extern "C" int quasar_debug_timeline3(long long* host) {
+  if (cudaMemcpyFromSymbol(host, g_timeline3, sizeof(long long) * 160 * 64) != cudaSuccess) return -1;
+  return 0;
+}
 extern "C" int quasar_debug_timeline2(long long* host) {
   if (cudaMemcpyFromSymbol(host, g_timeline2, sizeof(long long) * 160 * 16 * 40) != cudaSuccess) return -1;
   return 0;
