@@ -604,6 +604,14 @@ struct GemmPhase {
     float best = -INFINITY;   // LM head: this thread's running arg-max over the elements it finishes
     int best_i = 0x7fffffff;
 
+    // The first operand chunk is asked for before anything else: its round trip to L2 is the longest wait
+    // of the phase's prologue.  (Every warp is past its last use of the buffer's other tenants: the
+    // epilogue and the attention phase end in a CTA barrier.)
+    if (v.tiles > 0) {
+      if (warp == 0)
+        request_operand<W_INT8>(x_s, xsrc, ld, M, v.chunk, 0, min(v.chunk, jb.K), jb.gain, xbar, lane);
+      requested = true;
+    }
     for (int tg = 0; tg < v.ngroups; ++tg) {
       const int gt = min(GT, v.tiles - tg * GT);
       // The elements this thread finishes in the group's epilogue (element e = thread + it * kCT of the
