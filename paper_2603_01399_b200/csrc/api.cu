@@ -65,7 +65,7 @@ size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
 
 // Layout of the verify workspace; every offset is a multiple of 256 bytes.
 struct Workspace {
-  size_t x, h, qkv, attn, gu, act, logits, top1, anc, depth, valid, lin, att, cand, ss_part, amax, attn_count, barrier, total;
+  size_t x, h, qkv, attn, gu, act, attn16, act16, logits, top1, anc, depth, valid, lin, att, cand, ss_part, amax, attn_count, barrier, total;
   size_t lin_bytes, att_bytes;
 };
 
@@ -83,6 +83,8 @@ Workspace layout(const quasar_config& c, int B, int T_max, int s_max) {
   w.attn = take(M * (size_t)c.n_q_heads * c.head_dim * 2);
   w.gu = take(M * 2 * (size_t)c.ffn * 2);
   w.act = take(M * (size_t)c.ffn * 2);
+  w.attn16 = take(M * (size_t)c.n_q_heads * c.head_dim * 2);
+  w.act16 = take(M * (size_t)c.ffn * 2);
   w.logits = take(M * (size_t)c.vocab * 4);
   w.top1 = take(M * 4);
   w.anc = take(M * 8);
@@ -248,7 +250,9 @@ int verify_impl(quasar_model* m, const quasar_kv* kv, const int32_t* tokens, con
     p.rope_table = m->rope_table;
     p.tokens = tokens; p.parents = parents; p.block_len = block_len; p.seq_len = kv->seq_len;
     p.k_cache = reinterpret_cast<__nv_bfloat16*>(kv->k); p.v_cache = reinterpret_cast<__nv_bfloat16*>(kv->v);
-    p.x = x; p.qkv = qkv; p.attn = attn; p.act = act; p.logits = logits_out; p.top1 = top1; p.bi = bi;
+    p.x = x; p.qkv = qkv; p.attn = attn; p.act = act;
+    p.attn16 = reinterpret_cast<unsigned short*>(wsp + ws.attn16);
+    p.act16 = reinterpret_cast<unsigned short*>(wsp + ws.act16); p.logits = logits_out; p.top1 = top1; p.bi = bi;
     p.attn_nchunk = mega_attn_nchunk(kv->s_max);
     p.attn_rpad = mega_attn_rpad(T_max, Hq, Hkv);
     const size_t rows = (size_t)B * Hkv * p.attn_nchunk * p.attn_rpad;

@@ -577,6 +577,12 @@ struct GemmPhase {
     const bool residual = jb.kind == kJobO || jb.kind == kJobDown;
     const __nv_bfloat16* xsrc = jb.kind == kJobO ? p.attn : (jb.kind == kJobDown ? p.act : p.x);
     const int ld = jb.K;
+    // int8 weights: the operands of the o and down projections also exist as fp16, exactly what the
+    // conversion below would make of them as long as no row needs a scale (no element beyond 2^15).
+    // The phase asks for that copy first and falls back to the bf16 tensor if a row maximum says otherwise.
+    const bool has16 = W_INT8 && (jb.kind == kJobO || jb.kind == kJobDown);
+    const __nv_bfloat16* xsrc16 = reinterpret_cast<const __nv_bfloat16*>(jb.kind == kJobO ? p.attn16 : p.act16);
+    bool direct = has16;   // the staged chunk needs no conversion
 
     // The operand of the first chunk and the per-row factors, all in ONE round trip to L2: the
     // loads of the operand, of the gains and of the statistics are issued together.  Normed GEMMs:
@@ -609,7 +615,7 @@ struct GemmPhase {
     // epilogue and the attention phase end in a CTA barrier.)
     if (v.tiles > 0) {
       if (warp == 0)
-        request_operand<W_INT8>(x_s, xsrc, ld, M, v.chunk, 0, min(v.chunk, jb.K), jb.gain, xbar, lane);
+        request_operand<W_INT8>(x_s, direct ? xsrc16 : xsrc, ld, M, v.chunk, 0, min(v.chunk, jb.K), jb.gain, xbar, lane);
       requested = true;
     }
     for (int tg = 0; tg < v.ngroups; ++tg) {
@@ -642,10 +648,11 @@ struct GemmPhase {
           TL_MARK();
           // every warp is past its last use of the buffer's other tenants (epilogue / attention end in a CTA barrier)
           if (warp == 0 && !requested)
-            request_operand<W_INT8>(x_s + xb * xbuf_bytes, xsrc, ld, M, v.chunk, kc * v.chunk, min(v.chunk, jb.K - kc * v.chunk),
-                                    jb.gain, xbar, lane);
+            request_operand<W_INT8>(x_s + xb * xbuf_bytes, direct ? xsrc16 : xsrc, ld, M, v.chunk, kc * v.chunk,
+                                    min(v.chunk, jb.K - kc * v.chunk), jb.gain, xbar, lane);
           requested = false;
           TL_MARK();
+          bool again = false;   // the fp16 copy was asked for, but a row needs a scale
           if (first) {   // the row factors ride on the same round trip as the first chunk's loads
             first = false;
             float rnorm = 1.f, xscale = 1.f, inv = 1.f;
@@ -673,6 +680,14 @@ struct GemmPhase {
                 xscale = ldexpf(1.f, 15 - e);       // scaled row maximum <= 2^15
                 inv = ldexpf(1.f, e - 15);
               }
+              if (has16) {   // the same answer in every warp: all read the same eight maxima
+                float top = mx;   // (NaN compares false: such a row goes the converting way below)
+                top = fmaxf(top, __shfl_xor_sync(0xffffffffu, top, 4));
+                top = fmaxf(top, __shfl_xor_sync(0xffffffffu, top, 8));
+                top = fmaxf(top, __shfl_xor_sync(0xffffffffu, top, 16));
+                direct = __all_sync(0xffffffffu, mx <= 32768.f) && top <= 32768.f;
+                again = !direct;
+              }
             }
             if (warp == 0 && t == 0) {
               misc[kMiscRs + g] = rnorm * xscale;   // conversion factor of operand row g
@@ -687,7 +702,18 @@ struct GemmPhase {
             xphase ^= 1u;
           }
           TL_MARK();
-          if (W_INT8 || normed) {
+          if (again) {   // rare: fetch the chunk once more, from the bf16 tensor
+            cbar();      // every warp has seen the first copy land
+            if (warp == 0)
+              request_operand<W_INT8>(x_s + xb * xbuf_bytes, xsrc, ld, M, v.chunk, kc * v.chunk,
+                                      min(v.chunk, jb.K - kc * v.chunk), jb.gain, xbar, lane);
+            int got = 1;
+            if (lane == 0) got = mbar_wait(xbar, xphase, pipe.abort_flag, pipe.status) ? 1 : 0;
+            got = __shfl_sync(0xffffffffu, got, 0);
+            if (!got) return false;
+            xphase ^= 1u;
+          }
+          if (!direct && (W_INT8 || normed)) {
             cbar();   // the rows' factors are published
             convert_staged<W_INT8>(x_s + xb * xbuf_bytes, M, v.chunk, min(v.chunk, jb.K - kc * v.chunk), normed, misc + kMiscRs);
           }
@@ -698,7 +724,7 @@ struct GemmPhase {
             // other buffer while this one is multiplied
             const int nk = kc + 1 < v.nchunks ? kc + 1 : 0;
             if (warp == 0)
-              request_operand<W_INT8>(x_s + (xb ^ 1) * xbuf_bytes, xsrc, ld, M, v.chunk, nk * v.chunk,
+              request_operand<W_INT8>(x_s + (xb ^ 1) * xbuf_bytes, direct ? xsrc16 : xsrc, ld, M, v.chunk, nk * v.chunk,
                                       min(v.chunk, jb.K - nk * v.chunk), jb.gain, xbar, lane);
             requested = true;
           }
@@ -847,6 +873,7 @@ struct GemmPhase {
         const float up = bf16_round_f(reduce_at(red, tile, row + 8, col) * unit * d1);
         const __nv_bfloat16 av = __float2bfloat16_rn(gate / (1.0f + expf(-gate)) * up);
         p.act[(size_t)col * v.units + unit_idx] = av;
+        if (W_INT8) p.act16[(size_t)col * v.units + unit_idx] = __half_as_ushort(__float2half_rn(__bfloat162float(av)));
         a = fabsf(__bfloat162float(av));
       }
       if (W_INT8) {   // row maximum of the next GEMM's operand (8 consecutive lanes share a row)
@@ -1067,7 +1094,11 @@ __device__ __noinline__ void attention_phase(const MegaParams& p, int layer, boo
     const int b = m / p.T_max, i = m % p.T_max;
     if (!p.bi.valid[b] || i >= p.block_len[b]) {
       uint4* dst = reinterpret_cast<uint4*>(p.attn + (size_t)m * p.Hq * D);
-      for (int j = threadIdx.x; j < p.Hq * D / 8; j += kCT) dst[j] = make_uint4(0, 0, 0, 0);
+      uint4* dst16 = reinterpret_cast<uint4*>(p.attn16 + (size_t)m * p.Hq * D);
+      for (int j = threadIdx.x; j < p.Hq * D / 8; j += kCT) {
+        dst[j] = make_uint4(0, 0, 0, 0);
+        dst16[j] = make_uint4(0, 0, 0, 0);
+      }
     }
   }
 
@@ -1373,13 +1404,15 @@ __device__ __noinline__ void attention_phase(const MegaParams& p, int layer, boo
           const float inv = 1.0f / dsum;
           const int i = r / G, hq = hk * G + (r % G);
           const int m = b * p.T_max + i;
-          __nv_bfloat16* dst = p.attn + (size_t)m * p.Hq * D + (size_t)hq * D + lane * (D / 32);
+          const size_t off = (size_t)m * p.Hq * D + (size_t)hq * D + lane * (D / 32);
+          __nv_bfloat16* dst = p.attn + off;
           float amax = 0.f;
 #pragma unroll
           for (int e = 0; e < D / 64; ++e) {
             const __nv_bfloat162 pr = __floats2bfloat162_rn(tot[2 * e] * inv, tot[2 * e + 1] * inv);
             reinterpret_cast<__nv_bfloat162*>(dst)[e] = pr;
             const float2 back = __bfloat1622float2(pr);
+            if (want_amax) reinterpret_cast<__half2*>(p.attn16 + off)[e] = __floats2half2_rn(back.x, back.y);
             amax = fmaxf(amax, fmaxf(fabsf(back.x), fabsf(back.y)));
           }
           if (want_amax) {   // row maximum of the o projection's operand

@@ -35,6 +35,9 @@ struct MegaParams {
   __nv_bfloat16 *k_cache, *v_cache;
   // workspace
   __nv_bfloat16 *x, *qkv, *attn, *act;
+  // int8 weights: the o projection's and the down projection's operands once more as fp16 (what the MMA
+  // takes), written beside the bf16 tensors by the phases that produce them
+  unsigned short *attn16, *act16;
   float* logits;            // [M][V] or nullptr
   int32_t* top1;
   BlockInfo bi;

@@ -6,7 +6,7 @@ import torch
 import oracle
 from oracle import quasar_oracle as qo
 from paper_2603_01399_b200 import binding, synth
-from tests.common import (gpu_model, logits_close, margins, oracle_greedy_continuation, oracle_model,
+from tests.common import (gpu_model, logits_close, margins, master_getter, oracle_greedy_continuation, oracle_model,
                           prefill_oracle)
 
 pytestmark = pytest.mark.gpu
@@ -310,3 +310,37 @@ def test_persistent_kernel_refuses_blocks_it_cannot_hold(world):
         assert e.value.code == -2
     finally:
         gm.set_path(0)
+
+
+@pytest.mark.parametrize("path", [1, 2])
+def test_activations_beyond_the_fp16_range(path):
+    """Gate/up weights scaled up until SiLU(gate)*up exceeds 65504: the int8 path multiplies fp16 operands,
+    so such rows must go through their power-of-two scale (and the persistent kernel must fall back from
+    its ready-made fp16 copy of the activations to the bf16 tensor).  bf16 holds these values without
+    trouble, and so does the oracle."""
+    shape = synth.SHAPES["tiny_qknorm"]
+    base = master_getter(shape, 0, "cpu")
+
+    def get(kind, layer=0):
+        w = base(kind, layer)
+        return (w.float() * 400.0).to(torch.bfloat16) if kind == "gateup" else w
+
+    om = oracle.build_model(shape, lambda kind, layer: synth.bf16_bits(get(kind, layer)), int8=True)
+    gm = binding.Model.from_master(shape, get, S_MAX, int8=True)
+    okv = oracle.new_kv(om, 1, S_MAX)
+    toks = synth.uniform_tokens((24,), shape.vocab, synth.sub_seed(2, "tokens")).numpy()
+    prefill_oracle(om, okv, toks[:19], chunk=8)
+    tokens = toks[19:24].reshape(1, 5).astype(np.int32)
+    bl = np.array([5], np.int32)
+    r = oracle.verify(om, _copy(okv), tokens, None, bl, want_trace=True)
+    assert max(np.abs(r.trace[f"l{l}.act.b0"]).max() for l in range(shape.n_layers)) > 65504.0
+    kv, buf, _ = _run_gpu(shape, gm, okv, tokens, None, bl, path=path)
+    assert int(buf.status[0]) == 0
+    got = buf.logits.cpu().numpy()[0].astype(np.float64)
+    want = r.logits[0].astype(np.float64)
+    assert np.isfinite(got).all()
+    # the logits are as large as the activations: tolerance relative to the row's spread
+    tol = 1e-2 * np.maximum(np.abs(want), want.std(axis=-1, keepdims=True)) + 2e-2
+    assert np.all(np.abs(got - want) <= tol), float(np.abs(got - want).max())
+    safe = margins(r.logits[0]) > 0.05 * want.std()
+    assert np.array_equal(got.argmax(-1)[safe], r.top1[0][safe])
