@@ -84,7 +84,7 @@ static_assert(kSmemBytes <= 227 * 1024, "shared memory budget of one SM");
 // misc region (floats): [0,128) per-warp row sums, [128,136) running arg-max values, [136,144) its
 // indices, [144,152) 1/scale of the operand rows, [152,184) per-tile sums of squares, [200] abort flag, [256,512) candidates / per-warp
 // row maxima, byte 1536.. the mbarriers.
-constexpr int kMiscRowSum = 0, kMiscRunV = 128, kMiscRunI = 136, kMiscInvScale = 144, kMiscPart = 152, kMiscFlag = 190, kMiscRs = 192, kMiscAbort = 200,
+constexpr int kMiscRowSum = 0, kMiscRunV = 128, kMiscRunI = 136, kMiscInvScale = 144, kMiscPart = 152, kMiscFlag = 190, kMiscRs = 192, kMiscAbort = 200, kMiscJob = 208 /* two descriptors of 40 bytes */,
               kMiscCand = 256, kMiscBarBytes = 1536;   // 2 kStages + 1 barriers of 8 bytes
 
 __device__ __forceinline__ void mma16816_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
@@ -299,6 +299,14 @@ __device__ __forceinline__ void job_split(int kind, int N, int K, int cta, int n
 }
 
 template <bool W_INT8>
+__device__ __forceinline__ JobView job_view_of(const MegaJob& jb, int cta, int ncta) {
+  JobView v;
+  job_split(jb.kind, jb.N, jb.K, cta, ncta, v);
+  const size_t row_bytes = (size_t)jb.K * (W_INT8 ? 1 : 2);
+  v.wp = reinterpret_cast<const unsigned char*>(jb.wp) + (size_t)(jb.kind == kJobGateUp ? 2 * v.u0 : v.u0) * row_bytes;
+  return v;
+}
+template <bool W_INT8>
 __device__ __forceinline__ JobView job_view(const MegaJob* jobs, int j, int cta, int ncta) {
   JobView v;
   const MegaJob jb = jobs[j];
@@ -470,14 +478,16 @@ __device__ __forceinline__ void request_operand(unsigned char* buf, const __nv_b
 template <bool W_INT8>
 __device__ __forceinline__ void convert_staged(unsigned char* buf, int M, int chunk, int len, bool has_gain,
                                                const float* rs_row) {
-  const int row = threadIdx.x >> 5;
-  if (row >= M) return;
   const int pitch = x_pitch<W_INT8>(chunk);
-  const float rs = rs_row[row];
-  unsigned char* xrow = buf + row * pitch;
   const unsigned char* gain = buf + 8 * pitch;
+  // the M rows' 16-byte pieces, dealt to all threads in turn (a power-of-two row length keeps the
+  // division a shift in the common case; neighbours in a warp take neighbouring pieces)
+  const int per_row = len / 8;
 #pragma unroll 2
-  for (int c = (threadIdx.x & 31) * 16; c < len * 2; c += 512) {
+  for (int i = threadIdx.x; i < M * per_row; i += kCT) {
+    const int row = i / per_row, c = (i - row * per_row) * 16;
+    const float rs = rs_row[row];
+    unsigned char* xrow = buf + row * pitch;
     uint4 xv = *reinterpret_cast<const uint4*>(xrow + c);
     uint4 gv = make_uint4(0x3f803f80u, 0x3f803f80u, 0x3f803f80u, 0x3f803f80u);   // bf16 ones
     if (has_gain) gv = *reinterpret_cast<const uint4*>(gain + c);
@@ -570,8 +580,13 @@ struct GemmPhase {
     long long stage_prev = clock64();
 #endif
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
-    const JobView v = job_view<W_INT8>(p.jobs, job, cta, ncta);
-    const MegaJob jb = p.jobs[job];
+    // The phase's descriptor was fetched into shared memory during the phase before (a load from global
+    // memory here would be the first thing every warp waits for); thread 0 now fetches the next one into
+    // the other slot, which nobody has read since the phase before last.
+    MegaJob* job_s = reinterpret_cast<MegaJob*>(misc + kMiscJob);
+    const MegaJob jb = job_s[job & 1];
+    if (threadIdx.x == 0 && job + 1 < p.n_jobs) job_s[(job + 1) & 1] = p.jobs[job + 1];
+    const JobView v = job_view_of<W_INT8>(jb, cta, ncta);
     const int M = p.M;
     const bool normed = jb.gain != nullptr;
     const bool residual = jb.kind == kJobO || jb.kind == kJobDown;
@@ -1506,6 +1521,7 @@ __global__ void __launch_bounds__(kThreads, 1) verify_megakernel(const MegaParam
     mbar_init(xbar + 1, 1);
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
   }
+  if (threadIdx.x == 32) reinterpret_cast<MegaJob*>(misc + kMiscJob)[0] = p.jobs[0];
   if (threadIdx.x < 8) {  // running arg-max of this CTA
     misc[kMiscRunV + threadIdx.x] = -INFINITY;
     reinterpret_cast<int*>(misc + kMiscRunI)[threadIdx.x] = 0x7fffffff;
