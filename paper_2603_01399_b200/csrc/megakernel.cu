@@ -565,8 +565,6 @@ __device__ __forceinline__ int block_offset(int r, int pb, int warp, int u, int 
 template <bool W_INT8>
 struct GemmPhase {
   static constexpr int kElemBytes = W_INT8 ? 1 : 2;
-  static constexpr int kStageElems = kRowBytes / kElemBytes;
-  static constexpr int SPC = kChunk / kStageElems;   // stages per chunk: 4 (int8) or 8 (bf16)
   static constexpr int kItems = GT * 128 / kCT;   // epilogue elements per consumer thread and tile group
   static_assert(kItems * kCT == GT * 128 && kCT % 128 == 0, "epilogue elements divide evenly; a thread keeps its operand row");
 
