@@ -5,27 +5,30 @@
 //
 //  * Each weight matrix is cut into contiguous row ranges, one per CTA, balanced to a single
 //    row, so all SMs stream the same number of bytes and no cross-CTA reduction exists.
-//    Inside a CTA the 16 consumer warps split the contraction index; their partial sums meet
+//    Inside a CTA the 8 consumer warps split the contraction index; their partial sums meet
 //    in shared memory in a fixed order (deterministic results).
 //  * At model creation the bytes of every CTA's row range are permuted (same size, same
 //    place) into the order in which that CTA consumes them: blocks of <= 16 rows x 1024
 //    bytes, each block contiguous, 16-byte pieces XOR-swizzled for conflict-free 128-bit
 //    shared-memory reads, int8 sign bits pre-flipped.  A ring stage is then ONE bulk
 //    asynchronous copy (cp.async.bulk) of up to 16 KB from a pointer that only moves forward:
-//    measured on B200, 16 KB copies stream at 7.0 TB/s where 1 KB row pieces reach 2.9 TB/s
+//    measured on B200, 16 KB copies stream at 6.2-7.0 TB/s where 1 KB row pieces reach 2.9 TB/s
 //    (the copy engine's cost is per request).
 //  * A dedicated producer warp walks a STATIC schedule covering every GEMM of the pass and
 //    fills the ring (completion counted in bytes by an mbarrier per stage).  The schedule
 //    does not depend on activations, so the producer keeps prefetching the next GEMM's
 //    weights while the consumer warps are in an epilogue, an attention phase or a grid
-//    barrier (160 KB in flight per SM), and loading costs the consumers no instructions.
-//  * int8 -> fp16 in registers at one instruction per weight: the byte, stored with its sign
+//    barrier (128 KB in flight per SM), and loading costs the consumers no instructions.
+//  * int8 -> fp16 in registers at one instruction per two weights: the byte, stored with its sign
 //    bit flipped, becomes the low mantissa byte of the fp16 number 1024 + (w + 128), and one
 //    packed subtraction of 1152 leaves w exactly.  The activations are bf16 values converted
 //    to fp16 (exact; a per-row power-of-two pre-scale keeps any bf16 row inside the fp16
 //    range), so mma.m16n8k16 f16 x f16 -> f32 computes the same products the bf16 operands
-//    would.  The weights are the 16-row operand, the <= 8 activation rows the 8-wide operand
-//    held in registers for a whole phase.
+//    would.  The weights are the 16-row operand, the <= 8 activation rows the 8-wide operand:
+//    they are brought into shared memory by bulk copy at the head of a phase, converted there
+//    once, and every stage reads its slice of them (the stage loop is rolled so that its code
+//    stays in the instruction cache).  The o and down projections find their operands already
+//    as fp16, written beside the bf16 tensors by the phases that produce them.
 //  * RMSNorm is fused into the operand load of the following GEMM, SwiGLU / residual adds
 //    into the GEMM epilogues, QK-RMSNorm + RoPE + KV append into the attention phase.
 //
@@ -60,7 +63,7 @@ constexpr unsigned long long kWaitBudgetNs = 2000000000ull;  // every device-sid
 
 // ---- shared memory map --------------------------------------------------------------------
 constexpr int kRingBytes = kStages * kStageBytes;                        // 131072
-constexpr int kRedBytes = NW * GT * 128 * 4;                             // 32768
+constexpr int kRedBytes = NW * GT * 128 * 4;                             // 16384
 constexpr int kKvTileBytes = kKeyTile * (128 + 8) * 2;                   // 17408 (D = 128)
 constexpr int kQTileBytes = kMaxRowsAttn * (128 + 8) * 2;                // 17408
 constexpr int kOTileBytes = kMaxRowsAttn * 128 * 4;                      // 16384: a CTA's partial output before it is stored
@@ -338,7 +341,7 @@ __device__ __forceinline__ int block_row_to_global(const JobView& v, int tile, i
 struct Pipe {
   unsigned char* ring;
   uint64_t* full;    // [kStages] producer -> consumers: the stage's bytes have landed
-  uint64_t* empty;   // [kStages] consumers -> producer: all 16 warps are done with the stage
+  uint64_t* empty;   // [kStages] consumers -> producer: every consumer warp is done with the stage
   volatile int* abort_flag;
   int32_t* status;
 };
@@ -869,7 +872,7 @@ struct GemmPhase {
     return s;
   }
 
-  // One output element per thread: sum the 16 warps' partials, apply the step size (and the operand's
+  // One output element per thread: sum the warps' partials, apply the step size (and the operand's
   // scale), then what the step of the pass asks for.
   __device__ __forceinline__ static void epilogue(const MegaParams& p, const MegaJob& jb, const JobView& v, int job,
                                                   const EpiItem& ei, float d0, float d1, float resid, float& best,
