@@ -344,3 +344,27 @@ def test_activations_beyond_the_fp16_range(path):
     assert np.all(np.abs(got - want) <= tol), float(np.abs(got - want).max())
     safe = margins(r.logits[0]) > 0.05 * want.std()
     assert np.array_equal(got.argmax(-1)[safe], r.top1[0][safe])
+
+
+def test_full_product_tree_of_28_nodes(world):
+    """The other reading of "depth 4, branching [4, 2, 1, 1]": the full product tree (4 + 8 + 8 + 8 nodes,
+    29 rows with the root), one branch following the int8 model's own greedy continuation."""
+    shape, om, gm, okv, root = world
+    par = synth.tree_parents_full((4, 2, 1, 1))
+    T = len(par)
+    assert T == 29 and max(synth.depths(par)) == 4
+    tokens = synth.uniform_tokens((1, T), shape.vocab, synth.sub_seed(5, "tokens")).numpy().astype(np.int32)
+    tokens[0, 0] = root
+    g = oracle_greedy_continuation(om, okv, root, 4)
+    node = 0
+    for t in g:   # walk down the LAST child at every level
+        node = [i for i, q in enumerate(par) if q == node][-1]
+        tokens[0, node] = t
+    parents = np.array([par], np.int32)
+    bl = np.array([T], np.int32)
+    r = oracle.verify(om, _copy(okv), tokens, parents, bl)
+    if margins(r.logits[0, :T]).min() > 5e-2:
+        assert int(r.accept_len[0]) == 4
+    kv, buf, _ = _run_gpu(shape, gm, okv, tokens, parents, bl)
+    assert int(buf.status[0]) == 0
+    _check_against_oracle(shape, r, buf, bl)
