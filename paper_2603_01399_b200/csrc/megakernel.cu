@@ -405,12 +405,19 @@ struct GridSync {
   unsigned ncta;
   unsigned epoch;
   volatile int* abort_flag;  // shared memory
-  __device__ bool sync() {
+  // The barrier in two halves.  arrive(): this CTA's part of the phase is done and visible.  wait():
+  // every CTA's part is.  Between the two a CTA may do whatever neither reads what other CTAs wrote in
+  // that phase nor overwrites what they may still be reading.
+  __device__ void arrive() {
     cbar();
+    ++epoch;
     if (threadIdx.x == 0) {
-      ++epoch;
       __threadfence();
       atomicAdd(counter, 1u);
+    }
+  }
+  __device__ bool wait() {
+    if (threadIdx.x == 0) {
       const unsigned target = epoch * ncta;
       const unsigned long long t0 = now_ns();
       unsigned polls = 0;
@@ -424,11 +431,13 @@ struct GridSync {
           break;
         }
       }
-    } else {
-      epoch++;
     }
     cbar();
     return *abort_flag == 0;
+  }
+  __device__ bool sync() {
+    arrive();
+    return wait();
   }
 };
 
@@ -573,7 +582,7 @@ struct GemmPhase {
 
   __device__ __forceinline__ static bool run(const MegaParams& p, int job, const Pipe& pipe, int& slot_io,
                                              uint32_t& phase_io, float* red, float* misc, unsigned char* x_s, uint64_t* xbar,
-                                             uint32_t& xphase, int cta, int ncta) {
+                                             uint32_t& xphase, int cta, int ncta, GridSync& gs) {
     int slot = slot_io;
     uint32_t phase = phase_io;
 #ifdef QUASAR_GEMM_TIMER
@@ -626,14 +635,9 @@ struct GemmPhase {
     float best = -INFINITY;   // LM head: this thread's running arg-max over the elements it finishes
     int best_i = 0x7fffffff;
 
-    // The first operand chunk is asked for before anything else: its round trip to L2 is the longest wait
-    // of the phase's prologue.  (Every warp is past its last use of the buffer's other tenants: the
-    // epilogue and the attention phase end in a CTA barrier.)
-    if (v.tiles > 0) {
-      if (warp == 0)
-        request_operand<W_INT8>(x_s, direct ? xsrc16 : xsrc, ld, M, v.chunk, 0, min(v.chunk, jb.K), jb.gain, xbar, lane);
-      requested = true;
-    }
+    // The caller has arrived at the grid barrier that ends the phase before; this phase waits for it only
+    // where it first needs that phase's results (below, after the loads that do not depend on them).
+    if (v.ngroups == 0 && !gs.wait()) return false;
     for (int tg = 0; tg < v.ngroups; ++tg) {
       const int gt = min(GT, v.tiles - tg * GT);
       // The elements this thread finishes in the group's epilogue (element e = thread + it * kCT of the
@@ -652,6 +656,17 @@ struct GemmPhase {
           }
           if (residual) resid[it] = ld_early_bf16_cg(p.x + (size_t)ei.col * jb.N + ei.unit);
         }
+      }
+      if (tg == 0) {
+        // (the step sizes and residuals above do not depend on the phase before: the residual stream was
+        // last written two phases ago)  Now the operand: every CTA's part of it must be there.
+        if (!gs.wait()) return false;
+        // Its first chunk is asked for at once: the round trip to L2 is the longest wait of the prologue.
+        // (Every warp is past its last use of the buffer's other tenants: the epilogue and the attention
+        // phase end in a CTA barrier.)
+        if (warp == 0)
+          request_operand<W_INT8>(x_s, direct ? xsrc16 : xsrc, ld, M, v.chunk, 0, min(v.chunk, jb.K), jb.gain, xbar, lane);
+        requested = true;
       }
 
       // Accumulators live for one tile and one chunk; each warp then parks them in its own part of
@@ -1545,20 +1560,22 @@ __global__ void __launch_bounds__(kThreads, 1) verify_megakernel(const MegaParam
   PHASE_MARK();
   prep_phase(p, misc, cta, ncta);
   PHASE_MARK();
-  ok = gs.sync();
+  gs.arrive();
   PHASE_MARK();
   // the GEMMs of the pass in order (qkv, o, gate+up, down per layer, then the LM head); attention follows every qkv
   for (int job = 0; job < p.n_jobs && ok; ++job) {
-    if (!(ok = GemmPhase<W_INT8>::run(p, job, pipe, slot, phase, red, misc, x_s, xbar, xphase, cta, ncta))) break;
-    if ((job & 3) == 0 && job != p.n_jobs - 1) attention_prefetch<D>(p, job >> 2, k_s, v_s, cta);
+    // (every GEMM phase waits, inside, for the grid barrier that the phase before it arrived at)
+    if (!(ok = GemmPhase<W_INT8>::run(p, job, pipe, slot, phase, red, misc, x_s, xbar, xphase, cta, ncta, gs))) break;
     PHASE_MARK();
     if (job == p.n_jobs - 1) break;   // the LM head is followed by the candidate exchange below
-    if (!(ok = gs.sync())) break;
+    gs.arrive();
     PHASE_MARK();
     if ((job & 3) == 0) {
+      attention_prefetch<D>(p, job >> 2, k_s, v_s, cta);   // reads the cached prefix only: nothing of this phase
+      if (!(ok = gs.wait())) break;
       attention_phase<D>(p, job >> 2, W_INT8, k_s, v_s, q_s, misc, xbar, xphase, xphase2, cta, ncta);
       PHASE_MARK();
-      if (!(ok = gs.sync())) break;
+      gs.arrive();
       PHASE_MARK();
     }
   }
