@@ -25,7 +25,11 @@ namespace {
 constexpr int kWarps = 4;
 constexpr int kThreads = kWarps * 32;
 constexpr int kBlockN = kWarps * 16;  // output channels per CTA
-constexpr int kSub = 512;             // contraction elements staged in shared memory at a time
+constexpr int kSub = 512;             // contraction elements staged in shared memory at a time (blocks of up to 32 rows)
+// Wider blocks stage half as much at a time: the activations of 72 rows would otherwise take 72 KB per CTA
+// and leave an SM with three CTAs (12 warps) to hide the weight loads behind.
+template <int NT>
+__host__ __device__ constexpr int sub_of() { return NT > 4 ? 256 : 512; }
 constexpr int kMaxSplit = 32;
 // The arrival counters of the split-K reduction take a region of fixed size at the start of the
 // workspace, so that calls of different widths can share one workspace: no call's partial sums
@@ -93,6 +97,7 @@ __device__ __forceinline__ float epilogue_value(float acc, float d, const __nv_b
 template <int NT, bool W_INT8>
 __global__ void __launch_bounds__(kThreads) skinny_gemm_kernel(GemmArgs a) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
+  constexpr int kSub = sub_of<NT>();
   uint4* xs = reinterpret_cast<uint4*>(smem_raw);  // [NT*8][kSub/8] 16-byte chunks, swizzled
   constexpr int kChunksPerRow = kSub / 8;
   constexpr int kStepK = W_INT8 ? 64 : 32;  // contraction elements one warp step covers
@@ -256,7 +261,7 @@ SplitPlan plan_split(int64_t N, int64_t K) {
 
 template <int NT, bool W_INT8>
 int launch_nt(const GemmArgs& a, const SplitPlan& p, cudaStream_t stream) {
-  const size_t smem = (size_t)NT * 8 * kSub * sizeof(__nv_bfloat16);
+  const size_t smem = (size_t)NT * 8 * sub_of<NT>() * sizeof(__nv_bfloat16);
   static bool configured = false;
   if (smem > 48 * 1024 && !configured) {
     QUASAR_CUDA_CHECK(cudaFuncSetAttribute(skinny_gemm_kernel<NT, W_INT8>,
