@@ -202,6 +202,22 @@ def test_qwen3_8b_width_chain_block():
     _assert_statistically_close(buf2.logits.cpu().numpy(), buf1.logits.cpu().numpy(), "the two GPU paths")
 
 
+def test_qwen3_8b_width_bf16_weight_sibling():
+    """The bf16-weight pass (same kernels, no quantisation) at full width, one layer deep, through both paths."""
+    shape = _cut(synth.SHAPES["qwen3_8b"], 1, "qwen3_8b_1l_bf16")
+    s_max = 1040
+    get = master_getter(shape, 0, "cpu")
+    om = oracle.build_model(shape, lambda kind, layer: synth.bf16_bits(get(kind, layer)), int8=False)
+    gm = binding.Model.from_master(shape, get, s_max, int8=False)
+    okv, kv = _caches(shape, 1, s_max, [1024])
+    tokens = synth.uniform_tokens((1, 6), shape.vocab, synth.sub_seed(2, "tokens")).numpy()
+    bl = np.array([6], np.int32)
+    r = oracle.verify(om, okv, tokens, None, bl)
+    for path in (2, 1):
+        buf, _ = _run(gm, kv, tokens, None, bl, path=path)
+        _compare_end_to_end(r, buf, bl, f"bf16 weights, path {path}")
+
+
 def test_qwen3_8b_width_ragged_batch_of_eight():
     """Eight sequences, prefixes drawn from 512..4096, chains of 8 drafts (72 rows), one layer deep."""
     shape = _cut(synth.SHAPES["qwen3_8b"], 1, "qwen3_8b_1l")
