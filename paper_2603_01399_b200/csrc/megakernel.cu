@@ -412,8 +412,9 @@ struct GridSync {
     cbar();
     ++epoch;
     if (threadIdx.x == 0) {
-      __threadfence();
-      atomicAdd(counter, 1u);
+      // release at GPU scope: everything this CTA wrote before the barrier above (it orders the other
+      // threads' writes before this one) is visible to whoever acquires the count
+      asm volatile("red.release.gpu.global.add.u32 [%0], %1;\n" ::"l"(counter), "r"(1u) : "memory");
     }
   }
   __device__ bool wait() {
