@@ -1394,44 +1394,76 @@ __device__ __noinline__ void attention_phase(const MegaParams& p, int layer, boo
     cbar();
     ATTN_T(3);
     if (*last_flag) {
-      // warp w adds the chunks w, w + NW, ... of a row (lane l: four output dimensions), then the
-      // warps' sums meet in shared memory in warp order
+      // Two rows at a time, half of the warps each: warp ws of a half adds the chunks ws, ws + NW/2, ...
+      // of its row (lane l: four output dimensions); the warps' sums meet in shared memory in warp order.
+      // All loads of a row - every chunk's (m, l) for the row maximum, this warp's chunks' partial
+      // outputs - are issued before the first of them is used: one round trip to L2 per pair of rows.
       float* part = o_s;                                   // [NW][D + 4] floats; the partial has left
       constexpr int kPS = 128 + 4;
+      constexpr int kHalf = NW / 2, kPre = 4;
+      const int half = warp / kHalf, ws = warp % kHalf;
 #pragma unroll 1
-      for (int r = c; r < R; r += nch) {
-        float mx = -INFINITY;
-        for (int cc = lane; cc < nch; cc += 32) mx = fmaxf(mx, __ldcg(p.ml_part + (slot0 + (size_t)cc * p.attn_rpad + r) * 2));
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+      for (int r0 = c; r0 < R; r0 += 2 * nch) {
+        const int r = r0 + half * nch;
+        const bool live = r < R;
         float acc[4] = {0.f, 0.f, 0.f, 0.f};
         float den = 0.f;
+        if (live) {
+          float2 ml[kPre];
+          float4 ov[kPre];
+#pragma unroll
+          for (int q = 0; q < kPre; ++q) {
+            const int cc = ws + q * kHalf;
+            ml[q] = make_float2(-INFINITY, 0.f);
+            ov[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (cc < nch) {
+              const size_t sidx = slot0 + (size_t)cc * p.attn_rpad + r;
+              ml[q] = __ldcg(reinterpret_cast<const float2*>(p.ml_part + sidx * 2));
+              if constexpr (D == 128) {
+                ov[q] = __ldcg(reinterpret_cast<const float4*>(p.o_part + sidx * D) + lane);
+              } else {
+                const float2 o2 = __ldcg(reinterpret_cast<const float2*>(p.o_part + sidx * D) + lane);
+                ov[q] = make_float4(o2.x, o2.y, 0.f, 0.f);
+              }
+            }
+          }
+          float mx = -INFINITY;
+          for (int cc = lane; cc < nch; cc += 32) mx = fmaxf(mx, __ldcg(p.ml_part + (slot0 + (size_t)cc * p.attn_rpad + r) * 2));
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+#pragma unroll
+          for (int q = 0; q < kPre; ++q) {   // chunks in ascending order, as below
+            const float w = ml[q].x == -INFINITY ? 0.f : exp2f(ml[q].x - mx);
+            den += w * ml[q].y;
+            acc[0] += w * ov[q].x; acc[1] += w * ov[q].y; acc[2] += w * ov[q].z; acc[3] += w * ov[q].w;
+          }
 #pragma unroll 1
-        for (int cc = warp; cc < nch; cc += NW) {
-          const size_t sidx = slot0 + (size_t)cc * p.attn_rpad + r;
-          const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.ml_part + sidx * 2));
-          const float w = ml.x == -INFINITY ? 0.f : exp2f(ml.x - mx);
-          den += w * ml.y;
-          if constexpr (D == 128) {
-            const float4 ov = __ldcg(reinterpret_cast<const float4*>(p.o_part + sidx * D) + lane);
-            acc[0] += w * ov.x; acc[1] += w * ov.y; acc[2] += w * ov.z; acc[3] += w * ov.w;
-          } else {
-            const float2 ov = __ldcg(reinterpret_cast<const float2*>(p.o_part + sidx * D) + lane);
-            acc[0] += w * ov.x; acc[1] += w * ov.y;
+          for (int cc = ws + kPre * kHalf; cc < nch; cc += kHalf) {   // long sequences: the chunks beyond the first kPre per warp
+            const size_t sidx = slot0 + (size_t)cc * p.attn_rpad + r;
+            const float2 m2 = __ldcg(reinterpret_cast<const float2*>(p.ml_part + sidx * 2));
+            const float w = m2.x == -INFINITY ? 0.f : exp2f(m2.x - mx);
+            den += w * m2.y;
+            if constexpr (D == 128) {
+              const float4 o4 = __ldcg(reinterpret_cast<const float4*>(p.o_part + sidx * D) + lane);
+              acc[0] += w * o4.x; acc[1] += w * o4.y; acc[2] += w * o4.z; acc[3] += w * o4.w;
+            } else {
+              const float2 o2 = __ldcg(reinterpret_cast<const float2*>(p.o_part + sidx * D) + lane);
+              acc[0] += w * o2.x; acc[1] += w * o2.y;
+            }
           }
         }
-        cbar();   // the previous row's sums have been read
+        cbar();   // the previous rows' sums have been read
         *reinterpret_cast<float4*>(part + warp * kPS + lane * 4) = make_float4(acc[0], acc[1], acc[2], acc[3]);
         if (lane == 0) part[warp * kPS + 128] = den;
         cbar();
-        if (warp == 0) {
+        if (ws == 0 && live) {
           float tot[4] = {0.f, 0.f, 0.f, 0.f};
           float dsum = 0.f;
 #pragma unroll
-          for (int w = 0; w < NW; ++w) {
-            const float4 v = *reinterpret_cast<const float4*>(part + w * kPS + lane * 4);
+          for (int w = 0; w < kHalf; ++w) {
+            const float4 v = *reinterpret_cast<const float4*>(part + (half * kHalf + w) * kPS + lane * 4);
             tot[0] += v.x; tot[1] += v.y; tot[2] += v.z; tot[3] += v.w;
-            dsum += part[w * kPS + 128];
+            dsum += part[(half * kHalf + w) * kPS + 128];
           }
           const float inv = 1.0f / dsum;
           const int i = r / G, hq = hk * G + (r % G);
