@@ -766,28 +766,35 @@ struct GemmPhase {
         const int pb_last = cb - (nst - 1) * kRowBytes;                   // bytes of a row's last piece
         // this lane's share of operand row g: the elements that meet the warp's weight bytes, stage by stage
         const unsigned char* xlane = x_s + xb * xbuf_bytes + g * xpitch + (warp * kWarpBytes + t * 16) * (2 / kElemBytes);
+        // Block rows behind MMA rows g and g + 8: rows g and g + 8 of the stage (rows past a tile stay inside
+        // the stage and feed accumulator rows that are never stored); only a gate/up tile with fewer than 8
+        // pairs keeps its up rows elsewhere (right behind its gate rows).  This lane's byte offsets in a
+        // stage of full pieces and in the stage of the rows' last pieces are the same for every such tile.
+        int oa_full[kSub], ob_full[kSub], oa_last[kSub], ob_last[kSub];
+        unsigned mask_last = 0;
+#pragma unroll
+        for (int u = 0; u < kSub; ++u) {
+          // a lane past the end of a short piece reads inside the stage (offset < 16 KB) but not its own data
+          const bool lane_valid = warp * kWarpBytes + u * 64 + t * 16 < pb_last;
+          mask_last |= (lane_valid ? 1u : 0u) << u;
+          oa_full[u] = block_offset(g, kRowBytes, warp, u, t);
+          ob_full[u] = block_offset(g + 8, kRowBytes, warp, u, t);
+          oa_last[u] = lane_valid ? block_offset(g, pb_last, warp, u, t) : 0;
+          ob_last[u] = lane_valid ? block_offset(g + 8, pb_last, warp, u, t) : 0;
+        }
 #pragma unroll 1
         for (int tile = 0; tile < gt; ++tile) {
-          // block rows behind MMA rows g and g + 8 (rows past the tile stay inside the stage and feed
-          // accumulator rows that are never stored)
-          const int ra = g;
-          const int rb = v.kind == kJobGateUp ? tile_units(v, tg * GT + tile) + g : g + 8;
+          if (v.kind == kJobGateUp && tile_units(v, tg * GT + tile) != 8) {   // the short last tile of a gate/up range
+            const int rb = tile_units(v, tg * GT + tile) + g;
+#pragma unroll
+            for (int u = 0; u < kSub; ++u) {
+              ob_full[u] = block_offset(rb, kRowBytes, warp, u, t);
+              ob_last[u] = ((mask_last >> u) & 1u) ? block_offset(rb, pb_last, warp, u, t) : 0;
+            }
+          }
           float ch[4][4];
 #pragma unroll
           for (int i = 0; i < 4; ++i) ch[i][0] = ch[i][1] = ch[i][2] = ch[i][3] = 0.f;
-          // this lane's byte offsets in a stage of full pieces and in the stage of the rows' last pieces
-          int oa_full[kSub], ob_full[kSub], oa_last[kSub], ob_last[kSub];
-          unsigned mask_last = 0;
-#pragma unroll
-          for (int u = 0; u < kSub; ++u) {
-            // a lane past the end of a short piece reads inside the stage (offset < 16 KB) but not its own data
-            const bool lane_valid = warp * kWarpBytes + u * 64 + t * 16 < pb_last;
-            mask_last |= (lane_valid ? 1u : 0u) << u;
-            oa_full[u] = block_offset(ra, kRowBytes, warp, u, t);
-            ob_full[u] = block_offset(rb, kRowBytes, warp, u, t);
-            oa_last[u] = lane_valid ? block_offset(ra, pb_last, warp, u, t) : 0;
-            ob_last[u] = lane_valid ? block_offset(rb, pb_last, warp, u, t) : 0;
-          }
 #pragma unroll 1
           for (int st = 0; st < nst; ++st) {   // rolled: the stage's code stays in the instruction cache
             const bool last = st == nst - 1;
