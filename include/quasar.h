@@ -195,8 +195,9 @@ int quasar_workspace_bytes(const quasar_model* m, int32_t B, int32_t T_max, size
  * block_len  int32 [B], 1 <= block_len[b] <= T_max <= QUASAR_MAX_BLOCK; rows
  *            beyond it are ignored (1 = one plain decode step).
  * logits_out fp32 [B][T_max][V] or NULL.  Row i predicts the token after row i.
- * accept_len int32 [B]: number of accepted DRAFT tokens, in [0, block_len-1].
- * bonus      int32 [B]: the verifier's token after the last accepted row.
+ * accept_len int32 [B]: number of accepted DRAFT tokens, in [0, block_len-1]; -1 for a
+ *            sequence that was skipped because of a device-detected error (see status).
+ * bonus      int32 [B]: the verifier's token after the last accepted row (-1 if skipped).
  * accept_path int32 [B][T_max] or NULL: accept_path[b][d] = block row accepted at
  *            depth d (entry 0 is the root, entries past accept_len are -1).
  * status     int32 [1]: left untouched on success, else a negative code.
@@ -215,6 +216,8 @@ int quasar_verify(quasar_model* m, const quasar_kv* kv /* host struct */, const 
  * iterations).  Chain (accept_path NULL): seq_len[b] += 1 + accept_len[b].
  * Tree: K,V of the accepted row at depth d move to slot seq_len[b] + d for
  * d = 1..accept_len[b], then the same bump.  The only call that changes seq_len.
+ * A sequence whose accept_len is negative (skipped by quasar_verify) is left untouched:
+ * its K/V rows were never written, so committing them would publish garbage.
  * ---------------------------------------------------------------------- */
 int quasar_kv_commit(quasar_model* m, const quasar_kv* kv /* host struct */, const int32_t* accept_len,
                      const int32_t* accept_path, int32_t B, int32_t T_max, void* stream);

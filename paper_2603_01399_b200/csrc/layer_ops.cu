@@ -215,8 +215,8 @@ __global__ void accept_kernel(const int32_t* __restrict__ tokens, const int32_t*
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b >= B) return;
   const int base = b * T_max;
-  if (!bi.valid[b]) {
-    accept_len[b] = 0;
+  if (!bi.valid[b]) {   // a skipped sequence: -1 tells quasar_kv_commit to leave its cache and seq_len alone
+    accept_len[b] = -1;
     bonus[b] = -1;
     if (accept_path) for (int d = 0; d < T_max; ++d) accept_path[base + d] = -1;
     return;

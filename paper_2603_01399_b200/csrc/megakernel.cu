@@ -167,59 +167,6 @@ __device__ __forceinline__ unsigned long long now_ns() {
   return t;
 }
 
-#ifdef QUASAR_TIMELINE
-__device__ long long g_timeline[160][256];
-#ifndef QUASAR_TL_KIND
-#define QUASAR_TL_KIND 4
-#endif
-__device__ long long g_timeline2[160][16][40];
-__device__ long long g_timeline3[160][64];   // producer: clock at the issue of each stage of the watched phase
-#define TL2_MARK() do { if (tl_on && lane == 0 && tl2_n[warp] < 40) s_tl2[warp][tl2_n[warp]++] = clock64(); } while (0)
-#define TL_DECL __shared__ long long s_tl[256]; int tl_n = 0;
-#define TL_MARK() do { if (threadIdx.x == 0 && tl_on && tl_n < 256) s_tl[tl_n++] = clock64(); } while (0)
-#define TL_FLUSH() do { if (threadIdx.x == 0 && tl_on) { for (int i__ = 0; i__ < tl_n; ++i__) g_timeline[blockIdx.x][i__] = s_tl[i__]; g_timeline[blockIdx.x][255] = tl_n; } } while (0)
-#else
-#define TL_DECL
-#define TL2_MARK() do { } while (0)
-#define TL_MARK() do { } while (0)
-#define TL_FLUSH() do { } while (0)
-#endif
-#ifdef QUASAR_PHASE_TIMER
-// Diagnostic build only: thread 0 of every CTA stamps the SM clock at each phase boundary.
-constexpr int kMaxMarks = 640;
-__device__ long long g_phase_clk[160][kMaxMarks];
-__device__ int g_phase_n[160];
-__device__ long long g_gemm_clk[160][8];
-__device__ int g_clk_on_dummy;
-#ifndef QUASAR_TIMER_KIND
-#define QUASAR_TIMER_KIND 4
-#endif
-#define g_clk_on (jb.kind == QUASAR_TIMER_KIND)
-__device__ long long g_attn_clk[160][8];
-__device__ long long g_attn_tmp_unused;
-#define ATTN_T(i) do { if (threadIdx.x == 0) { const long long c__ = clock64(); s_attn_clk[i] += c__ - at0; at0 = c__; } } while (0)
-#define PHASE_MARK()                                                                         \
-  do {                                                                                       \
-    if (threadIdx.x == 0 && mark_n < kMaxMarks) g_phase_clk[blockIdx.x][mark_n++] = clock64(); \
-  } while (0)
-#ifdef QUASAR_GEMM_TIMER
-#define STAGE_CLK(i) do { const long long n__ = clock64(); tacc[i] += (unsigned)(n__ - stage_prev); stage_prev = n__; } while (0)
-#define GEMM_CLK(i, expr)                                           \
-  do {                                                              \
-    const long long c0__ = clock64();                               \
-    expr;                                                           \
-    tacc[i] += (unsigned)(clock64() - c0__);                          \
-  } while (0)
-#else
-#define GEMM_CLK(i, expr) do { expr; } while (0)
-#define STAGE_CLK(i) do { } while (0)
-#endif
-#else
-#define ATTN_T(i) do { } while (0)
-#define PHASE_MARK() do { } while (0)
-#define GEMM_CLK(i, expr) do { expr; } while (0)
-#define STAGE_CLK(i) do { } while (0)
-#endif
 
 // ---- mbarriers ----------------------------------------------------------------------------
 __device__ __forceinline__ void mbar_init(uint64_t* bar, int count) {
@@ -356,9 +303,6 @@ __device__ void producer_loop(const MegaParams& p, const Pipe& pipe, int cta, in
   uint32_t phase = 0;
   long long issued = 0;
   bool ok = true;
-#ifdef QUASAR_TIMELINE
-  int tl3_n = 0;
-#endif
   for (int job = 0; job < p.n_jobs && ok; ++job) {
     const JobView v = job_view<W_INT8>(p.jobs, job, cta, ncta);
     const unsigned char* src = v.wp;
@@ -373,9 +317,6 @@ __device__ void producer_loop(const MegaParams& p, const Pipe& pipe, int cta, in
           for (int b0 = 0; b0 < cb; b0 += kRowBytes) {
             const uint32_t bytes = (uint32_t)(rows * min(kRowBytes, cb - b0));
             if (!mbar_wait(pipe.empty + slot, phase ^ 1u, pipe.abort_flag, pipe.status)) { ok = false; break; }
-#ifdef QUASAR_TIMELINE
-            if (p.jobs[job].kind == QUASAR_TL_KIND && job >= p.n_jobs - 5 && tl3_n < 64) g_timeline3[blockIdx.x][tl3_n++] = clock64();
-#endif
             mbar_arrive_expect_tx(pipe.full + slot, bytes);
             bulk_copy(pipe.ring + slot * kStageBytes, src, bytes, pipe.full + slot, policy);
             src += bytes;
@@ -586,10 +527,6 @@ struct GemmPhase {
                                              uint32_t& xphase, int cta, int ncta, GridSync& gs) {
     int slot = slot_io;
     uint32_t phase = phase_io;
-#ifdef QUASAR_GEMM_TIMER
-    unsigned tacc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-    long long stage_prev = clock64();
-#endif
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
     // The phase's descriptor was fetched into shared memory during the phase before (a load from global
     // memory here would be the first thing every warp waits for); thread 0 now fetches the next one into
@@ -616,17 +553,6 @@ struct GemmPhase {
     // behind (each warp adds its share of the CTAs, the shares meet in shared memory: a fixed order);
     // the fp16 scale is the job's static one (|h| <= sqrt(K) * max|gain|).  Other GEMMs with int8
     // weights: a power-of-two scale from the row maximum gathered while the operand was written.
-    TL_DECL
-#ifdef QUASAR_TIMELINE
-    __shared__ long long s_tl2[16][40];
-    __shared__ int tl2_n[16];
-    if (threadIdx.x < 16) { tl2_n[threadIdx.x] = 0; for (int i = 0; i < 40; ++i) s_tl2[threadIdx.x][i] = 0; }
-    cbar();
-#endif
-#ifdef QUASAR_TIMELINE
-    const bool tl_on = jb.kind == QUASAR_TL_KIND && job >= p.n_jobs - 5;
-#endif
-    TL_MARK();
     bool have_x = false, first = true;
     bool requested = false;   // the next chunk's copy is already in flight
     int xb = 0;               // operand buffer in use (a long contraction alternates between two)
@@ -672,18 +598,13 @@ struct GemmPhase {
 
       // Accumulators live for one tile and one chunk; each warp then parks them in its own part of
       // `red` (summing over the chunks of a long contraction), where the epilogue adds the warps up.
-#ifdef QUASAR_GEMM_TIMER
-      const long long c_t0 = clock64();
-#endif
       for (int kc = 0; kc < v.nchunks; ++kc) {
         if (!have_x) {
-          TL_MARK();
           // every warp is past its last use of the buffer's other tenants (epilogue / attention end in a CTA barrier)
           if (warp == 0 && !requested)
             request_operand<W_INT8>(x_s + xb * xbuf_bytes, direct ? xsrc16 : xsrc, ld, M, v.chunk, kc * v.chunk,
                                     min(v.chunk, jb.K - kc * v.chunk), jb.gain, xbar, lane);
           requested = false;
-          TL_MARK();
           bool again = false;   // the fp16 copy was asked for, but a row needs a scale
           if (first) {   // the row factors ride on the same round trip as the first chunk's loads
             first = false;
@@ -696,9 +617,7 @@ struct GemmPhase {
               ss += __shfl_xor_sync(0xffffffffu, ss, 1);
               ss += __shfl_xor_sync(0xffffffffu, ss, 2);
               if (t == 0) misc[kMiscRowSum + warp * 8 + g] = ss;
-              TL_MARK();
               cbar();
-              TL_MARK();
               float tot = 0.f;
 #pragma unroll
               for (int w = 0; w < NW; ++w) tot += misc[kMiscRowSum + w * 8 + g];
@@ -733,7 +652,6 @@ struct GemmPhase {
             if (!got) return false;
             xphase ^= 1u;
           }
-          TL_MARK();
           if (again) {   // rare: fetch the chunk once more, from the bf16 tensor
             cbar();      // every warp has seen the first copy land
             if (warp == 0)
@@ -750,7 +668,6 @@ struct GemmPhase {
             convert_staged<W_INT8>(x_s + xb * xbuf_bytes, M, v.chunk, min(v.chunk, jb.K - kc * v.chunk), normed, misc + kMiscRs);
           }
           cbar();   // the chunk is ready; every warp is past the tiles of the chunk before it
-          TL_MARK();
           if (v.nchunks > 1 && (kc + 1 < v.nchunks || tg + 1 < v.ngroups)) {
             // a long contraction reloads its chunks for every tile group: the next one lands in the
             // other buffer while this one is multiplied
@@ -806,17 +723,11 @@ struct GemmPhase {
             }
             const unsigned valid_mask = last ? mask_last : (1u << kSub) - 1u;
             // every lane tests the stage's barrier itself (one instruction per warp, no broadcast afterwards)
-            STAGE_CLK(0);
             if (!__all_sync(0xffffffffu, mbar_wait(pipe.full + slot, phase, pipe.abort_flag, pipe.status))) return false;   // the warp leaves together
-            STAGE_CLK(1);
-            TL2_MARK();
             consume_stage<W_INT8>(pipe.ring + slot * kStageBytes, xlane + st * (kRowBytes * 2 / kElemBytes), oa, ob, valid_mask, ch);
             __syncwarp();
-            STAGE_CLK(2);
-            TL2_MARK();
             if (lane == 0) mbar_arrive(pipe.empty + slot);
             if (++slot == kStages) { slot = 0; phase ^= 1u; }
-            STAGE_CLK(3);
           }
           float* r = red + ((warp * GT + tile) * 16) * 8;
           float2 lo = make_float2((ch[0][0] + ch[1][0]) + (ch[2][0] + ch[3][0]), (ch[0][1] + ch[1][1]) + (ch[2][1] + ch[3][1]));
@@ -833,10 +744,6 @@ struct GemmPhase {
         if (v.nchunks > 1) xb ^= 1;   // the next chunk is (or will be) in the other buffer
         else have_x = true;           // a short contraction keeps its operand for every tile group
       }
-#ifdef QUASAR_GEMM_TIMER
-      tacc[5] += (unsigned)(clock64() - c_t0);
-#endif
-      TL_MARK();
       // ---- cross-warp reduction in a fixed order, then the fused epilogue ----
       cbar();
 #pragma unroll 1
@@ -850,24 +757,12 @@ struct GemmPhase {
         epilogue(p, jb, v, job, ei, e0, e1, er, best, best_i, red, misc);
       }
       cbar();
-      TL_MARK();
       if (residual && threadIdx.x < 8) {   // fixed order: tiles of the group, groups of the phase
         for (int tile = 0; tile < gt; ++tile) ss_run += misc[kMiscPart + tile * 8 + threadIdx.x];
       }
     }
     if (residual && threadIdx.x < 8) p.ss_part[cta * 8 + threadIdx.x] = ss_run;
     if (jb.kind == kJobLm) finish_argmax(best, best_i, misc);
-    TL_MARK();
-    TL_FLUSH();
-#ifdef QUASAR_TIMELINE
-    cbar();
-    if (tl_on && threadIdx.x < 16) for (int i = 0; i < 40; ++i) g_timeline2[blockIdx.x][threadIdx.x][i] = s_tl2[threadIdx.x][i];
-#endif
-#ifdef QUASAR_GEMM_TIMER
-    if (threadIdx.x == 0 && g_clk_on) {
-      for (int i = 0; i < 8; ++i) g_gemm_clk[blockIdx.x][i] += tacc[i];
-    }
-#endif
     slot_io = slot;
     phase_io = phase;
     return true;
@@ -1121,12 +1016,6 @@ __device__ __noinline__ void attention_phase(const MegaParams& p, int layer, boo
   __nv_bfloat16* vc_l = p.v_cache + (size_t)layer * layer_stride;
   const int n_items = p.B * p.Hkv * p.attn_nchunk;
   int* last_flag = reinterpret_cast<int*>(misc + kMiscFlag);
-#ifdef QUASAR_PHASE_TIMER
-  __shared__ long long s_attn_clk[8];
-  if (threadIdx.x < 8) s_attn_clk[threadIdx.x] = 0;
-  cbar();
-  long long at0 = clock64();
-#endif
 
   // rows that take no part (beyond a block's length, or of a skipped sequence) give zero attention output
   for (int m = cta; m < p.M; m += ncta) {
@@ -1234,8 +1123,6 @@ __device__ __noinline__ void attention_phase(const MegaParams& p, int layer, boo
       }
     }
     cbar();  // block-level visibility of the K/V rows just stored and of q_s
-    ATTN_T(0);
-
     // (b) stage the K / V tile (zero beyond the end of the sequence); cached rows of a prefetched
     //     tile are already on their way
     const int first_row = prefetched ? max(0, min(kKeyTile, P - key_begin)) : 0;
@@ -1251,8 +1138,6 @@ __device__ __noinline__ void attention_phase(const MegaParams& p, int layer, boo
     }
     asm volatile("cp.async.wait_all;\n" ::: "memory");
     cbar();
-    ATTN_T(1);
-
     // (c) one warp per 16 query rows
     const int row_tiles = (R + 15) / 16;
     if (warp < row_tiles) {
@@ -1370,7 +1255,6 @@ __device__ __noinline__ void attention_phase(const MegaParams& p, int layer, boo
     const int nch = (Lk + kKeyTile - 1) / kKeyTile;
     const size_t slot0 = ((size_t)b * p.Hkv + hk) * p.attn_nchunk * p.attn_rpad;
     unsigned* arrivals = p.attn_count + (size_t)layer * p.B * p.Hkv + b * p.Hkv + hk;
-    ATTN_T(2);
     cbar();   // o_s and ml_s are complete
     if (threadIdx.x == 0) {
       const size_t slot = slot0 + (size_t)c * p.attn_rpad;
@@ -1399,7 +1283,6 @@ __device__ __noinline__ void attention_phase(const MegaParams& p, int layer, boo
       *last_flag = ok_flag;
     }
     cbar();
-    ATTN_T(3);
     if (*last_flag) {
       // Two rows at a time, half of the warps each: warp ws of a half adds the chunks ws, ws + NW/2, ...
       // of its row (lane l: four output dimensions); the warps' sums meet in shared memory in warp order.
@@ -1495,10 +1378,6 @@ __device__ __noinline__ void attention_phase(const MegaParams& p, int layer, boo
       }
     }
   }
-  ATTN_T(4);
-#ifdef QUASAR_PHASE_TIMER
-  if (threadIdx.x == 0) for (int i = 0; i < 8; ++i) g_attn_clk[blockIdx.x][i] += s_attn_clk[i];
-#endif
   asm volatile("cp.async.wait_all;\n" ::: "memory");   // a prefetch whose item was skipped has landed before the tiles are reused
 }
 
@@ -1524,8 +1403,8 @@ __device__ void accept_phase(const MegaParams& p, int ncta) {
   cbar();
   if ((int)threadIdx.x < p.B) {
     const int b = threadIdx.x, base = b * p.T_max;
-    if (!p.bi.valid[b]) {
-      p.accept_len[b] = 0;
+    if (!p.bi.valid[b]) {   // a skipped sequence: -1 tells quasar_kv_commit to leave its cache and seq_len alone
+      p.accept_len[b] = -1;
       p.bonus[b] = -1;
       if (p.accept_path) for (int d = 0; d < p.T_max; ++d) p.accept_path[base + d] = -1;
     } else {
@@ -1593,30 +1472,19 @@ __global__ void __launch_bounds__(kThreads, 1) verify_megakernel(const MegaParam
   uint32_t phase = 0, xphase = 0, xphase2 = 0;
   GridSync gs{p.barrier, p.status, (unsigned)ncta, 0u, abort_flag};
   bool ok = true;
-#ifdef QUASAR_PHASE_TIMER
-  int mark_n = 0;
-#endif
-
-  PHASE_MARK();
   prep_phase(p, misc, cta, ncta);
-  PHASE_MARK();
   gs.arrive();
-  PHASE_MARK();
   // the GEMMs of the pass in order (qkv, o, gate+up, down per layer, then the LM head); attention follows every qkv
   for (int job = 0; job < p.n_jobs && ok; ++job) {
     // (every GEMM phase waits, inside, for the grid barrier that the phase before it arrived at)
     if (!(ok = GemmPhase<W_INT8>::run(p, job, pipe, slot, phase, red, misc, x_s, xbar, xphase, cta, ncta, gs))) break;
-    PHASE_MARK();
     if (job == p.n_jobs - 1) break;   // the LM head is followed by the candidate exchange below
     gs.arrive();
-    PHASE_MARK();
     if ((job & 3) == 0) {
       attention_prefetch<D>(p, job >> 2, k_s, v_s, cta);   // reads the cached prefix only: nothing of this phase
       if (!(ok = gs.wait())) break;
       attention_phase<D>(p, job >> 2, W_INT8, k_s, v_s, q_s, misc, xbar, xphase, xphase2, cta, ncta);
-      PHASE_MARK();
       gs.arrive();
-      PHASE_MARK();
     }
   }
   if (ok) {
@@ -1626,12 +1494,8 @@ __global__ void __launch_bounds__(kThreads, 1) verify_megakernel(const MegaParam
       p.cand_idx[(size_t)cta * 8 + threadIdx.x] = reinterpret_cast<int*>(misc + kMiscRunI)[threadIdx.x];
     }
     ok = gs.sync();
-    PHASE_MARK();
     if (ok && cta == 0) accept_phase(p, ncta);
   }
-#ifdef QUASAR_PHASE_TIMER
-  if (threadIdx.x == 0) g_phase_n[blockIdx.x] = mark_n;
-#endif
   if (!ok && threadIdx.x == 0) {
     *abort_flag = 1;  // tells the producer to stop issuing
     // an operand chunk may have been requested and never waited for: let it land (it takes a few
@@ -1700,39 +1564,6 @@ int launch_variant(const MegaParams& p, int ncta, cudaStream_t stream) {
 
 }  // namespace
 
-#ifdef QUASAR_PHASE_TIMER
-extern "C" int quasar_debug_phase_marks(long long* clk_host, int* n_host) {
-  if (cudaMemcpyFromSymbol(clk_host, g_phase_clk, sizeof(long long) * 160 * kMaxMarks) != cudaSuccess) return -1;
-  if (cudaMemcpyFromSymbol(n_host, g_phase_n, sizeof(int) * 160) != cudaSuccess) return -1;
-  return kMaxMarks;
-}
-#ifdef QUASAR_TIMELINE
-extern "C" int quasar_debug_timeline3(long long* host) {
-  if (cudaMemcpyFromSymbol(host, g_timeline3, sizeof(long long) * 160 * 64) != cudaSuccess) return -1;
-  return 0;
-}
-extern "C" int quasar_debug_timeline2(long long* host) {
-  if (cudaMemcpyFromSymbol(host, g_timeline2, sizeof(long long) * 160 * 16 * 40) != cudaSuccess) return -1;
-  return 0;
-}
-extern "C" int quasar_debug_timeline(long long* host) {
-  if (cudaMemcpyFromSymbol(host, g_timeline, sizeof(long long) * 160 * 256) != cudaSuccess) return -1;
-  return 0;
-}
-#endif
-extern "C" int quasar_debug_attn_clocks(long long* host) {
-  if (cudaMemcpyFromSymbol(host, g_attn_clk, sizeof(long long) * 160 * 8) != cudaSuccess) return -1;
-  return 0;
-}
-extern "C" int quasar_debug_gemm_clocks(long long* host, int reset) {
-  if (cudaMemcpyFromSymbol(host, g_gemm_clk, sizeof(long long) * 160 * 8) != cudaSuccess) return -1;
-  if (reset) {
-    static long long zero[160 * 8];
-    if (cudaMemcpyToSymbol(g_gemm_clk, zero, sizeof(zero)) != cudaSuccess) return -1;
-  }
-  return 0;
-}
-#endif
 
 int launch_repack(const void* w, void* wp, int N, int K, int kind, int weight_dtype, int ncta, cudaStream_t stream) {
   const int units = kind == kJobGateUp ? N / 2 : N;

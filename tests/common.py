@@ -69,3 +69,24 @@ def margins(logits):
     """top1 - top2 per row of fp32 logits [..., V]."""
     part = np.partition(logits, -2, axis=-1)
     return part[..., -1] - part[..., -2]
+
+
+# ---- agreement at the benchmark's full widths -------------------------------------------------
+# Every tensor of the pass is rounded to bf16 between steps, so two implementations that only ADD
+# differently (fp32 instead of fp64, another summation order) drift apart through flipped roundings.
+# tests/test_oracle_fullwidth_noise.py measures that drift with the oracle against itself on the CPU
+# (two layers at the Qwen3-8B widths, fp32 accumulation in eight interleaved slices): 98.7 % of the
+# logits inside max(2e-2, 1e-2 |o|), mean |d| 4.3e-3, worst 4.0e-2 at a logit spread of 1.33.  The
+# full-width GPU tests assert the benchmark's element test on a share of the logits that leaves twice
+# that many outside, and bound the mean and the worst element at 2.5 to 3 times that measured drift.
+FULLWIDTH_SHARE = 0.97
+FULLWIDTH_MEAN_TOL = 1.2e-2
+FULLWIDTH_WORST_TOL = 1e-1
+
+
+def fullwidth_stats(got, want):
+    """(share of elements with |g - o| <= max(2e-2, 1e-2 |o|), mean |g - o|, worst |g - o|)."""
+    got = np.asarray(got, np.float64)
+    want = np.asarray(want, np.float64)
+    d = np.abs(got - want)
+    return float(np.mean(d <= np.maximum(2e-2, 1e-2 * np.abs(want)))), float(d.mean()), float(d.max())

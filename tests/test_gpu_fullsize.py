@@ -27,7 +27,8 @@ import torch
 import oracle
 from oracle import quasar_oracle as qo
 from paper_2603_01399_b200 import binding, synth
-from tests.common import logits_close, margins, master_getter
+from tests.common import (FULLWIDTH_MEAN_TOL, FULLWIDTH_SHARE, FULLWIDTH_WORST_TOL, fullwidth_stats, logits_close, margins,
+                          master_getter)
 
 pytestmark = pytest.mark.gpu
 
@@ -72,15 +73,14 @@ def _run(gm, kv, tokens, parents, block_len, path, trace=False):
     return buf, (binding.split_trace(gm, tr, B, T) if trace else None)
 
 
-# What end-to-end agreement means at these widths (see the module docstring): the benchmark's element
-# test on at least 97 % of the logits, mean |d| <= 1.2e-2, worst |d| <= 1e-1.
-def _assert_statistically_close(got, want, what, share=0.97, mean_tol=1.2e-2, worst_tol=1e-1):
-    got = np.asarray(got, np.float64)
-    want = np.asarray(want, np.float64)
-    d = np.abs(got - want)
-    inside = float(np.mean(d <= np.maximum(2e-2, 1e-2 * np.abs(want))))
-    assert inside >= share and d.mean() <= mean_tol and d.max() <= worst_tol, \
-        f"{what}: {inside:.4f} of the logits inside max(2e-2, 1e-2|o|), mean |d| {d.mean():.3e}, worst {d.max():.3e}"
+# What end-to-end agreement means at these widths: the criterion that the oracle's drift from itself
+# under another accumulation fixes (tests/common.py, measured on the CPU by
+# tests/test_oracle_fullwidth_noise.py), not a comparison of GPU code with GPU code.
+def _assert_statistically_close(got, want, what, share=FULLWIDTH_SHARE, mean_tol=FULLWIDTH_MEAN_TOL,
+                                worst_tol=FULLWIDTH_WORST_TOL):
+    inside, mean, worst = fullwidth_stats(got, want)
+    assert inside >= share and mean <= mean_tol and worst <= worst_tol, \
+        f"{what}: {inside:.4f} of the logits inside max(2e-2, 1e-2|o|), mean |d| {mean:.3e}, worst {worst:.3e}"
 
 
 CLEAR_MARGIN = 0.25      # top-2 margin beyond which the rounding noise above cannot change the arg-max

@@ -206,6 +206,36 @@ def test_device_side_errors_set_status_and_skip(world):
     assert torch.equal(kv.k.cpu(), torch.from_numpy(full.k_bits.view(np.int16)).view(torch.bfloat16))
 
 
+@pytest.mark.parametrize("path", [1, 2])
+def test_commit_leaves_a_skipped_sequence_alone(world, path):
+    """Batch of two, the second sequence carries a token outside the vocabulary: it is skipped
+    (accept_len = bonus = -1), and a commit afterwards changes neither its seq_len nor its cache,
+    while the good sequence is committed as usual."""
+    shape, om, gm, okv1, root = world
+    okv = oracle.new_kv(om, 2, S_MAX)
+    for b in range(2):
+        okv.k_bits[:, b] = okv1.k_bits[:, 0]
+        okv.v_bits[:, b] = okv1.v_bits[:, 0]
+        okv.seq_len[b] = okv1.seq_len[0]
+    tokens = np.array([[root, 1, 2, 3], [root, 1, shape.vocab + 5, 3]], np.int32)
+    bl = np.array([4, 4], np.int32)
+    kv, buf, _ = _run_gpu(shape, gm, okv, tokens, None, bl, path=path)
+    assert int(buf.status[0]) == -7
+    assert int(buf.accept_len[1]) == -1 and int(buf.bonus[1]) == -1
+    assert 0 <= int(buf.accept_len[0]) <= 3 and 0 <= int(buf.bonus[0]) < shape.vocab
+    k_before, v_before = kv.k[:, 1].clone(), kv.v[:, 1].clone()
+    binding.quasar_kv_commit(gm, kv, buf)
+    torch.cuda.synchronize()
+    sl = kv.seq_len.cpu().numpy()
+    assert sl[1] == okv.seq_len[1], "a skipped sequence was committed"
+    assert sl[0] == okv.seq_len[0] + 1 + int(buf.accept_len[0])
+    assert torch.equal(kv.k[:, 1], k_before) and torch.equal(kv.v[:, 1], v_before)
+    # the good sequence of the batch is what the oracle computes for it alone
+    r = oracle.verify(om, _copy(okv), tokens[:1], None, bl[:1])
+    ok, mabs, _ = logits_close(buf.logits[0].cpu().numpy(), r.logits[0])
+    assert ok, mabs
+
+
 def test_host_side_errors(world):
     shape, om, gm, okv, root = world
     kv = _kv_to_gpu(shape, okv, 1)
