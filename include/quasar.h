@@ -22,9 +22,11 @@
  *    the caller, 16-byte aligned, valid until the work queued by the call has
  *    finished.  The library allocates no device memory per call; scratch comes
  *    from a caller-provided workspace (quasar_workspace_bytes).
- *  - `stream` is a cudaStream_t passed as void*.  Calls only enqueue work
- *    (no synchronisation, no allocation), so they may be stream-captured;
- *    results are valid once the stream has been synchronised.
+ *  - `stream` is a cudaStream_t passed as void*.  Unless a call says otherwise it only
+ *    enqueues work (no synchronisation, no allocation); results are valid once the
+ *    stream has been synchronised.  quasar_plan_create is the supported way to freeze a
+ *    pass for replay: it captures the kernel-per-step form into a CUDA graph itself and
+ *    keeps the persistent single-kernel form (a cooperative launch) as a plain launch.
  *  - Argument errors that the host can see are reported before anything is
  *    launched.  Errors only the device can see (a token id out of range, a
  *    malformed parent array, a sequence that would overflow its cache) set the
@@ -264,6 +266,14 @@ int quasar_set_trace(quasar_model* m, void* trace_buf, size_t bytes);
  * per step, 2 = require the persistent kernel (QUASAR_ERR_SHAPE if the call does not fit it).
  * Both compute the same pass (Section 3.1, 3.3); they differ in summation order only. */
 int quasar_set_path(quasar_model* m, int32_t path);
+
+/* Every wait inside the persistent kernel (grid barrier, stage barrier, attention arrival
+ * count) is bounded: after budget_ns (default 2e9) the waiting thread block sets `status` to
+ * QUASAR_ERR_TIMEOUT, tells its other warps to stop waiting and returns once its own copies
+ * in flight have landed; nothing traps and the context stays usable.  test_extra_arrivals is
+ * for tests of that path only and must be 0 otherwise: the grid barrier then expects that many
+ * arrivals more than there are thread blocks, so its first wait cannot complete and runs out. */
+int quasar_set_wait_budget(quasar_model* m, uint64_t budget_ns, int32_t test_extra_arrivals);
 
 /* Count of kernels the library has launched in this process (all calls). */
 int64_t quasar_kernel_launches(void);

@@ -76,6 +76,7 @@ SIGNATURES = {
     "quasar_trace_bytes": (C.c_int, [_vp, _i32, _i32, C.POINTER(_sz)]),
     "quasar_set_trace": (C.c_int, [_vp, _vp, _sz]),
     "quasar_set_path": (C.c_int, [_vp, _i32]),
+    "quasar_set_wait_budget": (C.c_int, [_vp, C.c_uint64, _i32]),
 }
 
 
@@ -237,6 +238,10 @@ class Model:
     def set_path(self, path: int) -> None:
         """0 automatic, 1 one kernel per step, 2 persistent single-kernel pass."""
         _check(lib().quasar_set_path(self.handle, path))
+
+    def set_wait_budget(self, budget_ns: int, test_extra_arrivals: int = 0) -> None:
+        """Bound of every device-side wait of the persistent kernel (default 2 s)."""
+        _check(lib().quasar_set_wait_budget(self.handle, budget_ns, test_extra_arrivals))
 
     def weight_bytes(self) -> int:
         return sum(v.numel() * v.element_size() for k, v in self.tensors.items()

@@ -43,6 +43,8 @@ struct quasar_model {
   unsigned char* mega_weights = nullptr;  // device: every matrix again, permuted for the persistent kernel
   int mega_ncta = 0;                // 0: not available on this device
   int path = 0;                     // 0 auto, 1 one kernel per step, 2 persistent kernel
+  unsigned long long wait_budget_ns = 2000000000ull;   // bound of every device-side wait of the persistent kernel
+  unsigned barrier_extra = 0;       // test of the failure path only (quasar_set_wait_budget)
 };
 
 struct quasar_plan {
@@ -265,6 +267,7 @@ int verify_impl(quasar_model* m, const quasar_kv* kv, const int32_t* tokens, con
     p.attn_count = reinterpret_cast<unsigned*>(wsp + ws.attn_count);
     p.barrier = reinterpret_cast<unsigned*>(wsp + ws.barrier);
     p.accept_len = accept_len; p.bonus = bonus; p.accept_path = accept_path; p.status = status;
+    p.wait_budget_ns = m->wait_budget_ns; p.barrier_extra = m->barrier_extra;
     QUASAR_CUDA_CHECK(cudaMemsetAsync(p.barrier, 0, 256, stream));
     return launch_verify_mega(p, wd, D, m->mega_ncta, stream);
   }
@@ -508,6 +511,16 @@ int quasar_model_create(const quasar_config* cfg, const quasar_weights* w, quasa
 int quasar_set_path(quasar_model* m, int32_t path) {
   if (m == nullptr || path < 0 || path > 2) { set_error("set_path: bad argument"); return QUASAR_ERR_INVALID_ARG; }
   m->path = path;
+  return QUASAR_OK;
+}
+
+int quasar_set_wait_budget(quasar_model* m, uint64_t budget_ns, int32_t test_extra_arrivals) {
+  if (m == nullptr || budget_ns == 0 || test_extra_arrivals < 0 || test_extra_arrivals > 1024) {
+    set_error("set_wait_budget: bad argument");
+    return QUASAR_ERR_INVALID_ARG;
+  }
+  m->wait_budget_ns = budget_ns;
+  m->barrier_extra = (unsigned)test_extra_arrivals;
   return QUASAR_OK;
 }
 

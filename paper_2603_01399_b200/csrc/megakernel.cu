@@ -59,7 +59,6 @@ constexpr int GT = 4;                      // 16-row tiles accumulated together 
 constexpr int kKeyTile = 64;
 constexpr int kMaxRowsAttn = 32;           // query rows (heads-in-group x block rows) per kv head
 constexpr float kLog2e = 1.4426950408889634f;
-constexpr unsigned long long kWaitBudgetNs = 2000000000ull;  // every device-side wait gives up after 2 s
 
 // ---- shared memory map --------------------------------------------------------------------
 constexpr int kRingBytes = kStages * kStageBytes;                        // 131072
@@ -191,7 +190,11 @@ __device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
   return ok != 0;
 }
 // Waits for the phase of `bar` with the given parity.  Gives up when another thread of the CTA
-// has raised the abort flag or after kWaitBudgetNs (then raises the flag and the status itself).
+// has raised the abort flag or after the launch's wait budget (then raises the flag and the status itself).
+// The budget sits in shared memory two words behind the abort flag.
+__device__ __forceinline__ unsigned long long wait_budget(volatile int* abort_flag) {
+  return *reinterpret_cast<volatile unsigned long long*>(abort_flag + 2);
+}
 __device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
   const unsigned long long t0 = now_ns();
   unsigned it = 0;
@@ -199,7 +202,7 @@ __device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, vola
     if (mbar_try(bar, parity)) return true;
     if ((++it & 63u) == 0) {
       if (*abort_flag) return false;
-      if (now_ns() - t0 > kWaitBudgetNs) {
+      if (now_ns() - t0 > wait_budget(abort_flag)) {
         atomicMin(status, QUASAR_ERR_TIMEOUT);
         *abort_flag = 1;
         return false;
@@ -334,7 +337,7 @@ __device__ void producer_loop(const MegaParams& p, const Pipe& pipe, int cta, in
     if (--slot < 0) { slot = kStages - 1; phase ^= 1u; }
     const unsigned long long t0 = now_ns();
     while (!mbar_try(pipe.full + slot, phase)) {
-      if (now_ns() - t0 > kWaitBudgetNs) { atomicMin(pipe.status, QUASAR_ERR_TIMEOUT); break; }
+      if (now_ns() - t0 > wait_budget(pipe.abort_flag)) { atomicMin(pipe.status, QUASAR_ERR_TIMEOUT); break; }
     }
   }
 }
@@ -367,7 +370,7 @@ struct GridSync {
         unsigned v;
         asm volatile("ld.acquire.gpu.global.u32 %0, [%1];\n" : "=r"(v) : "l"(counter) : "memory");
         if (v >= target) break;
-        if ((++polls & 255u) == 0 && (*abort_flag || now_ns() - t0 > kWaitBudgetNs)) {
+        if ((++polls & 255u) == 0 && (*abort_flag || now_ns() - t0 > wait_budget(abort_flag))) {
           atomicMin(status, QUASAR_ERR_TIMEOUT);
           *abort_flag = 1;
           break;
@@ -1272,7 +1275,7 @@ __device__ __noinline__ void attention_phase(const MegaParams& p, int layer, boo
           unsigned v;
           asm volatile("ld.acquire.gpu.global.u32 %0, [%1];\n" : "=r"(v) : "l"(arrivals) : "memory");
           if (v >= (unsigned)nch) break;
-          if ((++polls & 63u) == 0 && (*abort_flag || now_ns() - t0 > kWaitBudgetNs)) {
+          if ((++polls & 63u) == 0 && (*abort_flag || now_ns() - t0 > wait_budget(abort_flag))) {
             atomicMin(p.status, QUASAR_ERR_TIMEOUT);
             *abort_flag = 1;
             ok_flag = 0;
@@ -1448,6 +1451,7 @@ __global__ void __launch_bounds__(kThreads, 1) verify_megakernel(const MegaParam
 
   if (threadIdx.x == 0) {
     *abort_flag = 0;
+    *reinterpret_cast<volatile unsigned long long*>(abort_flag + 2) = p.wait_budget_ns;
     for (int s = 0; s < kStages; ++s) {
       mbar_init(pipe.full + s, 1);     // the producer's arrive.expect_tx; the bytes complete the phase
       mbar_init(pipe.empty + s, NW);   // one arrival per consumer warp
@@ -1470,7 +1474,9 @@ __global__ void __launch_bounds__(kThreads, 1) verify_megakernel(const MegaParam
 
   int slot = 0;
   uint32_t phase = 0, xphase = 0, xphase2 = 0;
-  GridSync gs{p.barrier, p.status, (unsigned)ncta, 0u, abort_flag};
+  // (barrier_extra is zero except in the test of the failure path: a barrier that expects more arrivals than
+  // there are thread blocks cannot complete, so its first wait runs into the budget)
+  GridSync gs{p.barrier, p.status, (unsigned)ncta + p.barrier_extra, 0u, abort_flag};
   bool ok = true;
   prep_phase(p, misc, cta, ncta);
   gs.arrive();

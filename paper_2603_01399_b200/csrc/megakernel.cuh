@@ -49,6 +49,8 @@ struct MegaParams {
   unsigned* attn_count;     // [L][B*Hkv] chunks of a (sequence, kv head) whose attention partial is complete
   unsigned* amax_buf;       // [n_jobs][8] row maxima (float bits) of the un-normed GEMM operands
   unsigned* barrier;        // zeroed before every launch
+  unsigned long long wait_budget_ns;   // every device-side wait gives up after this long
+  unsigned barrier_extra;   // 0; tests of the failure path make the grid barrier expect this many more arrivals
   int32_t *accept_len, *bonus, *accept_path, *status;
 };
 
