@@ -119,6 +119,63 @@ def linear(x: np.ndarray, w: np.ndarray, delta: Optional[np.ndarray]) -> np.ndar
 
 
 # --------------------------------------------------------------------------
+# The paper's W8A8 form of the linear layer (Section 3.2 Eq. 4-8, Section 3.3 Eq. 9-10):
+# smoothing, int8 activations per token, exact integer accumulation, dequantisation.
+# Readings where the paper is silent: the activation step size is one per token (row of X),
+# absmax / 127 with the same fp32 division, rounding and zero-row rule as the weights; the
+# smoothed operands W / s and X * s are formed in fp32; the factors are computed in fp64 and
+# stored as fp32, and a channel whose activation or weight maximum is zero gets s = 1.
+# The paper is at odds with itself on the direction of s: Eq. 4 and Eq. 9 MULTIPLY the activations by
+# s and divide the weights, while Eq. 5 prints the factor of the method it builds on, which divides the
+# activations; taken together an outlier channel would be scaled UP.  Reading: Eq. 4 and Eq. 9 stand as
+# printed (two places agree), and Eq. 5 gives the factor the activations are divided by, so the s of
+# Eq. 4 / Eq. 9 is its reciprocal, max|W_j|^(1-alpha) / max|X_j|^alpha.  With alpha = 1/2 both smoothed
+# operands then have the channel maximum sqrt(max|X_j| max|W_j|), which is the stated purpose.
+# --------------------------------------------------------------------------
+
+
+def smoothing_factors(act_absmax: np.ndarray, w_f32: np.ndarray, alpha: float = 0.5) -> np.ndarray:
+    """Eq. 5 under the reading above: the factor X is multiplied by in Eq. 4 / Eq. 9,
+    s_j = max|W_j|^(1 - alpha) / max|X_j|^alpha for input channel j.
+    act_absmax: fp32 [K] calibration maxima of the layer's input; w_f32: [N][K].  Returns fp32 [K]."""
+    a = np.asarray(act_absmax, dtype=np.float32).astype(np.float64)
+    wmax = np.max(np.abs(np.asarray(w_f32, dtype=np.float32)), axis=0).astype(np.float64)
+    ok = (a > 0) & (wmax > 0)
+    with np.errstate(divide="ignore", invalid="ignore"):
+        s = np.power(wmax, 1.0 - alpha) / np.power(a, alpha)
+    return np.where(ok, s, 1.0).astype(np.float32)
+
+
+def smooth_weights(w_f32: np.ndarray, s: np.ndarray) -> np.ndarray:
+    """W diag(s)^-1 of Eq. 4 (offline weight preparation, Section 3.3), in fp32."""
+    return (np.asarray(w_f32, dtype=np.float32) / np.asarray(s, dtype=np.float32)[None, :]).astype(np.float32)
+
+
+def quantize_activations(x: np.ndarray, s: Optional[np.ndarray]):
+    """Eq. 9: X_int8 = Q(X * s, delta_x), one step size per token.  x: [M][K] holding bf16 values;
+    s: fp32 [K] or None (no smoothing).  Returns (int8 [M][K], fp32 [M])."""
+    xt = np.asarray(x, dtype=np.float32)
+    if s is not None:
+        xt = (xt * np.asarray(s, dtype=np.float32)[None, :]).astype(np.float32)
+    return quantize(xt)
+
+
+def int_matmul(xq: np.ndarray, wq: np.ndarray) -> np.ndarray:
+    """Y_int32 = W_int8 x X_int8 (Eq. 8 / Eq. 10), exact; returns int64 [M][N] (checked to fit int32)."""
+    acc = xq.astype(np.int64) @ wq.astype(np.int64).T
+    assert np.all(np.abs(acc) < 2 ** 31)
+    return acc
+
+
+def linear_w8a8(x: np.ndarray, s: Optional[np.ndarray], wq: np.ndarray, delta_w: np.ndarray) -> np.ndarray:
+    """Y ~= Y_int32 * (delta_w * delta_x) (Eq. 10).  x: [M][K] holding bf16 values; wq: int8 [N][K] =
+    Q(W diag(s)^-1, delta_w).  Returns fp64 [M][N], not yet rounded."""
+    xq, delta_x = quantize_activations(x, s)
+    acc = int_matmul(xq, wq)
+    return acc.astype(np.float64) * (delta_w.astype(np.float64)[None, :] * delta_x.astype(np.float64)[:, None])
+
+
+# --------------------------------------------------------------------------
 # Steps S2, S4, S6: RMSNorm, RoPE, SwiGLU
 # --------------------------------------------------------------------------
 
@@ -224,6 +281,8 @@ def accept_greedy(tokens: List[int], parents: List[int], top1: List[int]):
 class Linear:
     w: np.ndarray                    # int8 [N][K], or uint16 bf16 bits [N][K]
     delta: Optional[np.ndarray]      # fp32 [N] for int8 weights, None for bf16 weights
+    act_int8: bool = False           # W8A8: the input is quantised per token (Eq. 9)
+    smooth: Optional[np.ndarray] = None   # fp32 [K] smoothing factors folded into w (Eq. 4), W8A8 only
 
     def weight_for_matmul(self) -> np.ndarray:
         if self.delta is None:
@@ -231,6 +290,8 @@ class Linear:
         return self.w
 
     def __call__(self, x: np.ndarray) -> np.ndarray:
+        if self.act_int8:
+            return linear_w8a8(x, self.smooth, self.w, self.delta)
         return linear(x, self.weight_for_matmul(), self.delta)
 
 

@@ -68,7 +68,7 @@ SHAPES = {
 _KIND_IDS = {
     "embed": 1, "attn_norm": 2, "qkv": 3, "q_norm": 4, "k_norm": 5, "o": 6,
     "mlp_norm": 7, "gateup": 8, "down": 9, "final_norm": 10, "lm_head": 11,
-    "kv_k": 12, "kv_v": 13, "tokens": 14, "draft": 15, "x": 16,
+    "kv_k": 12, "kv_v": 13, "tokens": 14, "draft": 15, "x": 16, "act_absmax": 17,
 }
 
 
@@ -118,6 +118,18 @@ def gain(shape: ModelShape, kind: str, layer: int, seed: int = 0, device="cpu") 
     """Norm gain ~ U(0.5, 1.5) so that a dropped gain shows up in parity."""
     n = shape.head_dim if kind in ("q_norm", "k_norm") else shape.hidden
     return uniform_bf16((n,), 0.5, 1.5, sub_seed(seed, kind, layer), device)
+
+
+def activation_absmax(shape: ModelShape, kind: str, layer: int, seed: int = 0, device="cpu") -> torch.Tensor:
+    """Stand-in for the calibration statistic max|X_j| of a linear layer's input (fp32 [K]): most channels
+    ~ U(0.5, 4), about one in a hundred an outlier 20 times larger - the "systematic outliers in specific
+    activation channels" that smoothing is there for (Section 3.2)."""
+    dims = {nm: k for nm, _, k in shape.linear_shapes()}
+    k = dims[kind]
+    g = _gen(sub_seed(seed, "act_absmax", layer) + 7919 * _KIND_IDS[kind], device)
+    base = torch.empty(k, dtype=torch.float32, device=device).uniform_(0.5, 4.0, generator=g)
+    outlier = torch.rand(k, generator=g, device=device) < 0.01
+    return torch.where(outlier, base * 20.0, base)
 
 
 def kv_prefix(shape: ModelShape, batch: int, s_max: int, seed: int = 1, device="cpu"):
