@@ -91,6 +91,38 @@ int quasar_linear(const void* x, const void* w, const float* delta, int32_t weig
                   size_t workspace_bytes, void* stream);
 
 /* ------------------------------------------------------------------------
+ * The paper's W8A8 form (Section 3.2 Eq. 4-8, Section 3.3 Eq. 9-10): activations are quantised
+ * too, per token, after a per-channel smoothing that moves outliers from the activations into
+ * the weights.  Q(., delta) is the operator of quasar_quantize throughout.
+ *
+ * quasar_smoothing_factors (Eq. 5, offline calibration): act_absmax fp32 [K] = max|X_j| of the
+ *   layer's input over calibration data; w_bf16 [N][K].  s_out fp32 [K]:
+ *     s_j = max|W_j|^(1-alpha) / max|X_j|^alpha   (fp64 arithmetic, stored as fp32; 1 where either
+ *     maximum is zero).  This is the factor the activations are MULTIPLIED by in Eq. 4 / Eq. 9,
+ *     i.e. the reciprocal of the expression printed as Eq. 5 (see the note in w8a8.cu).
+ * quasar_quantize_weights_smoothed (Section 3.3 "Offline Weight Preparation"):
+ *     W_int8 = Q(W diag(s)^-1, delta_w), W / s in fp32; s == NULL: same as quasar_quantize.
+ * quasar_quantize_activations (Eq. 9, fused smoothing + quantisation): x bf16 [M][K],
+ *     X_int8 = Q(X * s, delta_x), one step size per token (row), x * s in fp32; s may be NULL.
+ * quasar_linear_w8a8 (Eq. 8, Eq. 10): quantises x as above into the workspace, then
+ *     Y_int32 = W_int8 x X_int8 (exact), Y = Y_int32 * (delta_w[n] * delta_x[m]) in fp32
+ *     (+ residual as in quasar_linear).  acc_out: int32 [M][N] or NULL - the raw accumulators,
+ *     for callers that want to check them.  K % 16 == 0; workspace as for quasar_linear
+ *     (first 64 KiB zero on first use), size from quasar_linear_w8a8_workspace_bytes.
+ * All bit-exact in the integer codes and accumulators; K % 8 == 0 for the quantisers.
+ * ---------------------------------------------------------------------- */
+int quasar_smoothing_factors(const float* act_absmax, const void* w_bf16, int64_t N, int64_t K, float alpha,
+                             float* s_out, void* stream);
+int quasar_quantize_weights_smoothed(const void* w_bf16, const float* s, int64_t N, int64_t K, int8_t* q_out,
+                                     float* delta_out, void* stream);
+int quasar_quantize_activations(const void* x_bf16, const float* s, int64_t M, int64_t K, int8_t* q_out,
+                                float* delta_out, void* stream);
+int quasar_linear_w8a8_workspace_bytes(int64_t M, int64_t N, int64_t K, size_t* bytes_out /* host */);
+int quasar_linear_w8a8(const void* x, const float* s, const int8_t* w, const float* delta_w, int64_t M, int64_t N,
+                       int64_t K, void* y, int32_t y_is_f32, const void* residual, int32_t* acc_out, void* workspace,
+                       size_t workspace_bytes, void* stream);
+
+/* ------------------------------------------------------------------------
  * quasar_linear for callers that may not allocate device memory.  (The paper has no
  * counterpart: this is a convenience of the library, not a step of the method.)
  *

@@ -62,6 +62,11 @@ SIGNATURES = {
     "quasar_quantize": (C.c_int, [_vp, _i64, _i64, _vp, _vp, _vp]),
     "quasar_linear_workspace_bytes": (C.c_int, [_i64, _i64, _i64, C.POINTER(_sz)]),
     "quasar_linear": (C.c_int, [_vp, _vp, _vp, _i32, _i64, _i64, _i64, _vp, _i32, _vp, _vp, _sz, _vp]),
+    "quasar_smoothing_factors": (C.c_int, [_vp, _vp, _i64, _i64, C.c_float, _vp, _vp]),
+    "quasar_quantize_weights_smoothed": (C.c_int, [_vp, _vp, _i64, _i64, _vp, _vp, _vp]),
+    "quasar_quantize_activations": (C.c_int, [_vp, _vp, _i64, _i64, _vp, _vp, _vp]),
+    "quasar_linear_w8a8_workspace_bytes": (C.c_int, [_i64, _i64, _i64, C.POINTER(_sz)]),
+    "quasar_linear_w8a8": (C.c_int, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _vp, _i32, _vp, _vp, _vp, _sz, _vp]),
     "quasar_linear_static_scratch_bytes": (_sz, []),
     "quasar_linear_static": (C.c_int, [_vp, _vp, _vp, _i32, _i64, _i64, _i64, _vp, _i32, _vp, _vp]),
     "quasar_model_create": (C.c_int, [C.POINTER(Config), C.POINTER(Weights), C.POINTER(_vp)]),
@@ -143,6 +148,49 @@ def quasar_linear(x: torch.Tensor, w: torch.Tensor, delta: Optional[torch.Tensor
     _check(lib().quasar_linear(_ptr(x), _ptr(w), _ptr(delta), wd, m, n, k, _ptr(out), 1 if out_f32 else 0,
                                _ptr(residual), _ptr(workspace), workspace.numel(), _stream()))
     return out
+
+
+def quasar_smoothing_factors(act_absmax: torch.Tensor, w_bf16: torch.Tensor, alpha: float = 0.5) -> torch.Tensor:
+    """fp32 [K] calibration maxima + bf16 [N][K] weights -> fp32 [K] smoothing factors (Eq. 5)."""
+    assert act_absmax.is_cuda and act_absmax.dtype == torch.float32 and w_bf16.dtype == torch.bfloat16
+    n, k = w_bf16.shape
+    s = torch.empty(k, dtype=torch.float32, device=w_bf16.device)
+    _check(lib().quasar_smoothing_factors(_ptr(act_absmax), _ptr(w_bf16), n, k, alpha, _ptr(s), _stream()))
+    return s
+
+
+def quasar_quantize_weights_smoothed(w_bf16: torch.Tensor, s: Optional[torch.Tensor]):
+    """Q(W diag(s)^-1, delta_w): bf16 [N][K] (+ fp32 [K]) -> (int8 [N][K], fp32 [N])."""
+    n, k = w_bf16.shape
+    q = torch.empty((n, k), dtype=torch.int8, device=w_bf16.device)
+    d = torch.empty((n,), dtype=torch.float32, device=w_bf16.device)
+    _check(lib().quasar_quantize_weights_smoothed(_ptr(w_bf16), _ptr(s), n, k, _ptr(q), _ptr(d), _stream()))
+    return q, d
+
+
+def quasar_quantize_activations(x_bf16: torch.Tensor, s: Optional[torch.Tensor]):
+    """Q(X * s, delta_x) per token: bf16 [M][K] (+ fp32 [K]) -> (int8 [M][K], fp32 [M])."""
+    m, k = x_bf16.shape
+    q = torch.empty((m, k), dtype=torch.int8, device=x_bf16.device)
+    d = torch.empty((m,), dtype=torch.float32, device=x_bf16.device)
+    _check(lib().quasar_quantize_activations(_ptr(x_bf16), _ptr(s), m, k, _ptr(q), _ptr(d), _stream()))
+    return q, d
+
+
+def quasar_linear_w8a8(x: torch.Tensor, s: Optional[torch.Tensor], w: torch.Tensor, delta_w: torch.Tensor, residual=None,
+                       out_f32=False, want_acc=False):
+    """x bf16 [M][K]; s fp32 [K] or None; w int8 [N][K]; delta_w fp32 [N].  Returns y (and the int32
+    accumulators when want_acc)."""
+    m, k = x.shape
+    n = w.shape[0]
+    y = torch.empty((m, n), dtype=torch.float32 if out_f32 else torch.bfloat16, device=x.device)
+    acc = torch.empty((m, n), dtype=torch.int32, device=x.device) if want_acc else None
+    nbytes = _sz(0)
+    _check(lib().quasar_linear_w8a8_workspace_bytes(m, n, k, C.byref(nbytes)))
+    ws = torch.zeros(int(nbytes.value), dtype=torch.uint8, device=x.device)
+    _check(lib().quasar_linear_w8a8(_ptr(x), _ptr(s), _ptr(w), _ptr(delta_w), m, n, k, _ptr(y), 1 if out_f32 else 0,
+                                    _ptr(residual), _ptr(acc), _ptr(ws), ws.numel(), _stream()))
+    return (y, acc) if want_acc else y
 
 
 def quasar_linear_static_scratch_bytes() -> int:

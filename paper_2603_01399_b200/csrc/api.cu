@@ -359,6 +359,61 @@ int quasar_linear(const void* x, const void* w, const float* delta, int32_t weig
                        (cudaStream_t)stream);
 }
 
+int quasar_smoothing_factors(const float* act_absmax, const void* w_bf16, int64_t N, int64_t K, float alpha,
+                             float* s_out, void* stream) {
+  if (N <= 0 || K <= 0 || !(alpha >= 0.f && alpha <= 1.f)) { set_error("smoothing_factors: bad size or alpha"); return QUASAR_ERR_INVALID_ARG; }
+  REQUIRE_PTR(act_absmax, "act_absmax");
+  REQUIRE_PTR(w_bf16, "w_bf16");
+  REQUIRE_PTR(s_out, "s_out");
+  return launch_smoothing_factors(act_absmax, reinterpret_cast<const __nv_bfloat16*>(w_bf16), N, K, alpha, s_out,
+                                  (cudaStream_t)stream);
+}
+
+static int quantize_smoothed_checked(const char* what, const void* v, const float* s, int mode, int64_t rows, int64_t K,
+                                     int8_t* q_out, float* delta_out, void* stream) {
+  if (rows < 0 || K < 0) { set_error("%s: negative size", what); return QUASAR_ERR_INVALID_ARG; }
+  if (rows == 0 || K == 0) return QUASAR_OK;
+  if (K % 8 != 0 || rows > 0x7fffffffLL) { set_error("%s: K=%lld must be a multiple of 8", what, (long long)K); return QUASAR_ERR_SHAPE; }
+  REQUIRE_PTR(v, "input");
+  REQUIRE_PTR(q_out, "q_out");
+  REQUIRE_PTR(delta_out, "delta_out");
+  if (s && !aligned16(s)) { set_error("%s: s is not 16-byte aligned", what); return QUASAR_ERR_ALIGN; }
+  return launch_quantize_smoothed(reinterpret_cast<const __nv_bfloat16*>(v), s, mode, rows, K, q_out, delta_out,
+                                  (cudaStream_t)stream);
+}
+
+int quasar_quantize_weights_smoothed(const void* w_bf16, const float* s, int64_t N, int64_t K, int8_t* q_out,
+                                     float* delta_out, void* stream) {
+  return quantize_smoothed_checked("quantize_weights_smoothed", w_bf16, s, 1, N, K, q_out, delta_out, stream);
+}
+
+int quasar_quantize_activations(const void* x_bf16, const float* s, int64_t M, int64_t K, int8_t* q_out,
+                                float* delta_out, void* stream) {
+  return quantize_smoothed_checked("quantize_activations", x_bf16, s, 2, M, K, q_out, delta_out, stream);
+}
+
+int quasar_linear_w8a8_workspace_bytes(int64_t M, int64_t N, int64_t K, size_t* bytes_out) {
+  if (bytes_out == nullptr || M <= 0 || N <= 0 || K <= 0) { set_error("linear_w8a8_workspace_bytes: bad argument"); return QUASAR_ERR_INVALID_ARG; }
+  *bytes_out = linear_w8a8_workspace_bytes(M, N, K);
+  return QUASAR_OK;
+}
+
+int quasar_linear_w8a8(const void* x, const float* s, const int8_t* w, const float* delta_w, int64_t M, int64_t N,
+                       int64_t K, void* y, int32_t y_is_f32, const void* residual, int32_t* acc_out, void* workspace,
+                       size_t workspace_bytes, void* stream) {
+  REQUIRE_PTR(x, "x");
+  REQUIRE_PTR(w, "w");
+  REQUIRE_PTR(delta_w, "delta_w");
+  REQUIRE_PTR(y, "y");
+  REQUIRE_PTR(workspace, "workspace");
+  if (s && !aligned16(s)) { set_error("s is not 16-byte aligned"); return QUASAR_ERR_ALIGN; }
+  if (residual && !aligned16(residual)) { set_error("residual is not 16-byte aligned"); return QUASAR_ERR_ALIGN; }
+  if (acc_out && !aligned16(acc_out)) { set_error("acc_out is not 16-byte aligned"); return QUASAR_ERR_ALIGN; }
+  return launch_linear_w8a8(reinterpret_cast<const __nv_bfloat16*>(x), s, w, delta_w, M, N, K, y, y_is_f32 != 0,
+                            reinterpret_cast<const __nv_bfloat16*>(residual), acc_out, workspace, workspace_bytes,
+                            (cudaStream_t)stream);
+}
+
 int quasar_linear_static(const void* x, const void* w, const float* delta, int32_t weight_dtype, int64_t M, int64_t N,
                          int64_t K, void* y, int32_t y_is_f32, const void* residual, void* stream) {
   if (weight_dtype != QUASAR_W_INT8 && weight_dtype != QUASAR_W_BF16) { set_error("linear_static: weight_dtype %d", weight_dtype); return QUASAR_ERR_INVALID_ARG; }

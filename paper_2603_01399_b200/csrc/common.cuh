@@ -50,6 +50,17 @@ int launch_linear_static(const __nv_bfloat16* x, const void* w, const float* del
                          int64_t N, int64_t K, void* y, bool y_is_f32, const __nv_bfloat16* residual,
                          cudaStream_t stream);
 
+// ---- W8A8 (Section 3.2 Eq. 4-8, Section 3.3 Eq. 9-10) ----
+int launch_smoothing_factors(const float* act_absmax, const __nv_bfloat16* w, int64_t N, int64_t K, float alpha,
+                             float* s_out, cudaStream_t stream);
+// mode 1: v / s (offline weights), mode 2: v * s (activations); s == nullptr: plain
+int launch_quantize_smoothed(const __nv_bfloat16* v, const float* s, int mode, int64_t rows, int64_t K, int8_t* q,
+                             float* delta, cudaStream_t stream);
+size_t linear_w8a8_workspace_bytes(int64_t M, int64_t N, int64_t K);
+int launch_linear_w8a8(const __nv_bfloat16* x, const float* smooth, const int8_t* w, const float* delta_w, int64_t M,
+                       int64_t N, int64_t K, void* y, bool y_is_f32, const __nv_bfloat16* residual, int32_t* acc_out,
+                       void* workspace, size_t workspace_bytes, cudaStream_t stream);
+
 // Per-call description of the draft blocks, derived on the device from tokens / parents / block_len.
 struct BlockInfo {
   uint64_t* anc;    // [B*T_max] bit j set: block row j is row i itself or an ancestor of it
