@@ -58,6 +58,9 @@ extern "C" {
 #define QUASAR_W_INT8 0
 #define QUASAR_W_BF16 1
 
+#define QUASAR_A_BF16 0 /* activations stay bf16 (weight-only quantisation)                      */
+#define QUASAR_A_INT8 1 /* the paper's W8A8: every linear layer quantises its input per token    */
+
 #define QUASAR_MAX_BLOCK 64 /* rows of one sequence's draft block (root + drafts / tree nodes) */
 
 const char* quasar_last_error(void);
@@ -169,6 +172,8 @@ typedef struct quasar_config {
   float rms_eps;
   int32_t weight_dtype; /* QUASAR_W_INT8 or QUASAR_W_BF16                     */
   int32_t max_seq;      /* cache capacity S_max (positions) the RoPE table covers */
+  int32_t act_dtype;    /* QUASAR_A_BF16, or QUASAR_A_INT8 (needs weight_dtype QUASAR_W_INT8; the
+                           weights must then be Q(W diag(s)^-1) for the smoothing vectors below) */
 } quasar_config;
 
 typedef struct quasar_layer_weights {
@@ -184,6 +189,12 @@ typedef struct quasar_layer_weights {
   const float* gateup_delta;
   const void* down_w;     /* [H][F]                                               */
   const float* down_delta;
+  /* act_dtype == QUASAR_A_INT8 only: smoothing factors of each linear layer's input (Eq. 4-5, Eq. 9),
+   * fp32 over the layer's input channels, or NULL for no smoothing                                   */
+  const float* qkv_smooth;    /* [H]     */
+  const float* o_smooth;      /* [Hq D]  */
+  const float* gateup_smooth; /* [H]     */
+  const float* down_smooth;   /* [F]     */
 } quasar_layer_weights;
 
 typedef struct quasar_weights {
@@ -192,6 +203,7 @@ typedef struct quasar_weights {
   const void* final_norm;             /* bf16 [H]                                  */
   const void* lm_w;                   /* [V][H]                                    */
   const float* lm_delta;              /* fp32 [V]                                  */
+  const float* lm_smooth;             /* fp32 [H] or NULL (act_dtype == QUASAR_A_INT8 only) */
 } quasar_weights;
 
 /* KV cache of the context x_<t (Section 3.1): bf16, [L][B][Hkv][S_max][D], K

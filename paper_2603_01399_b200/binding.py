@@ -17,6 +17,8 @@ LIB_PATH = os.path.join(_HERE, "libquasar.so")
 
 QUASAR_W_INT8 = 0
 QUASAR_W_BF16 = 1
+QUASAR_A_BF16 = 0
+QUASAR_A_INT8 = 1
 QUASAR_MAX_BLOCK = 64
 
 ERROR_NAMES = {0: "OK", -1: "INVALID_ARG", -2: "SHAPE", -3: "CAPACITY", -4: "ALIGN", -5: "CUDA", -6: "TIMEOUT",
@@ -33,18 +35,18 @@ class Config(C.Structure):
     _fields_ = [("n_layers", C.c_int32), ("hidden", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
                 ("head_dim", C.c_int32), ("ffn", C.c_int32), ("vocab", C.c_int32), ("qk_norm", C.c_int32),
                 ("rope_theta", C.c_float), ("rms_eps", C.c_float), ("weight_dtype", C.c_int32),
-                ("max_seq", C.c_int32)]
+                ("max_seq", C.c_int32), ("act_dtype", C.c_int32)]
 
 
 class LayerWeights(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in
                 ("attn_norm", "qkv_w", "qkv_delta", "q_norm", "k_norm", "o_w", "o_delta", "mlp_norm", "gateup_w",
-                 "gateup_delta", "down_w", "down_delta")]
+                 "gateup_delta", "down_w", "down_delta", "qkv_smooth", "o_smooth", "gateup_smooth", "down_smooth")]
 
 
 class Weights(C.Structure):
     _fields_ = [("embed", C.c_void_p), ("layers", C.POINTER(LayerWeights)), ("final_norm", C.c_void_p),
-                ("lm_w", C.c_void_p), ("lm_delta", C.c_void_p)]
+                ("lm_w", C.c_void_p), ("lm_delta", C.c_void_p), ("lm_smooth", C.c_void_p)]
 
 
 class KV(C.Structure):
@@ -219,35 +221,48 @@ class Model:
     `l{l}.attn_norm`, `.qkv_w`, `.qkv_delta`, `.q_norm`, `.k_norm`, `.o_w`, `.o_delta`, `.mlp_norm`,
     `.gateup_w`, `.gateup_delta`, `.down_w`, `.down_delta` (deltas absent for bf16 weights)."""
 
-    def __init__(self, shape, tensors: Dict[str, torch.Tensor], max_seq: int, weight_dtype: int = QUASAR_W_INT8):
+    def __init__(self, shape, tensors: Dict[str, torch.Tensor], max_seq: int, weight_dtype: int = QUASAR_W_INT8,
+                 act_dtype: int = QUASAR_A_BF16):
         self.shape = shape
         self.tensors = tensors
         self.weight_dtype = weight_dtype
+        self.act_dtype = act_dtype
         self.max_seq = max_seq
         self.cfg = Config(shape.n_layers, shape.hidden, shape.n_q_heads, shape.n_kv_heads, shape.head_dim, shape.ffn,
                           shape.vocab, 1 if shape.qk_norm else 0, shape.rope_theta, shape.rms_eps, weight_dtype,
-                          max_seq)
+                          max_seq, act_dtype)
         layers = (LayerWeights * max(shape.n_layers, 1))()
         for l in range(shape.n_layers):
             for name, _ in LayerWeights._fields_:
                 setattr(layers[l], name, _ptr(tensors.get(f"l{l}.{name}")))
         self._layers = layers
         w = Weights(_ptr(tensors["embed"]), layers, _ptr(tensors["final_norm"]), _ptr(tensors["lm_w"]),
-                    _ptr(tensors.get("lm_delta")))
+                    _ptr(tensors.get("lm_delta")), _ptr(tensors.get("lm_smooth")))
         handle = _vp()
         _check(lib().quasar_model_create(C.byref(self.cfg), C.byref(w), C.byref(handle)))
         self.handle = handle
         self._trace = None
 
     @classmethod
-    def from_master(cls, shape, get_master, max_seq: int, int8: bool = True, device="cuda"):
+    def from_master(cls, shape, get_master, max_seq: int, int8: bool = True, device="cuda", act_int8: bool = False,
+                    get_act_absmax=None, alpha: float = 0.5):
         """get_master(kind, layer) -> bf16 master tensor (any device).  int8=True quantises every
-        matrix on the GPU with quasar_quantize (the offline weight preparation)."""
+        matrix on the GPU with quasar_quantize (the offline weight preparation).  act_int8=True builds the
+        W8A8 verifier: get_act_absmax(kind, layer) -> fp32 [K] calibration maxima of the layer's input give
+        the smoothing factors (quasar_smoothing_factors), which are folded into the weights before they are
+        quantised (quasar_quantize_weights_smoothed) and kept for the online activation smoothing."""
         t: Dict[str, torch.Tensor] = {}
+        assert int8 or not act_int8
 
         def put_linear(prefix, kind, layer):
             w = get_master(kind, layer).to(device)
-            if int8:
+            if int8 and act_int8:
+                s = None
+                if get_act_absmax is not None:
+                    s = quasar_smoothing_factors(get_act_absmax(kind, layer).to(device), w, alpha)
+                    t[prefix + "_smooth"] = s
+                t[prefix + "_w"], t[prefix + "_delta"] = quasar_quantize_weights_smoothed(w, s)
+            elif int8:
                 q, d = quasar_quantize(w)
                 t[prefix + "_w"], t[prefix + "_delta"] = q, d
             else:
@@ -267,7 +282,8 @@ class Model:
             put_linear(f"l{l}.gateup", "gateup", l)
             put_linear(f"l{l}.down", "down", l)
         torch.cuda.synchronize()
-        return cls(shape, t, max_seq, QUASAR_W_INT8 if int8 else QUASAR_W_BF16)
+        return cls(shape, t, max_seq, QUASAR_W_INT8 if int8 else QUASAR_W_BF16,
+                   QUASAR_A_INT8 if act_int8 else QUASAR_A_BF16)
 
     def workspace_bytes(self, batch: int, t_max: int) -> int:
         out = _sz(0)

@@ -99,7 +99,11 @@ Workspace layout(const quasar_config& c, int B, int T_max, int s_max) {
                                 {c.hidden, c.ffn},
                                 {c.vocab, c.hidden}};
   for (auto& s : shapes) {
-    const size_t b = linear_workspace_bytes((int64_t)M, s[0], s[1]);
+    size_t b = linear_workspace_bytes((int64_t)M, s[0], s[1]);
+    if (c.act_dtype == QUASAR_A_INT8) {
+      const size_t b8 = linear_w8a8_workspace_bytes((int64_t)M, s[0], s[1]);
+      b = b8 > b ? b8 : b;
+    }
     lin = b > lin ? b : lin;
   }
   w.lin_bytes = lin;
@@ -128,6 +132,10 @@ int check_cfg(const quasar_config& c) {
   }
   if (c.weight_dtype != QUASAR_W_INT8 && c.weight_dtype != QUASAR_W_BF16) {
     set_error("config: weight_dtype %d", c.weight_dtype);
+    return QUASAR_ERR_INVALID_ARG;
+  }
+  if (c.act_dtype != QUASAR_A_BF16 && !(c.act_dtype == QUASAR_A_INT8 && c.weight_dtype == QUASAR_W_INT8)) {
+    set_error("config: act_dtype %d (int8 activations need int8 weights)", c.act_dtype);
     return QUASAR_ERR_INVALID_ARG;
   }
   if ((c.head_dim != 64 && c.head_dim != 128) || c.hidden % 16 || c.ffn % 16 || c.n_q_heads % c.n_kv_heads ||
@@ -234,6 +242,15 @@ int verify_impl(quasar_model* m, const quasar_kv* kv, const int32_t* tokens, con
   const int H = c.hidden, D = c.head_dim, Hq = c.n_q_heads, Hkv = c.n_kv_heads, F = c.ffn;
   const int qkv_w = (Hq + 2 * Hkv) * D;
   const int wd = c.weight_dtype;
+  const bool a8 = c.act_dtype == QUASAR_A_INT8;
+  // one linear layer of the pass: weight-only (Eq. 8 with bf16 activations) or the paper's W8A8 form (Eq. 9-10)
+  auto linear = [&](const __nv_bfloat16* in, const void* w, const float* delta, const float* smooth, int64_t N, int64_t K,
+                    void* out, bool out_f32, const __nv_bfloat16* res) -> int {
+    if (a8)
+      return launch_linear_w8a8(in, smooth, reinterpret_cast<const int8_t*>(w), delta, M, N, K, out, out_f32, res, nullptr,
+                                lin, ws.lin_bytes, stream);
+    return launch_linear(in, w, delta, wd, M, N, K, out, out_f32, res, lin, ws.lin_bytes, stream);
+  };
   const size_t layer_stride = (size_t)kv->batch * Hkv * (size_t)kv->s_max * D;
   TraceCursor tr{reinterpret_cast<unsigned char*>(m->trace_buf), 0, m->trace_bytes, stream};
 
@@ -284,7 +301,7 @@ int verify_impl(quasar_model* m, const quasar_kv* kv, const int32_t* tokens, con
     __nv_bfloat16* vc = reinterpret_cast<__nv_bfloat16*>(kv->v) + (size_t)l * layer_stride;
     TRY(launch_rmsnorm(x, reinterpret_cast<const __nv_bfloat16*>(L.attn_norm), M, H, c.rms_eps, h, stream));
     TRY(tr.put(h, (size_t)M * H * 2));
-    TRY(launch_linear(h, L.qkv_w, L.qkv_delta, wd, M, qkv_w, H, qkv, false, nullptr, lin, ws.lin_bytes, stream));
+    TRY(linear(h, L.qkv_w, L.qkv_delta, L.qkv_smooth, qkv_w, H, qkv, false, nullptr));
     TRY(tr.put(qkv, (size_t)M * qkv_w * 2));
     TRY(launch_rope_append(qkv, reinterpret_cast<const __nv_bfloat16*>(c.qk_norm ? L.q_norm : nullptr),
                            reinterpret_cast<const __nv_bfloat16*>(c.qk_norm ? L.k_norm : nullptr), m->rope_table,
@@ -293,18 +310,18 @@ int verify_impl(quasar_model* m, const quasar_kv* kv, const int32_t* tokens, con
     TRY(launch_attention(qkv, kc, vc, kv->seq_len, block_len, bi, B, T_max, Hq, Hkv, D, kv->s_max, attn, att,
                          ws.att_bytes, stream));
     TRY(tr.put(attn, (size_t)M * Hq * D * 2));
-    TRY(launch_linear(attn, L.o_w, L.o_delta, wd, M, H, Hq * D, x, false, x, lin, ws.lin_bytes, stream));
+    TRY(linear(attn, L.o_w, L.o_delta, L.o_smooth, H, Hq * D, x, false, x));
     TRY(tr.put(x, (size_t)M * H * 2));
     TRY(launch_rmsnorm(x, reinterpret_cast<const __nv_bfloat16*>(L.mlp_norm), M, H, c.rms_eps, h, stream));
-    TRY(launch_linear(h, L.gateup_w, L.gateup_delta, wd, M, 2 * F, H, gu, false, nullptr, lin, ws.lin_bytes, stream));
+    TRY(linear(h, L.gateup_w, L.gateup_delta, L.gateup_smooth, 2 * F, H, gu, false, nullptr));
     TRY(launch_swiglu(gu, M, F, act, stream));
     TRY(tr.put(act, (size_t)M * F * 2));
-    TRY(launch_linear(act, L.down_w, L.down_delta, wd, M, H, F, x, false, x, lin, ws.lin_bytes, stream));
+    TRY(linear(act, L.down_w, L.down_delta, L.down_smooth, H, F, x, false, x));
     TRY(tr.put(x, (size_t)M * H * 2));
   }
   TRY(launch_rmsnorm(x, reinterpret_cast<const __nv_bfloat16*>(m->w.final_norm), M, H, c.rms_eps, h, stream));
   TRY(tr.put(h, (size_t)M * H * 2));
-  TRY(launch_linear(h, m->w.lm_w, m->w.lm_delta, wd, M, c.vocab, H, logits, true, nullptr, lin, ws.lin_bytes, stream));
+  TRY(linear(h, m->w.lm_w, m->w.lm_delta, m->w.lm_smooth, c.vocab, H, logits, true, nullptr));
   TRY(launch_argmax(logits, M, c.vocab, top1, stream));
   TRY(launch_accept(tokens, parents, block_len, top1, bi, B, T_max, accept_len, bonus, accept_path, stream));
   return QUASAR_OK;
@@ -480,7 +497,8 @@ int quasar_model_create(const quasar_config* cfg, const quasar_weights* w, quasa
   // The persistent kernel: its grid, a permuted copy of every matrix in the order each CTA streams it,
   // and the table of the GEMMs of the pass in execution order.
   int ncta = 0;
-  if (mega_grid_size(cfg->weight_dtype, cfg->head_dim, &ncta) == QUASAR_OK && ncta > 0 && ncta <= kMaxGrid) {
+  if (cfg->act_dtype == QUASAR_A_BF16 && mega_grid_size(cfg->weight_dtype, cfg->head_dim, &ncta) == QUASAR_OK && ncta > 0 &&
+      ncta <= kMaxGrid) {
     std::vector<MegaJob> jobs;
     std::vector<MegaLayer> mls;
     std::vector<const void*> src;

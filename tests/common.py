@@ -19,9 +19,11 @@ def master_getter(shape, seed=0, device="cpu"):
     return get
 
 
-def oracle_model(shape, seed=0, int8=True, device="cpu"):
+def oracle_model(shape, seed=0, int8=True, device="cpu", act_int8=False):
     get = master_getter(shape, seed, device)
-    return oracle.build_model(shape, lambda kind, layer: synth.bf16_bits(get(kind, layer)), int8=int8)
+    absmax = (lambda kind, layer: synth.activation_absmax(shape, kind, layer, seed).numpy()) if act_int8 else None
+    return oracle.build_model(shape, lambda kind, layer: synth.bf16_bits(get(kind, layer)), int8=int8,
+                              act_int8=act_int8, get_act_absmax=absmax)
 
 
 def oracle_greedy_continuation(model, kv, root_token, n):
@@ -51,9 +53,11 @@ def prefill_oracle(model, kv, tokens_1d, chunk):
 
 
 # ---- CUDA-path side (imports nothing from oracle) ------------------------------------------
-def gpu_model(shape, seed=0, int8=True, max_seq=128, gen_device="cpu"):
+def gpu_model(shape, seed=0, int8=True, max_seq=128, gen_device="cpu", act_int8=False):
     from paper_2603_01399_b200 import binding
-    return binding.Model.from_master(shape, master_getter(shape, seed, gen_device), max_seq, int8=int8)
+    absmax = (lambda kind, layer: synth.activation_absmax(shape, kind, layer, seed)) if act_int8 else None
+    return binding.Model.from_master(shape, master_getter(shape, seed, gen_device), max_seq, int8=int8,
+                                     act_int8=act_int8, get_act_absmax=absmax)
 
 
 def logits_close(gpu, ref, abs_tol=2e-2, rel_tol=1e-2):
