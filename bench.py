@@ -261,16 +261,26 @@ def run_ours(args):
     rel_diff = float((cmp_logits["int8"] - cmp_logits["bf16"]).abs().mean() / cmp_logits["bf16"].std())
     del cmp_logits
 
-    batch8 = time_batch8(binding, m_int8, shape, max(3, args.steps // 5)) if rank == 0 else None
+    peaks, peak_kind = measured_peaks()
+    hbm_peak = float(peaks["hbm_gbs"])
+    batch8 = time_batch8(binding, m_int8, shape, max(3, args.steps // 5), hbm_peak) if rank == 0 else None
 
     # the per-step skinny GEMM (used for blocks of more than 8 rows) over the model's 145 matrices in pass order
     gemm = time_gemm_sweep(binding, m_int8, shape, BATCH * t_rows, max(3, args.steps // 4))
 
     # bf16-weight sibling pass (the "BF16 verifier" of Section 3.4, same kernels)
     bf16_ms, bbuf, bplan, _, _ = timed_plan(m_bf16, max(3, args.steps // 4), 3, False)
+    bplan.close()
+    del bbuf, bplan
+    m_bf16.close()
+    del m_bf16
+    torch.cuda.empty_cache()
+    extra = {}
+    if rank == 0 and not args.headline_only:
+        extra["w8a8"] = time_w8a8(binding, shape, kv, tokens_host, max(3, args.steps // 4), hbm_peak)
+        extra["linear_sweep"] = linear_sweep_summary(binding, hbm_peak)
+        extra["tree14b"] = time_tree14b(binding, max(3, args.steps // 5), hbm_peak)
 
-    peaks, peak_kind = measured_peaks()
-    hbm_peak = float(peaks["hbm_gbs"])
     ab = algorithmic_bytes(shape, BATCH, t_rows, PREFIX * BATCH, 1)
     ab16 = algorithmic_bytes(shape, BATCH, t_rows, PREFIX * BATCH, 2)
     pass_gbs = ab["total"] / (ms_step * 1e-3) / 1e9
@@ -288,7 +298,7 @@ def run_ours(args):
         "verify_latency_ms": ms_step, "verify_latency_ms_median_of_100": lat_median, "verify_latency_ms_min_of_100": lat_min,
         "int8_vs_bf16": {"top1_agreement": agree, "mean_abs_logit_diff_over_logit_std": rel_diff,
                          "note": "random-initialised weights: quantisation noise through 36 random layers decorrelates the logits"},
-        "batch8_ragged": batch8,
+        "batch8_ragged": batch8, **extra,
         "accepted_per_pass": accepted, "accepted_drafts_per_pass": accepted_drafts,
         "accepted_drafts_tok_s": accepted_drafts_job / (ms_step * 1e-3), "device_status": status,
         "own_draft": {"what": "draft = the int8 model's own greedy continuation, each token replaced w.p. 0.3",
@@ -316,7 +326,7 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-def time_batch8(binding, model, shape, reps):
+def time_batch8(binding, model, shape, reps, hbm_peak):
     """Not the headline: the same model on 8 sequences with seeded prefixes in 512..4096 and chains of 8
     drafts (72 block rows), which runs one kernel per step (a CUDA graph).  Latency and bytes only."""
     import numpy as np
@@ -339,12 +349,117 @@ def time_batch8(binding, model, shape, reps):
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1) / reps
     ab = algorithmic_bytes(shape, 8, 9, sum(prefix), 1)
+    gbs = ab["total"] / (ms * 1e-3) / 1e9
     out = {"workload": "B=8, prefixes U(512,4096) (sum %d), chain gamma=8, 72 block rows, int8 weights" % sum(prefix),
-           "verify_latency_ms": ms, "pass_bytes": ab["total"], "pass_hbm_gbs": ab["total"] / (ms * 1e-3) / 1e9,
-           "device_status": int(buf.status[0])}
+           "verify_latency_ms": ms, "pass_bytes": ab["total"], "pass_hbm_gbs": gbs,
+           "roofline": {"bound": "hbm", "achieved": gbs, "peak": hbm_peak, "unit": "GB/s", "frac": gbs / hbm_peak},
+           "launch": "one kernel per step, replayed as a CUDA graph", "device_status": int(buf.status[0])}
     plan.close()
     del kv, buf, kk, vv
     return out
+
+
+def _time_plan(plan, reps, warm=3):
+    for _ in range(warm):
+        plan.launch()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        plan.launch()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / reps
+
+
+def time_tree14b(binding, reps, hbm_peak):
+    """Not the headline: the Qwen3-14B-shaped model (40 layers, hidden 5120, 40/8 heads, FFN 17408), B=4,
+    2048 cached positions, the 16-node draft tree (17 rows per sequence, 68 block rows), int8 weights."""
+    shape = synth.SHAPES["qwen3_14b"]
+    s_max = 2048 + 32
+    model = binding.Model.from_master(shape, master_getter(shape, 0, "cuda"), s_max, int8=True)
+    kk, vv = synth.kv_prefix(shape, 4, s_max, seed=1, device="cuda")
+    kv = binding.KVCache(shape, 4, s_max, k=kk, v=vv, seq_len=torch.full((4,), 2048, dtype=torch.int32, device="cuda"))
+    buf = binding.VerifyBuffers(model, 4, 17, want_logits=False, tree=True)
+    buf.tokens.copy_(synth.uniform_tokens((4, 17), shape.vocab, synth.sub_seed(2, "tokens")))
+    buf.parents.copy_(torch.tensor([synth.tree_parents_16()] * 4, dtype=torch.int32))
+    plan = binding.Plan(model, kv, buf)
+    ms = _time_plan(plan, reps)
+    ab = algorithmic_bytes(shape, 4, 17, 4 * 2048, 1)
+    gbs = ab["total"] / (ms * 1e-3) / 1e9
+    out = {"workload": "qwen3-14b-shaped, B=4, prefix 2048, tree of 16 nodes (17 rows per sequence, 68 block rows), int8 weights",
+           "verify_latency_ms": ms, "pass_bytes": ab["total"], "pass_hbm_gbs": gbs,
+           "accepted_per_pass": int((buf.accept_len + 1).sum()),
+           "roofline": {"bound": "hbm", "achieved": gbs, "peak": hbm_peak, "unit": "GB/s", "frac": gbs / hbm_peak},
+           "launch": "one kernel per step, replayed as a CUDA graph", "device_status": int(buf.status[0])}
+    plan.close()
+    model.close()
+    del model, kv, buf, kk, vv
+    torch.cuda.empty_cache()
+    return out
+
+
+def time_w8a8(binding, shape, kv, tokens_host, reps, hbm_peak):
+    """The paper's W8A8 verifier (Section 3.2-3.3) on the headline workload: smoothing factors from synthetic
+    calibration maxima, int8 activations per token, integer tensor-core GEMMs."""
+    model = binding.Model.from_master(shape, master_getter(shape, 0, "cuda"), PREFIX + 16, int8=True, act_int8=True,
+                                      get_act_absmax=lambda kind, layer: synth.activation_absmax(shape, kind, layer, 0, "cuda"))
+    buf = binding.VerifyBuffers(model, BATCH, GAMMA + 1, want_logits=False)
+    buf.tokens.copy_(tokens_host)
+    plan = binding.Plan(model, kv, buf)
+    ms = _time_plan(plan, reps)
+    ab = algorithmic_bytes(shape, BATCH, GAMMA + 1, PREFIX * BATCH, 1)
+    smooth = (2 * shape.hidden + shape.q_dim + shape.ffn) * 4 * shape.n_layers + shape.hidden * 4
+    total = ab["total"] + smooth
+    gbs = total / (ms * 1e-3) / 1e9
+    out = {"workload": WORKLOAD.replace("int8 weights", "int8 weights and int8 activations (W8A8, smoothed)"),
+           "verify_latency_ms": ms, "pass_bytes": total, "pass_hbm_gbs": gbs,
+           "accepted_per_pass": int((buf.accept_len + 1).sum()),
+           "roofline": {"bound": "hbm", "achieved": gbs, "peak": hbm_peak, "unit": "GB/s", "frac": gbs / hbm_peak},
+           "launch": model.launch_kind(BATCH, GAMMA + 1), "device_status": int(buf.status[0])}
+    plan.close()
+    model.close()
+    del model, buf
+    torch.cuda.empty_cache()
+    return out
+
+
+def linear_sweep_summary(binding, hbm_peak):
+    """Compact form of `--linear-sweep` for the bench line: int8 weights, the five Qwen3-8B matrix shapes, row
+    counts 1..64; per shape the best and the worst cell as a fraction of the copy bandwidth.  Distinct weight
+    copies (>= 1 GB in total) per cell so that no launch finds its matrix in L2."""
+    shapes = [("qkv", 4096, 6144), ("o", 4096, 4096), ("gateup", 4096, 24576), ("down", 12288, 4096), ("lm_head", 4096, 151936)]
+    rows = [1, 2, 4, 5, 8, 16, 40, 64]
+    out = {}
+    for name, k, n in shapes:
+        copies = max(2, -(-(1 << 30) // (n * k)))
+        master = synth.normal_bf16((n, k), 0.02, seed=k + n, device="cuda")
+        q, d = binding.quasar_quantize(master)
+        ws_list = [q] + [q.clone() for _ in range(copies - 1)]
+        cells = {}
+        for m in rows:
+            x = synth.normal_bf16((m, k), 1.0, seed=m, device="cuda")
+            y = torch.empty((m, n), dtype=torch.bfloat16, device="cuda")
+            ws = torch.zeros(binding.quasar_linear_workspace_bytes(m, n, k), dtype=torch.uint8, device="cuda")
+            for w in ws_list:
+                binding.quasar_linear(x, w, d, workspace=ws, out=y)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(2):
+                for w in ws_list:
+                    binding.quasar_linear(x, w, d, workspace=ws, out=y)
+            e1.record()
+            torch.cuda.synchronize()
+            us = e0.elapsed_time(e1) * 1e3 / (2 * copies)
+            cells[m] = (n * k + 4 * n) / (us * 1e-6) / 1e9 / hbm_peak
+        best, worst = max(cells, key=cells.get), min(cells, key=cells.get)
+        out[name] = {"K": k, "N": n, "best": {"M": best, "frac": cells[best]}, "worst": {"M": worst, "frac": cells[worst]},
+                     "frac_by_rows": {str(m): round(f, 4) for m, f in cells.items()}}
+        del ws_list, master, q
+        torch.cuda.empty_cache()
+    return {"what": "quantised linear layer alone (quasar_linear, int8 weights), fraction of the measured copy bandwidth",
+            "shapes": out}
 
 
 def run_linear_sweep(args):
@@ -497,18 +612,21 @@ def run_reference(args):
         return
     shape = synth.SHAPES["qwen3_8b"]
     sample = OracleSample(shape)
-    times = []
+    times, sampled = [], []
     for i in range(args.warmup + args.steps):
-        _, _, full = sample.time_once()
+        per_layer, head, full = sample.time_once()
         if i >= args.warmup:
             times.append(full)
+            sampled.append(per_layer + head)
     full = sum(times) / len(times)
+    step_s = sum(sampled) / len(sampled)   # what a step of this arm really ran: the bounded sample
     accepted = 1.0   # the oracle's pass emits at least the bonus token; drafts are not generated on this arm
     val = accepted / full
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": val,
         "unit": "accepted tok/s", "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": full * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "ms_per_step": step_s * 1e3, "ms_per_pass_extrapolated": full * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
         "data": "synthetic", "config": {"workload": WORKLOAD},
         "cpu_baseline": {"value": val, "unit": "accepted tok/s", "kind": "oracle", "cores": sample.threads,
                          "sample": "each step: 1 of 36 decoder layers + LM head at full widths, scaled to 36 layers; "
@@ -553,11 +671,26 @@ def main():
                     help="run one eager verify pass inside cudaProfilerStart/Stop (for ncu), no timing")
     ap.add_argument("--profile-layers", type=int, default=0, help="with --profile-pass: cut the model to this many layers")
     ap.add_argument("--linear-sweep", action="store_true", help="time the quantised linear layer alone over shapes and row counts")
+    ap.add_argument("--headline-only", action="store_true", help="skip the side workloads (W8A8, linear sweep, 14B tree)")
     args = ap.parse_args()
     if args.profile_pass:
         return run_profile_pass(args)
     if args.linear_sweep:
         return run_linear_sweep(args)
+    # --gpus N: N independent replicas (the pass has no exchange step), one process per GPU.  Launched
+    # without a process launcher the replicas are started here; under torchrun the world size must agree.
+    world_env = os.environ.get("WORLD_SIZE")
+    if world_env is not None and int(world_env) != args.gpus:
+        print(f"bench.py: --gpus {args.gpus} but WORLD_SIZE={world_env}", file=sys.stderr)
+        sys.exit(2)
+    if world_env is None and args.gpus > 1:
+        import socket
+        with socket.socket() as sock:
+            sock.bind(("127.0.0.1", 0))
+            port = sock.getsockname()[1]
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+               "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+        sys.exit(subprocess.call(cmd))
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
         run_reference(args)

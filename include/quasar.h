@@ -311,6 +311,10 @@ int quasar_set_trace(quasar_model* m, void* trace_buf, size_t bytes);
  * Both compute the same pass (Section 3.1, 3.3); they differ in summation order only. */
 int quasar_set_path(quasar_model* m, int32_t path);
 
+/* 1 if quasar_verify would run a block of this size as the persistent single kernel (with the
+ * current quasar_set_path setting and no trace), 0 if as one kernel per step, negative on error. */
+int quasar_uses_persistent_kernel(const quasar_model* m, int32_t B, int32_t T_max);
+
 /* Every wait inside the persistent kernel (grid barrier, stage barrier, attention arrival
  * count) is bounded: after budget_ns (default 2e9) the waiting thread block sets `status` to
  * QUASAR_ERR_TIMEOUT, tells its other warps to stop waiting and returns once its own copies

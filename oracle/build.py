@@ -12,8 +12,24 @@ import numpy as np
 from . import quasar_oracle as qo
 
 
+def quantize_rows_in_parallel(w_f32: np.ndarray, workers: int = 0):
+    """qo.quantize applied to blocks of rows on a thread pool (every row is quantised on its own, so
+    the result is the one call's; numpy releases the interpreter lock inside its loops).  For building
+    full-size models in reasonable time."""
+    import os
+    from concurrent.futures import ThreadPoolExecutor
+    workers = workers or min(32, os.cpu_count() or 1)
+    n = w_f32.shape[0]
+    step = max(64, -(-n // (4 * workers)))
+    blocks = [(i, min(n, i + step)) for i in range(0, n, step)]
+    with ThreadPoolExecutor(workers) as ex:
+        parts = list(ex.map(lambda b: qo.quantize(w_f32[b[0]:b[1]]), blocks))
+    return np.concatenate([p[0] for p in parts], axis=0), np.concatenate([p[1] for p in parts])
+
+
 def build_model(shape, get_bits: Callable[[str, int], np.ndarray], int8: bool = True, act_int8: bool = False,
-                get_act_absmax: Optional[Callable[[str, int], np.ndarray]] = None, alpha: float = 0.5) -> qo.Model:
+                get_act_absmax: Optional[Callable[[str, int], np.ndarray]] = None, alpha: float = 0.5,
+                parallel: bool = False) -> qo.Model:
     """shape: any object with n_layers, hidden, n_q_heads, n_kv_heads, head_dim,
     ffn, vocab, qk_norm, rope_theta, rms_eps attributes.
     act_int8: the paper's W8A8 verifier (Section 3.2-3.3): every linear layer quantises its input per
@@ -31,7 +47,7 @@ def build_model(shape, get_bits: Callable[[str, int], np.ndarray], int8: bool = 
         if act_int8 and get_act_absmax is not None:
             s = qo.smoothing_factors(get_act_absmax(kind, layer), w, alpha)
             w = qo.smooth_weights(w, s)
-        q, delta = qo.quantize(w)                            # Section 3.3 "Offline Weight Preparation"
+        q, delta = quantize_rows_in_parallel(w) if parallel else qo.quantize(w)   # Section 3.3 "Offline Weight Preparation"
         return qo.Linear(q, delta, act_int8=act_int8, smooth=s)
 
     layers = []

@@ -84,6 +84,7 @@ SIGNATURES = {
     "quasar_set_trace": (C.c_int, [_vp, _vp, _sz]),
     "quasar_set_path": (C.c_int, [_vp, _i32]),
     "quasar_set_wait_budget": (C.c_int, [_vp, C.c_uint64, _i32]),
+    "quasar_uses_persistent_kernel": (C.c_int, [_vp, _i32, _i32]),
 }
 
 
@@ -302,6 +303,11 @@ class Model:
     def set_path(self, path: int) -> None:
         """0 automatic, 1 one kernel per step, 2 persistent single-kernel pass."""
         _check(lib().quasar_set_path(self.handle, path))
+
+    def launch_kind(self, batch: int, t_max: int) -> str:
+        """How quasar_verify runs a block of this size (for reports)."""
+        persistent = int(lib().quasar_uses_persistent_kernel(self.handle, batch, t_max)) == 1
+        return "one persistent cooperative kernel per step" if persistent else "one kernel per step, replayed as a CUDA graph"
 
     def set_wait_budget(self, budget_ns: int, test_extra_arrivals: int = 0) -> None:
         """Bound of every device-side wait of the persistent kernel (default 2 s)."""

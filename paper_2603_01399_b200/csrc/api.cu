@@ -587,6 +587,11 @@ int quasar_set_path(quasar_model* m, int32_t path) {
   return QUASAR_OK;
 }
 
+int quasar_uses_persistent_kernel(const quasar_model* m, int32_t B, int32_t T_max) {
+  if (m == nullptr || B < 1 || T_max < 1) { set_error("uses_persistent_kernel: bad argument"); return QUASAR_ERR_INVALID_ARG; }
+  return uses_persistent_kernel(m, B, T_max) ? 1 : 0;
+}
+
 int quasar_set_wait_budget(quasar_model* m, uint64_t budget_ns, int32_t test_extra_arrivals) {
   if (m == nullptr || budget_ns == 0 || test_extra_arrivals < 0 || test_extra_arrivals > 1024) {
     set_error("set_wait_budget: bad argument");

@@ -40,6 +40,25 @@ def test_two_rank_reductions_over_gloo(tmp_path):
 
 def test_reference_arm_only_works_on_rank_zero():
     env = dict(os.environ, RANK="1", LOCAL_RANK="1", WORLD_SIZE="2")
-    p = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--steps", "1", "--warmup", "0"],
-                       env=env, capture_output=True, text=True, timeout=120)
+    p = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--impl", "reference", "--steps", "1",
+                        "--warmup", "0"], env=env, capture_output=True, text=True, timeout=120)
     assert p.returncode == 0 and p.stdout.strip() == ""
+
+
+def test_gpus_flag_starts_the_replicas_itself_and_checks_the_world_size():
+    """`bench.py --gpus 2` without a launcher starts two replica processes (here: the reference arm, on CPU):
+    exactly one JSON line comes back, from rank 0, with n_gpus 2; under a launcher a world size that
+    disagrees with --gpus is refused."""
+    import json
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_ADDR", "MASTER_PORT")}
+    p = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--impl", "reference", "--steps", "1",
+                        "--warmup", "0"], env=env, capture_output=True, text=True, timeout=900)
+    assert p.returncode == 0, p.stderr[-2000:]
+    lines = [l for l in p.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    rec = json.loads(lines[0])
+    assert rec["impl"] == "reference" and rec["n_gpus"] == 2 and rec["value"] > 0
+    assert rec["ms_per_step"] < rec["ms_per_pass_extrapolated"]
+    bad = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "4", "--impl", "reference"],
+                         env=dict(env, WORLD_SIZE="2", RANK="0", LOCAL_RANK="0"), capture_output=True, text=True, timeout=120)
+    assert bad.returncode == 2 and "WORLD_SIZE" in bad.stderr
