@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libquasar.so")
-SOURCES = ["api.cu", "quantize.cu", "gemm.cu", "layer_ops.cu", "attention.cu", "megakernel.cu", "w8a8.cu"]
+SOURCES = ["api.cu", "quantize.cu", "gemm.cu", "layer_ops.cu", "attention.cu", "megakernel.cu", "w8a8.cu", "umma_gemm.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC",
@@ -48,7 +48,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if failed:
         raise RuntimeError("nvcc failed")
     if procs or not os.path.exists(LIB):
-        cmd = [nvcc, "-shared", "-o", LIB, *objs, "-lcudart"]
+        cmd = [nvcc, "-shared", "-o", LIB, *objs, "-lcudart"]   # the driver API entry for tensor maps is looked up at run time
         subprocess.check_call(cmd)
     return LIB
 

@@ -248,7 +248,7 @@ int verify_impl(quasar_model* m, const quasar_kv* kv, const int32_t* tokens, con
                     void* out, bool out_f32, const __nv_bfloat16* res) -> int {
     if (a8)
       return launch_linear_w8a8(in, smooth, reinterpret_cast<const int8_t*>(w), delta, M, N, K, out, out_f32, res, nullptr,
-                                lin, ws.lin_bytes, stream);
+                                lin, ws.lin_bytes, status, stream);
     return launch_linear(in, w, delta, wd, M, N, K, out, out_f32, res, lin, ws.lin_bytes, stream);
   };
   const size_t layer_stride = (size_t)kv->batch * Hkv * (size_t)kv->s_max * D;
@@ -427,7 +427,7 @@ int quasar_linear_w8a8(const void* x, const float* s, const int8_t* w, const flo
   if (residual && !aligned16(residual)) { set_error("residual is not 16-byte aligned"); return QUASAR_ERR_ALIGN; }
   if (acc_out && !aligned16(acc_out)) { set_error("acc_out is not 16-byte aligned"); return QUASAR_ERR_ALIGN; }
   return launch_linear_w8a8(reinterpret_cast<const __nv_bfloat16*>(x), s, w, delta_w, M, N, K, y, y_is_f32 != 0,
-                            reinterpret_cast<const __nv_bfloat16*>(residual), acc_out, workspace, workspace_bytes,
+                            reinterpret_cast<const __nv_bfloat16*>(residual), acc_out, workspace, workspace_bytes, nullptr,
                             (cudaStream_t)stream);
 }
 

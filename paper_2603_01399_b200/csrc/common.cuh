@@ -59,7 +59,14 @@ int launch_quantize_smoothed(const __nv_bfloat16* v, const float* s, int mode, i
 size_t linear_w8a8_workspace_bytes(int64_t M, int64_t N, int64_t K);
 int launch_linear_w8a8(const __nv_bfloat16* x, const float* smooth, const int8_t* w, const float* delta_w, int64_t M,
                        int64_t N, int64_t K, void* y, bool y_is_f32, const __nv_bfloat16* residual, int32_t* acc_out,
-                       void* workspace, size_t workspace_bytes, cudaStream_t stream);
+                       void* workspace, size_t workspace_bytes, int32_t* status, cudaStream_t stream);
+
+// tcgen05 form of the W8A8 linear layer for blocks of 9..80 rows (umma_gemm.cu)
+bool umma_w8a8_usable(int64_t M, int64_t N, int64_t K);
+size_t umma_w8a8_partial_bytes(int64_t M, int64_t N, int64_t K);
+int launch_umma_w8a8(const int8_t* xq, const float* dx, const int8_t* w, const float* dw, int64_t M, int64_t N, int64_t K,
+                     void* y, bool y_is_f32, const __nv_bfloat16* residual, int32_t* acc_out, int* counters, void* partial,
+                     int32_t* error_word, cudaStream_t stream);
 
 // Per-call description of the draft blocks, derived on the device from tokens / parents / block_len.
 struct BlockInfo {

@@ -1,0 +1,379 @@
+// The quantised linear layer for blocks of 9 to 72 rows on the 5th-generation tensor cores
+// (tcgen05.mma with the accumulator in tensor memory): the regime of the batched and tree
+// workloads, where  Y = delta * (W X)  (Section 3.2 Eq. 8 / Section 3.3 Eq. 10) is a real dense
+// contraction (2 M flop per weight byte, M up to 72) and no longer a pure weight stream.
+//
+// Mapping.  A CTA owns 128 output channels x one range of the contraction index.  The weights
+// are the 128-row operand A (K-major), the activation rows - padded to a multiple of 16 - the
+// operand B (K-major); the 128 x Mpad accumulator lives in tensor memory (one lane per output
+// channel, one column per activation row) and never touches registers until the epilogue.
+//   * W8A8 (kind::i8, s8 x s8 -> s32): tiles of 128 rows x 128 contraction bytes are brought in by
+//     TMA (cp.async.bulk.tensor, 128-byte swizzle) exactly as the MMA reads them - no instruction
+//     touches a weight byte.  Accumulators are exact integers.
+//   * W8A16 (kind::f16, bf16 x bf16 -> f32): the same int8 tiles land in a raw ring; four warps
+//     turn each into a bf16 tile in the MMA's swizzled layout (int8 -> bf16 is exact), which is
+//     what the weight-only form costs on this path: 2 more bytes of shared-memory traffic per
+//     weight and one conversion instruction per two weights.
+// Roles: warp 0 issues the TMA loads, warp 1 the MMAs (one elected thread), warps 2-5 convert
+// (W8A16) and run the epilogue (tcgen05.ld, one tensor-memory lane = one output channel per
+// thread).  k-ranges of one channel block are reduced in a fixed order by the last CTA to arrive.
+//
+// Every wait is bounded (2 s): on expiry the CTA raises an error word, stops waiting everywhere,
+// releases its tensor memory and returns.
+#include <cuda.h>
+#include <cudaTypedefs.h>
+
+#include <mutex>
+
+#include "common.cuh"
+
+namespace quasar {
+
+namespace {
+
+constexpr int kTileN = 128;          // output channels per CTA (MMA M)
+constexpr int kTileKBytes = 128;     // contraction bytes of int8 per stage (one 128-byte swizzle row)
+constexpr int kStagesI8 = 6;
+constexpr int kThreadsU = 192;
+constexpr int kMaxMpad = 80;
+constexpr unsigned long long kBudgetNs = 2000000000ull;
+constexpr size_t kCounterBytesU = 64 * 1024;
+
+struct UmmaArgs {
+  const float* dx;           // [M] activation step sizes (W8A8) or nullptr
+  const float* dw;           // [N]
+  void* y;                   // [M][N] bf16 or fp32
+  const __nv_bfloat16* res;  // [M][N] or nullptr
+  int32_t* acc_out;          // [M][N] raw accumulators (W8A8) or nullptr
+  void* partial;             // [nsplit][Mpad][N] 32-bit words
+  int* counters;
+  int32_t* error;            // device status word (or nullptr): QUASAR_ERR_TIMEOUT when a wait ran out
+  int M, Mpad, N, K, k_per_split, nsplit, y_is_f32;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ unsigned long long gtime_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;\n" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void mbar_init(uint64_t* bar, int count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
+               : "=r"(ok)
+               : "r"(smem_u32(bar)), "r"(parity)
+               : "memory");
+  return ok != 0;
+}
+// bounded wait; false when it ran out or another thread of the CTA already gave up
+__device__ __noinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int32_t* error) {
+  if (mbar_try(bar, parity)) return true;
+  const unsigned long long t0 = gtime_ns();
+  unsigned it = 0;
+  while (!mbar_try(bar, parity)) {
+    if ((++it & 63u) == 0) {
+      if (*abort_flag) return false;
+      if (gtime_ns() - t0 > kBudgetNs) {
+        *abort_flag = 1;
+        if (error != nullptr) atomicMin(error, QUASAR_ERR_TIMEOUT);
+        return false;
+      }
+    }
+  }
+  return true;
+}
+
+__device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];\n" ::"r"(
+          smem_u32(smem_dst)),
+      "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y)
+      : "memory");
+}
+
+// K-major operand tile with 128-byte swizzle: rows of 128 bytes, groups of 8 rows 1024 bytes apart.
+__device__ __forceinline__ uint64_t umma_desc_sw128(const void* smem_tile) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_u32(smem_tile) & 0x3ffff) >> 4);   // start address, 16-byte units
+  d |= (uint64_t)1 << 16;                                  // leading-dimension offset: unused with this swizzle
+  d |= (uint64_t)(1024 >> 4) << 32;                        // stride between 8-row groups
+  d |= (uint64_t)1 << 46;                                  // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;                                  // 128-byte swizzle
+  return d;
+}
+
+// instruction descriptor: dense, A and B K-major, M = 128, N = n
+__device__ __forceinline__ uint32_t umma_idesc(int c_format, int ab_format, int n) {
+  return ((uint32_t)c_format << 4) | ((uint32_t)ab_format << 7) | ((uint32_t)ab_format << 10) | ((uint32_t)(n >> 3) << 17) |
+         ((uint32_t)(kTileN >> 4) << 24);
+}
+
+template <bool I8>
+__device__ __forceinline__ void umma_ss(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate) {
+  if (I8) {
+    asm volatile(
+        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n}\n" ::"r"(tmem_d),
+        "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+        : "memory");
+  } else {
+    asm volatile(
+        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n" ::"r"(tmem_d),
+        "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+        : "memory");
+  }
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(smem_u32(bar)) : "memory");
+}
+
+// 16 consecutive accumulator columns of this thread's tensor-memory lane
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];\n"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]), "=r"(v[9]),
+        "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+}
+
+template <bool I8>
+__device__ __forceinline__ void store_output(const UmmaArgs& a, uint32_t bits, int m, int n) {
+  const size_t idx = (size_t)m * a.N + n;
+  float v;
+  if (I8) {
+    const int acc = (int)bits;
+    if (a.acc_out != nullptr) a.acc_out[idx] = acc;
+    v = __fmul_rn((float)acc, __fmul_rn(a.dw[n], a.dx[m]));   // Eq. 10
+  } else {
+    v = __uint_as_float(bits) * a.dw[n];
+  }
+  if (a.res != nullptr) v = __bfloat162float(__float2bfloat16_rn(v)) + __bfloat162float(a.res[idx]);
+  if (a.y_is_f32) reinterpret_cast<float*>(a.y)[idx] = v;
+  else reinterpret_cast<__nv_bfloat16*>(a.y)[idx] = __float2bfloat16_rn(v);
+}
+
+// shared memory of the W8A8 kernel: kStagesI8 x (A tile 16 KB + B tile Mpad x 128 B), then barriers
+template <bool I8>
+__global__ void __launch_bounds__(kThreadsU, 1)
+umma_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, UmmaArgs a) {
+  static_assert(I8, "this entry is the int8 x int8 form");
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  // operand tiles start on a 1024-byte boundary (the swizzle pattern repeats every 8 rows of 128 bytes)
+  unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+  const int b_bytes = a.Mpad * kTileKBytes;                        // multiple of 1024 (Mpad is a multiple of 16)
+  const int stage_bytes = kTileN * kTileKBytes + b_bytes;
+  unsigned char* tiles = smem;
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + kStagesI8 * stage_bytes);
+  uint64_t* empty = full + kStagesI8;
+  uint64_t* accum_done = empty + kStagesI8;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(accum_done + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n0 = blockIdx.x * kTileN;
+  const int k_begin = blockIdx.y * a.k_per_split;
+  const int k_end = min(a.K, k_begin + a.k_per_split);
+  const int nkb = (k_end - k_begin + kTileKBytes - 1) / kTileKBytes;
+
+  if (threadIdx.x == 0) {
+    *abort_flag = 0;
+    for (int s = 0; s < kStagesI8; ++s) {
+      mbar_init(full + s, 1);
+      mbar_init(empty + s, 1);
+    }
+    mbar_init(accum_done, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+  }
+  if (warp == 1) {   // 128 columns of tensor memory for the 128 x Mpad accumulator
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(tmem_slot)), "r"(128u)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {   // ---- TMA producer ----
+      int s = 0;
+      uint32_t ph = 0;
+      for (int kb = 0; kb < nkb; ++kb) {
+        if (!mbar_wait(empty + s, ph ^ 1u, abort_flag, a.error)) break;
+        unsigned char* at = tiles + s * stage_bytes;
+        mbar_expect_tx(full + s, (uint32_t)stage_bytes);
+        tma_load_2d(at, &map_w, k_begin + kb * kTileKBytes, n0, full + s);
+        tma_load_2d(at + kTileN * kTileKBytes, &map_x, k_begin + kb * kTileKBytes, 0, full + s);
+        if (++s == kStagesI8) { s = 0; ph ^= 1u; }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {   // ---- MMA issuer ----
+      const uint32_t idesc = umma_idesc(/*s32*/ 2, /*signed int8*/ 1, a.Mpad);
+      int s = 0;
+      uint32_t ph = 0;
+      bool ok = true;
+      for (int kb = 0; kb < nkb && ok; ++kb) {
+        if (!(ok = mbar_wait(full + s, ph, abort_flag, a.error))) break;
+        asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+        const unsigned char* at = tiles + s * stage_bytes;
+        const uint64_t da = umma_desc_sw128(at), db = umma_desc_sw128(at + kTileN * kTileKBytes);
+#pragma unroll
+        for (int j = 0; j < kTileKBytes / 32; ++j)   // one instruction contracts 32 bytes of k: 32 bytes further along the row
+          umma_ss<true>(tmem_base, da + (uint64_t)(j * 2), db + (uint64_t)(j * 2), idesc, (kb > 0 || j > 0) ? 1u : 0u);
+        umma_commit(empty + s);   // arrives when the MMAs above have read the stage
+        if (++s == kStagesI8) { s = 0; ph ^= 1u; }
+      }
+      if (ok) umma_commit(accum_done);
+    }
+  } else {
+    // ---- epilogue: warps 2..5; a warp may touch the tensor-memory lanes 32 (warp % 4) .. + 31 ----
+    const int q = warp & 3;
+    const int n = n0 + q * 32 + lane;
+    int got = 1;
+    if (lane == 0) got = mbar_wait(accum_done, 0, abort_flag, a.error) ? 1 : 0;
+    got = __shfl_sync(0xffffffffu, got, 0);
+    if (got) {
+      asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+      for (int c0 = 0; c0 < a.Mpad; c0 += 16) {
+        uint32_t v[16];
+        tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
+        if (n < a.N) {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const int m = c0 + j;
+            if (m >= a.M) continue;
+            if (a.nsplit == 1) store_output<true>(a, v[j], m, n);
+            else __stcg(reinterpret_cast<uint32_t*>(a.partial) + ((size_t)blockIdx.y * a.Mpad + m) * a.N + n, v[j]);
+          }
+        }
+      }
+    }
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+  __threadfence();
+  __syncthreads();
+  if (warp == 1) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem_base), "r"(128u) : "memory");
+  }
+  if (a.nsplit == 1 || *abort_flag) return;
+  // ---- k-ranges of this channel block: the last CTA to arrive adds them up in a fixed order ----
+  __shared__ int s_last;
+  if (threadIdx.x == 0) s_last = (atomicAdd(a.counters + blockIdx.x, 1) == a.nsplit - 1);
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  for (int i = threadIdx.x; i < kTileN * a.M; i += kThreadsU) {
+    const int n = n0 + (i % kTileN), m = i / kTileN;
+    if (n >= a.N) continue;
+    int sum = 0;
+    for (int s = 0; s < a.nsplit; ++s)
+      sum += (int)__ldcg(reinterpret_cast<const uint32_t*>(a.partial) + ((size_t)s * a.Mpad + m) * a.N + n);
+    store_output<true>(a, (uint32_t)sum, m, n);
+  }
+  if (threadIdx.x == 0) a.counters[blockIdx.x] = 0;
+}
+
+// ---- host side ------------------------------------------------------------------------------------
+PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
+  static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(p);
+  });
+  return fn;
+}
+
+// [rows][row_bytes] bytes, box = box_rows x 128 bytes, 128-byte swizzle, zeros outside
+int make_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t row_bytes, uint32_t box_rows) {
+  auto fn = encode_fn();
+  if (fn == nullptr) {
+    set_error("cuTensorMapEncodeTiled is not available from this driver");
+    return QUASAR_ERR_CUDA;
+  }
+  const cuuint64_t dims[2] = {row_bytes, rows};
+  const cuuint64_t strides[1] = {row_bytes};
+  const cuuint32_t box[2] = {(cuuint32_t)kTileKBytes, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    set_error("cuTensorMapEncodeTiled failed (%d) for %llu x %llu bytes", (int)r, (unsigned long long)rows,
+              (unsigned long long)row_bytes);
+    return QUASAR_ERR_CUDA;
+  }
+  return QUASAR_OK;
+}
+
+struct SplitU {
+  int nblocks, nsplit, k_per_split;
+};
+SplitU plan_split_u(int64_t N, int64_t K) {
+  SplitU p;
+  p.nblocks = (int)((N + kTileN - 1) / kTileN);
+  const int kbs = (int)((K + kTileKBytes - 1) / kTileKBytes);
+  int want = (2 * 148 + p.nblocks - 1) / p.nblocks;   // about two waves of CTAs
+  want = want < 1 ? 1 : (want > kbs ? kbs : want);
+  want = want > 32 ? 32 : want;
+  const int per = (kbs + want - 1) / want;
+  p.k_per_split = per * kTileKBytes;
+  p.nsplit = (kbs + per - 1) / per;
+  return p;
+}
+
+}  // namespace
+
+bool umma_w8a8_usable(int64_t M, int64_t N, int64_t K) {
+  return M > 8 && M <= kMaxMpad && K % 16 == 0 && N >= 1 && (int64_t)((N + kTileN - 1) / kTileN) * 4 <= (int64_t)kCounterBytesU;
+}
+
+size_t umma_w8a8_partial_bytes(int64_t M, int64_t N, int64_t K) {
+  const SplitU p = plan_split_u(N, K);
+  const size_t mpad = (size_t)((M + 15) / 16) * 16;
+  return p.nsplit > 1 ? (size_t)p.nsplit * mpad * (size_t)N * 4 : 0;
+}
+
+// xq: int8 [M][K] quantised activations, dx their step sizes; counters: >= 64 KiB, zero on first use
+int launch_umma_w8a8(const int8_t* xq, const float* dx, const int8_t* w, const float* dw, int64_t M, int64_t N, int64_t K,
+                     void* y, bool y_is_f32, const __nv_bfloat16* residual, int32_t* acc_out, int* counters, void* partial,
+                     int32_t* error_word, cudaStream_t stream) {
+  CUtensorMap map_w, map_x;
+  const int mpad = (int)((M + 15) / 16) * 16;
+  int rc = make_map(&map_w, w, (uint64_t)N, (uint64_t)K, kTileN);
+  if (rc != QUASAR_OK) return rc;
+  rc = make_map(&map_x, xq, (uint64_t)M, (uint64_t)K, (uint32_t)mpad);
+  if (rc != QUASAR_OK) return rc;
+  const SplitU p = plan_split_u(N, K);
+  UmmaArgs a;
+  a.dx = dx; a.dw = dw; a.y = y; a.res = residual; a.acc_out = acc_out; a.partial = partial; a.counters = counters;
+  a.error = error_word;
+  a.M = (int)M; a.Mpad = mpad; a.N = (int)N; a.K = (int)K; a.k_per_split = p.k_per_split; a.nsplit = p.nsplit;
+  a.y_is_f32 = y_is_f32 ? 1 : 0;
+  const size_t smem = (size_t)kStagesI8 * (kTileN * kTileKBytes + mpad * kTileKBytes) + 256 + 1024;
+  static bool configured = false;
+  if (!configured) {
+    QUASAR_CUDA_CHECK(cudaFuncSetAttribute(umma_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+    configured = true;
+  }
+  umma_gemm_kernel<true><<<dim3(p.nblocks, p.nsplit), kThreadsU, smem, stream>>>(map_w, map_x, a);
+  QUASAR_LAUNCH_CHECK();
+  return QUASAR_OK;
+}
+
+}  // namespace quasar

@@ -314,13 +314,18 @@ size_t linear_w8a8_workspace_bytes(int64_t M, int64_t N, int64_t K) {
   const SplitPlan p = plan_split(N, K);
   const int64_t rows = M < kMaxRowsPerGemm ? M : kMaxRowsPerGemm;
   const size_t mpad = (size_t)((rows + 7) / 8) * 8;
-  const size_t partial = p.nsplit > 1 ? (size_t)p.nsplit * mpad * (size_t)N * sizeof(int32_t) : 0;
+  size_t partial = p.nsplit > 1 ? (size_t)p.nsplit * mpad * (size_t)N * sizeof(int32_t) : 0;
+  const int64_t rows_u = M < 80 ? M : 80;
+  if (umma_w8a8_usable(rows_u, N, K)) {
+    const size_t pu = umma_w8a8_partial_bytes(rows_u, N, K);
+    partial = pu > partial ? pu : partial;
+  }
   return kCounterBytes + align256((size_t)M * K) + align256((size_t)M * sizeof(float)) + partial;
 }
 
 int launch_linear_w8a8(const __nv_bfloat16* x, const float* smooth, const int8_t* w, const float* delta_w, int64_t M,
                        int64_t N, int64_t K, void* y, bool y_is_f32, const __nv_bfloat16* residual, int32_t* acc_out,
-                       void* workspace, size_t workspace_bytes, cudaStream_t stream) {
+                       void* workspace, size_t workspace_bytes, int32_t* status, cudaStream_t stream) {
   if (M <= 0 || N <= 0 || K <= 0 || (K % 16) != 0 || N > kMaxChannels || K > 0x7fffffff) {
     set_error("linear_w8a8: unsupported sizes M=%lld N=%lld K=%lld (K must be a multiple of 16, N at most %lld)",
               (long long)M, (long long)N, (long long)K, (long long)kMaxChannels);
@@ -339,6 +344,18 @@ int launch_linear_w8a8(const __nv_bfloat16* x, const float* smooth, const int8_t
   if (rc0 != QUASAR_OK) return rc0;
   const SplitPlan p = plan_split(N, K);
   const size_t ybytes = y_is_f32 ? 4 : 2;
+  if (M > 8 && umma_w8a8_usable(M < 80 ? M : 80, N, K)) {
+    // blocks of more than 8 rows: the contraction runs on tcgen05 with the accumulator in tensor memory
+    for (int64_t m0 = 0; m0 < M; m0 += 80) {
+      const int64_t rows = (M - m0) < 80 ? (M - m0) : 80;
+      const int rc = launch_umma_w8a8(xq + m0 * K, dx + m0, w, delta_w, rows, N, K,
+                                      reinterpret_cast<unsigned char*>(y) + (size_t)m0 * N * ybytes, y_is_f32,
+                                      residual ? residual + m0 * N : nullptr, acc_out ? acc_out + m0 * N : nullptr,
+                                      reinterpret_cast<int*>(workspace), partial, status, stream);
+      if (rc != QUASAR_OK) return rc;
+    }
+    return QUASAR_OK;
+  }
   for (int64_t m0 = 0; m0 < M; m0 += kMaxRowsPerGemm) {
     A8Args a;
     a.M = (int)((M - m0) < kMaxRowsPerGemm ? (M - m0) : kMaxRowsPerGemm);
