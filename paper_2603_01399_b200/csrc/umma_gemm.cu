@@ -16,7 +16,7 @@
 //     weight and one conversion instruction per two weights.
 // Roles: warp 0 issues the TMA loads, warp 1 the MMAs (one elected thread), warps 2-5 convert
 // (W8A16) and run the epilogue (tcgen05.ld, one tensor-memory lane = one output channel per
-// thread).  k-ranges of one channel block are reduced in a fixed order by the last CTA to arrive.
+// thread).  k-ranges of one channel block are added up in a fixed order by a second, fully parallel kernel.
 //
 // Every wait is bounded (2 s): on expiry the CTA raises an error word, stops waiting everywhere,
 // releases its tensor memory and returns.
@@ -33,7 +33,7 @@ namespace {
 
 constexpr int kTileN = 128;          // output channels per CTA (MMA M)
 constexpr int kTileKBytes = 128;     // contraction bytes of int8 per stage (one 128-byte swizzle row)
-constexpr int kStagesI8 = 6;
+constexpr int kStagesI8 = 4;         // two CTAs share an SM: one's epilogue overlaps the other's stream
 constexpr int kThreadsU = 192;
 constexpr int kMaxMpad = 80;
 constexpr unsigned long long kBudgetNs = 2000000000ull;
@@ -165,7 +165,7 @@ __device__ __forceinline__ void store_output(const UmmaArgs& a, uint32_t bits, i
 
 // shared memory of the W8A8 kernel: kStagesI8 x (A tile 16 KB + B tile Mpad x 128 B), then barriers
 template <bool I8>
-__global__ void __launch_bounds__(kThreadsU, 1)
+__global__ void __launch_bounds__(kThreadsU, 2)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, UmmaArgs a) {
   static_assert(I8, "this entry is the int8 x int8 form");
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -267,22 +267,51 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
   if (warp == 1) {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem_base), "r"(128u) : "memory");
   }
-  if (a.nsplit == 1 || *abort_flag) return;
-  // ---- k-ranges of this channel block: the last CTA to arrive adds them up in a fixed order ----
-  __shared__ int s_last;
-  if (threadIdx.x == 0) s_last = (atomicAdd(a.counters + blockIdx.x, 1) == a.nsplit - 1);
-  __syncthreads();
-  if (!s_last) return;
-  __threadfence();
-  for (int i = threadIdx.x; i < kTileN * a.M; i += kThreadsU) {
-    const int n = n0 + (i % kTileN), m = i / kTileN;
-    if (n >= a.N) continue;
-    int sum = 0;
-    for (int s = 0; s < a.nsplit; ++s)
-      sum += (int)__ldcg(reinterpret_cast<const uint32_t*>(a.partial) + ((size_t)s * a.Mpad + m) * a.N + n);
-    store_output<true>(a, (uint32_t)sum, m, n);
+}
+
+// k-ranges of a channel block meet here: a second, fully parallel kernel adds the partial sums in a fixed
+// order (split 0, 1, ...) and applies the epilogue.  One thread per activation row and four channels.
+template <bool I8>
+__global__ void __launch_bounds__(256) umma_reduce_kernel(UmmaArgs a) {
+  const int n4 = (a.N + 3) / 4;
+  const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  if (i >= (int64_t)a.M * n4) return;
+  const int m = (int)(i / n4), n = (int)(i % n4) * 4;
+  const uint32_t* p0 = reinterpret_cast<const uint32_t*>(a.partial) + (size_t)m * a.N + n;
+  const size_t split_stride = (size_t)a.Mpad * a.N;
+  if (n + 4 <= a.N && (a.N & 3) == 0) {
+    uint4 v[8];
+    int ai[4] = {0, 0, 0, 0};
+    float af[4] = {0.f, 0.f, 0.f, 0.f};
+    for (int s0 = 0; s0 < a.nsplit; s0 += 8) {
+      const int cnt = min(8, a.nsplit - s0);
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        if (j < cnt) v[j] = __ldcg(reinterpret_cast<const uint4*>(p0 + (size_t)(s0 + j) * split_stride));
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        if (j >= cnt) continue;
+        const uint32_t w[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          if (I8) ai[e] += (int)w[e];
+          else af[e] += __uint_as_float(w[e]);
+        }
+      }
+    }
+#pragma unroll
+    for (int e = 0; e < 4; ++e) store_output<I8>(a, I8 ? (uint32_t)ai[e] : __float_as_uint(af[e]), m, n + e);
+  } else {
+    for (int e = 0; e < 4 && n + e < a.N; ++e) {
+      int si = 0;
+      float sf = 0.f;
+      for (int s = 0; s < a.nsplit; ++s) {
+        const uint32_t w = __ldcg(p0 + e + (size_t)s * split_stride);
+        if (I8) si += (int)w; else sf += __uint_as_float(w);
+      }
+      store_output<I8>(a, I8 ? (uint32_t)si : __float_as_uint(sf), m, n + e);
+    }
   }
-  if (threadIdx.x == 0) a.counters[blockIdx.x] = 0;
 }
 
 // ---- host side ------------------------------------------------------------------------------------
@@ -328,7 +357,7 @@ SplitU plan_split_u(int64_t N, int64_t K) {
   SplitU p;
   p.nblocks = (int)((N + kTileN - 1) / kTileN);
   const int kbs = (int)((K + kTileKBytes - 1) / kTileKBytes);
-  int want = (2 * 148 + p.nblocks - 1) / p.nblocks;   // about two waves of CTAs
+  int want = 148 / p.nblocks;                          // about one wave of CTAs; no split once the channel blocks fill the SMs
   want = want < 1 ? 1 : (want > kbs ? kbs : want);
   want = want > 32 ? 32 : want;
   const int per = (kbs + want - 1) / want;
@@ -368,11 +397,16 @@ int launch_umma_w8a8(const int8_t* xq, const float* dx, const int8_t* w, const f
   const size_t smem = (size_t)kStagesI8 * (kTileN * kTileKBytes + mpad * kTileKBytes) + 256 + 1024;
   static bool configured = false;
   if (!configured) {
-    QUASAR_CUDA_CHECK(cudaFuncSetAttribute(umma_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+    QUASAR_CUDA_CHECK(cudaFuncSetAttribute(umma_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 112 * 1024));
     configured = true;
   }
   umma_gemm_kernel<true><<<dim3(p.nblocks, p.nsplit), kThreadsU, smem, stream>>>(map_w, map_x, a);
   QUASAR_LAUNCH_CHECK();
+  if (p.nsplit > 1) {
+    const int64_t items = M * ((N + 3) / 4);
+    umma_reduce_kernel<true><<<(unsigned)((items + 255) / 256), 256, 0, stream>>>(a);
+    QUASAR_LAUNCH_CHECK();
+  }
   return QUASAR_OK;
 }
 
