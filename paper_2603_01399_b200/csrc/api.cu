@@ -249,7 +249,7 @@ int verify_impl(quasar_model* m, const quasar_kv* kv, const int32_t* tokens, con
     if (a8)
       return launch_linear_w8a8(in, smooth, reinterpret_cast<const int8_t*>(w), delta, M, N, K, out, out_f32, res, nullptr,
                                 lin, ws.lin_bytes, status, stream);
-    return launch_linear(in, w, delta, wd, M, N, K, out, out_f32, res, lin, ws.lin_bytes, stream);
+    return launch_linear(in, w, delta, wd, M, N, K, out, out_f32, res, lin, ws.lin_bytes, stream, status);
   };
   const size_t layer_stride = (size_t)kv->batch * Hkv * (size_t)kv->s_max * D;
   TraceCursor tr{reinterpret_cast<unsigned char*>(m->trace_buf), 0, m->trace_bytes, stream};

@@ -42,7 +42,7 @@ int launch_quantize(const __nv_bfloat16* w, int64_t N, int64_t K, int8_t* q, flo
 size_t linear_workspace_bytes(int64_t M, int64_t N, int64_t K);
 int launch_linear(const __nv_bfloat16* x, const void* w, const float* delta, int weight_dtype, int64_t M, int64_t N,
                   int64_t K, void* y, bool y_is_f32, const __nv_bfloat16* residual, void* workspace,
-                  size_t workspace_bytes, cudaStream_t stream);
+                  size_t workspace_bytes, cudaStream_t stream, int32_t* status = nullptr);
 
 // The same launch with the split-K scratch taken from a fixed array inside the library.
 size_t linear_static_scratch_bytes();
@@ -67,6 +67,11 @@ size_t umma_w8a8_partial_bytes(int64_t M, int64_t N, int64_t K);
 int launch_umma_w8a8(const int8_t* xq, const float* dx, const int8_t* w, const float* dw, int64_t M, int64_t N, int64_t K,
                      void* y, bool y_is_f32, const __nv_bfloat16* residual, int32_t* acc_out, int* counters, void* partial,
                      int32_t* error_word, cudaStream_t stream);
+
+bool umma_w8a16_usable(int64_t M, int64_t N, int64_t K);
+size_t umma_w8a16_scratch_bytes(int64_t M, int64_t N, int64_t K);
+int launch_umma_w8a16(const __nv_bfloat16* x, const int8_t* w, const float* dw, int64_t M, int64_t N, int64_t K, void* y,
+                      bool y_is_f32, const __nv_bfloat16* residual, void* scratch, int32_t* error_word, cudaStream_t stream);
 
 // Per-call description of the draft blocks, derived on the device from tokens / parents / block_len.
 struct BlockInfo {

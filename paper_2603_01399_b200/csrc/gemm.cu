@@ -298,13 +298,20 @@ size_t linear_workspace_bytes(int64_t M, int64_t N, int64_t K) {
   const int64_t rows = M < kMaxRowsPerGemm ? M : kMaxRowsPerGemm;
   const size_t mpad = (size_t)((rows + 7) / 8) * 8;
   const size_t counters = kCounterBytes;
-  const size_t partial = p.nsplit > 1 ? (size_t)p.nsplit * mpad * (size_t)N * sizeof(float) : 0;
+  size_t partial = p.nsplit > 1 ? (size_t)p.nsplit * mpad * (size_t)N * sizeof(float) : 0;
+  // blocks of more than 8 rows with int8 weights run on the tcgen05 kernel, which keeps an fp16 copy of the
+  // activation rows and its own partial sums here
+  const int64_t rows_u = M < 80 ? M : 80;
+  if (M > 8 && umma_w8a16_usable(rows_u, N, K)) {
+    const size_t su = umma_w8a16_scratch_bytes(rows_u, N, K);
+    partial = su > partial ? su : partial;
+  }
   return counters + partial;
 }
 
 int launch_linear(const __nv_bfloat16* x, const void* w, const float* delta, int weight_dtype, int64_t M, int64_t N,
                   int64_t K, void* y, bool y_is_f32, const __nv_bfloat16* residual, void* workspace,
-                  size_t workspace_bytes, cudaStream_t stream) {
+                  size_t workspace_bytes, cudaStream_t stream, int32_t* status) {
   if (M <= 0 || N <= 0 || K <= 0 || (K % 16) != 0 || N > kMaxChannels || K > 0x7fffffff) {
     set_error("linear: unsupported sizes M=%lld N=%lld K=%lld (K must be a multiple of 16, N at most %lld)",
               (long long)M, (long long)N, (long long)K, (long long)kMaxChannels);
@@ -317,6 +324,18 @@ int launch_linear(const __nv_bfloat16* x, const void* w, const float* delta, int
   const SplitPlan p = plan_split(N, K);
   const size_t counters = kCounterBytes;
   const size_t ybytes = y_is_f32 ? 4 : 2;
+  if (weight_dtype == QUASAR_W_INT8 && M > 8 && umma_w8a16_usable(M < 80 ? M : 80, N, K)) {
+    // a real dense contraction: tcgen05 MMAs with the accumulator in tensor memory (umma_gemm.cu)
+    for (int64_t m0 = 0; m0 < M; m0 += 80) {
+      const int64_t rows = (M - m0) < 80 ? (M - m0) : 80;
+      const int rc = launch_umma_w8a16(x + m0 * K, reinterpret_cast<const int8_t*>(w), delta, rows, N, K,
+                                       reinterpret_cast<unsigned char*>(y) + (size_t)m0 * N * ybytes, y_is_f32,
+                                       residual ? residual + m0 * N : nullptr,
+                                       reinterpret_cast<unsigned char*>(workspace) + counters, status, stream);
+      if (rc != QUASAR_OK) return rc;
+    }
+    return QUASAR_OK;
+  }
   for (int64_t m0 = 0; m0 < M; m0 += kMaxRowsPerGemm) {
     GemmArgs a;
     a.M = (int)((M - m0) < kMaxRowsPerGemm ? (M - m0) : kMaxRowsPerGemm);
@@ -384,7 +403,7 @@ int launch_linear_static(const __nv_bfloat16* x, const void* w, const float* del
   }
   // The arrival counters must start at zero; the array keeps whatever the last call left in it.
   QUASAR_CUDA_CHECK(cudaMemsetAsync(scratch, 0, kCounterBytes, stream));
-  return launch_linear(x, w, delta, weight_dtype, M, N, K, y, y_is_f32, residual, scratch, kStaticScratchBytes, stream);
+  return launch_linear(x, w, delta, weight_dtype, M, N, K, y, y_is_f32, residual, scratch, kStaticScratchBytes, stream, nullptr);
 }
 
 }  // namespace quasar

@@ -156,7 +156,7 @@ __device__ __forceinline__ void store_output(const UmmaArgs& a, uint32_t bits, i
     if (a.acc_out != nullptr) a.acc_out[idx] = acc;
     v = __fmul_rn((float)acc, __fmul_rn(a.dw[n], a.dx[m]));   // Eq. 10
   } else {
-    v = __uint_as_float(bits) * a.dw[n];
+    v = (__uint_as_float(bits) * a.dx[m]) * a.dw[n];   // the row's power-of-two scale back out (exact), then the step size
   }
   if (a.res != nullptr) v = __bfloat162float(__float2bfloat16_rn(v)) + __bfloat162float(a.res[idx]);
   if (a.y_is_f32) reinterpret_cast<float*>(a.y)[idx] = v;
@@ -314,6 +314,188 @@ __global__ void __launch_bounds__(256) umma_reduce_kernel(UmmaArgs a) {
   }
 }
 
+// ---- the weight-only form (int8 weights, 16-bit activations) on the same tensor cores -------------------
+// kind::f16 takes both operands as fp16.  The activations are turned into fp16 once per call by a
+// small pre-pass (exact: a bf16 value times a power of two that puts the row's maximum in [2^14, 2^15) is
+// an fp16 value unless it lies 2^-39 below that maximum), the weights per stage by four converter warps:
+// a stage's 128 rows x 64 contraction bytes land by TMA (64-byte swizzle), thread r turns row r into 64
+// fp16 values - the byte with its sign bit flipped under the high byte 0x64 reads 1024 + (w + 128), one
+// packed subtraction of 1152 leaves w - and stores them as row r of a K-major tile with the 128-byte
+// swizzle the MMA expects.  Per stage: raw weights 8 KB, fp16 weights 16 KB, activations Mpad x 128 B.
+constexpr int kStagesF16 = 3;
+constexpr int kRawBytes = kTileN * 64;          // 8 KB
+constexpr int kConvBytes = kTileN * 128;        // 16 KB
+
+__device__ __forceinline__ void s8x4_to_f16x4(uint32_t w, uint32_t& lo, uint32_t& hi) {
+  const uint32_t u = w ^ 0x80808080u;
+  const uint32_t l = __byte_perm(u, 0x64646464u, 0x4140);
+  const uint32_t h = __byte_perm(u, 0x64646464u, 0x4342);
+  const __half2 bias = __halves2half2(__ushort_as_half(0x6480), __ushort_as_half(0x6480));   // 1152
+  const __half2 lo2 = __hsub2(*reinterpret_cast<const __half2*>(&l), bias);
+  const __half2 hi2 = __hsub2(*reinterpret_cast<const __half2*>(&h), bias);
+  lo = *reinterpret_cast<const uint32_t*>(&lo2);
+  hi = *reinterpret_cast<const uint32_t*>(&hi2);
+}
+
+__global__ void __launch_bounds__(kThreadsU, 2)
+umma_w8a16_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, UmmaArgs a) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+  const int b_bytes = a.Mpad * 128;                               // Mpad rows x 64 fp16
+  const int stage_bytes = kConvBytes + b_bytes + kRawBytes;       // [fp16 weights][activations][raw weights]
+  unsigned char* tiles = smem;
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + kStagesF16 * stage_bytes);   // TMA landed (raw weights + activations)
+  uint64_t* conv = full + kStagesF16;                                              // fp16 weight tile written
+  uint64_t* empty = conv + kStagesF16;                                             // MMAs of the stage done
+  uint64_t* accum_done = empty + kStagesF16;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(accum_done + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n0 = blockIdx.x * kTileN;
+  const int k_begin = blockIdx.y * a.k_per_split;
+  const int k_end = min(a.K, k_begin + a.k_per_split);
+  const int nkb = (k_end - k_begin + 63) / 64;
+
+  if (threadIdx.x == 0) {
+    *abort_flag = 0;
+    for (int s = 0; s < kStagesF16; ++s) {
+      mbar_init(full + s, 1);
+      mbar_init(conv + s, 4);     // one arrival per converter warp
+      mbar_init(empty + s, 1);
+    }
+    mbar_init(accum_done, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(tmem_slot)), "r"(128u)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {   // ---- TMA producer ----
+      int s = 0;
+      uint32_t ph = 0;
+      for (int kb = 0; kb < nkb; ++kb) {
+        if (!mbar_wait(empty + s, ph ^ 1u, abort_flag, a.error)) break;
+        unsigned char* st = tiles + s * stage_bytes;
+        mbar_expect_tx(full + s, (uint32_t)(kRawBytes + b_bytes));
+        tma_load_2d(st + kConvBytes + b_bytes, &map_w, k_begin + kb * 64, n0, full + s);          // 128 rows x 64 int8
+        tma_load_2d(st + kConvBytes, &map_x, (k_begin + kb * 64) * 2, 0, full + s);               // Mpad rows x 64 fp16 (byte coordinate)
+        if (++s == kStagesF16) { s = 0; ph ^= 1u; }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {   // ---- MMA issuer ----
+      const uint32_t idesc = umma_idesc(/*f32*/ 1, /*fp16*/ 0, a.Mpad);
+      int s = 0;
+      uint32_t ph = 0;
+      bool ok = true;
+      for (int kb = 0; kb < nkb && ok; ++kb) {
+        if (!(ok = mbar_wait(conv + s, ph, abort_flag, a.error))) break;    // (the converters waited for the stage's TMA)
+        asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+        const unsigned char* st = tiles + s * stage_bytes;
+        const uint64_t da = umma_desc_sw128(st), db = umma_desc_sw128(st + kConvBytes);
+#pragma unroll
+        for (int j = 0; j < 4; ++j)   // one instruction contracts 16 fp16 values: 32 bytes further along the row
+          umma_ss<false>(tmem_base, da + (uint64_t)(j * 2), db + (uint64_t)(j * 2), idesc, (kb > 0 || j > 0) ? 1u : 0u);
+        umma_commit(empty + s);
+        if (++s == kStagesF16) { s = 0; ph ^= 1u; }
+      }
+      if (ok) umma_commit(accum_done);
+    }
+  } else {
+    // ---- converters, then the epilogue: warps 2..5, thread r = weight row r of the tile ----
+    const int r = (warp - 2) * 32 + lane;
+    int s = 0;
+    uint32_t ph = 0;
+    bool ok = true;
+    for (int kb = 0; kb < nkb; ++kb) {
+      int got = 1;
+      if (lane == 0) got = mbar_wait(full + s, ph, abort_flag, a.error) ? 1 : 0;
+      got = __shfl_sync(0xffffffffu, got, 0);
+      if (!got) { ok = false; break; }
+      unsigned char* st = tiles + s * stage_bytes;
+      const unsigned char* raw = st + kConvBytes + b_bytes + r * 64;          // 64-byte swizzle: piece c sits at c ^ ((r >> 1) & 3)
+      unsigned char* dst = st + (r >> 3) * 1024 + (r & 7) * 128;              // 128-byte swizzle: piece c sits at c ^ (r & 7)
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        const uint4 w = *reinterpret_cast<const uint4*>(raw + ((c ^ ((r >> 1) & 3)) << 4));
+        uint4 o0, o1;
+        s8x4_to_f16x4(w.x, o0.x, o0.y);
+        s8x4_to_f16x4(w.y, o0.z, o0.w);
+        s8x4_to_f16x4(w.z, o1.x, o1.y);
+        s8x4_to_f16x4(w.w, o1.z, o1.w);
+        *reinterpret_cast<uint4*>(dst + (((2 * c) ^ (r & 7)) << 4)) = o0;
+        *reinterpret_cast<uint4*>(dst + (((2 * c + 1) ^ (r & 7)) << 4)) = o1;
+      }
+      asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");   // the tensor core reads what these threads wrote
+      __syncwarp();
+      if (lane == 0) mbar_arrive(conv + s);
+      if (++s == kStagesF16) { s = 0; ph ^= 1u; }
+    }
+    const int q = warp & 3;
+    const int n = n0 + q * 32 + lane;
+    int got = ok ? 1 : 0;
+    if (ok && lane == 0) got = mbar_wait(accum_done, 0, abort_flag, a.error) ? 1 : 0;
+    got = __shfl_sync(0xffffffffu, got, 0);
+    if (got) {
+      asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+      for (int c0 = 0; c0 < a.Mpad; c0 += 16) {
+        uint32_t v[16];
+        tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
+        if (n < a.N) {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const int m = c0 + j;
+            if (m >= a.M) continue;
+            if (a.nsplit == 1) store_output<false>(a, v[j], m, n);
+            else __stcg(reinterpret_cast<uint32_t*>(a.partial) + ((size_t)blockIdx.y * a.Mpad + m) * a.N + n, v[j]);
+          }
+        }
+      }
+    }
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+  __threadfence();
+  __syncthreads();
+  if (warp == 1) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem_base), "r"(128u) : "memory");
+  }
+}
+
+// The activation pre-pass of the weight-only form: bf16 row -> fp16 row times a power of two, and the inverse
+// of that power for the epilogue.  One CTA per row.
+__global__ void __launch_bounds__(256) f16_rows_kernel(const __nv_bfloat16* __restrict__ x, int64_t K, __half* __restrict__ x16,
+                                                       float* __restrict__ inv_scale) {
+  const int64_t m = blockIdx.x;
+  const __nv_bfloat16* row = x + m * K;
+  float amax = 0.f;
+  for (int64_t k = threadIdx.x; k < K; k += 256) amax = fmaxf(amax, fabsf(__bfloat162float(row[k])));
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+  __shared__ float s_max[8];
+  if ((threadIdx.x & 31) == 0) s_max[threadIdx.x >> 5] = amax;
+  __syncthreads();
+  amax = s_max[0];
+#pragma unroll
+  for (int i = 1; i < 8; ++i) amax = fmaxf(amax, s_max[i]);
+  float scale = 1.f, inv = 1.f;
+  if (amax > 0.f && amax < 3.0e38f) {
+    int e;
+    (void)frexpf(amax, &e);            // amax = f * 2^e, f in [0.5, 1)
+    scale = ldexpf(1.f, 15 - e);       // scaled maximum in [2^14, 2^15)
+    inv = ldexpf(1.f, e - 15);
+  }
+  if (threadIdx.x == 0) inv_scale[m] = inv;
+  for (int64_t k = threadIdx.x; k < K; k += 256) x16[m * K + k] = __float2half_rn(__bfloat162float(row[k]) * scale);
+}
+
 // ---- host side ------------------------------------------------------------------------------------
 PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
   static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
@@ -328,8 +510,10 @@ PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
   return fn;
 }
 
-// [rows][row_bytes] bytes, box = box_rows x 128 bytes, 128-byte swizzle, zeros outside
-int make_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t row_bytes, uint32_t box_rows) {
+// [rows][row_bytes] bytes, box = box_rows x box_bytes (128 with the 128-byte swizzle, 64 with the 64-byte one),
+// zeros outside
+int make_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t row_bytes, uint32_t box_rows,
+             uint32_t box_bytes = kTileKBytes) {
   auto fn = encode_fn();
   if (fn == nullptr) {
     set_error("cuTensorMapEncodeTiled is not available from this driver");
@@ -337,10 +521,11 @@ int make_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t row_byt
   }
   const cuuint64_t dims[2] = {row_bytes, rows};
   const cuuint64_t strides[1] = {row_bytes};
-  const cuuint32_t box[2] = {(cuuint32_t)kTileKBytes, box_rows};
+  const cuuint32_t box[2] = {(cuuint32_t)box_bytes, box_rows};
   const cuuint32_t estr[2] = {1, 1};
   const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
-                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, box_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) {
     set_error("cuTensorMapEncodeTiled failed (%d) for %llu x %llu bytes", (int)r, (unsigned long long)rows,
@@ -405,6 +590,56 @@ int launch_umma_w8a8(const int8_t* xq, const float* dx, const int8_t* w, const f
   if (p.nsplit > 1) {
     const int64_t items = M * ((N + 3) / 4);
     umma_reduce_kernel<true><<<(unsigned)((items + 255) / 256), 256, 0, stream>>>(a);
+    QUASAR_LAUNCH_CHECK();
+  }
+  return QUASAR_OK;
+}
+
+
+// ---- weight-only form ----
+bool umma_w8a16_usable(int64_t M, int64_t N, int64_t K) {
+  return M > 8 && M <= kMaxMpad && K % 16 == 0 && N >= 1;
+}
+
+// bytes of scratch: fp16 copy of the activation rows, their inverse scales, partial sums of the k-ranges
+size_t umma_w8a16_scratch_bytes(int64_t M, int64_t N, int64_t K) {
+  const SplitU p = plan_split_u(N, K);
+  const size_t mpad = (size_t)((M + 15) / 16) * 16;
+  const size_t partial = p.nsplit > 1 ? (size_t)p.nsplit * mpad * (size_t)N * 4 : 0;
+  return ((size_t)M * K * 2 + 255) / 256 * 256 + ((size_t)M * 4 + 255) / 256 * 256 + partial;
+}
+
+int launch_umma_w8a16(const __nv_bfloat16* x, const int8_t* w, const float* dw, int64_t M, int64_t N, int64_t K, void* y,
+                      bool y_is_f32, const __nv_bfloat16* residual, void* scratch, int32_t* error_word, cudaStream_t stream) {
+  unsigned char* sc = reinterpret_cast<unsigned char*>(scratch);
+  __half* x16 = reinterpret_cast<__half*>(sc);
+  float* inv = reinterpret_cast<float*>(sc + ((size_t)M * K * 2 + 255) / 256 * 256);
+  void* partial = sc + ((size_t)M * K * 2 + 255) / 256 * 256 + ((size_t)M * 4 + 255) / 256 * 256;
+  f16_rows_kernel<<<(unsigned)M, 256, 0, stream>>>(x, K, x16, inv);
+  QUASAR_LAUNCH_CHECK();
+  CUtensorMap map_w, map_x;
+  const int mpad = (int)((M + 15) / 16) * 16;
+  int rc = make_map(&map_w, w, (uint64_t)N, (uint64_t)K, kTileN, 64);
+  if (rc != QUASAR_OK) return rc;
+  rc = make_map(&map_x, x16, (uint64_t)M, (uint64_t)K * 2, (uint32_t)mpad, 128);
+  if (rc != QUASAR_OK) return rc;
+  const SplitU p = plan_split_u(N, K);
+  UmmaArgs a;
+  a.dx = inv; a.dw = dw; a.y = y; a.res = residual; a.acc_out = nullptr; a.partial = partial; a.counters = nullptr;
+  a.error = error_word;
+  a.M = (int)M; a.Mpad = mpad; a.N = (int)N; a.K = (int)K; a.k_per_split = p.k_per_split; a.nsplit = p.nsplit;
+  a.y_is_f32 = y_is_f32 ? 1 : 0;
+  const size_t smem = (size_t)kStagesF16 * (kConvBytes + mpad * 128 + kRawBytes) + 256 + 1024;
+  static bool configured = false;
+  if (!configured) {
+    QUASAR_CUDA_CHECK(cudaFuncSetAttribute(umma_w8a16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 112 * 1024));
+    configured = true;
+  }
+  umma_w8a16_kernel<<<dim3(p.nblocks, p.nsplit), kThreadsU, smem, stream>>>(map_w, map_x, a);
+  QUASAR_LAUNCH_CHECK();
+  if (p.nsplit > 1) {
+    const int64_t items = M * ((N + 3) / 4);
+    umma_reduce_kernel<false><<<(unsigned)((items + 255) / 256), 256, 0, stream>>>(a);
     QUASAR_LAUNCH_CHECK();
   }
   return QUASAR_OK;
