@@ -457,3 +457,58 @@ def kv_commit(kv: KVCache, accept_len: np.ndarray, accept_path: Optional[np.ndar
                     kv.k_bits[:, b, :, P + d, :] = kv.k_bits[:, b, :, P + j, :]
                     kv.v_bits[:, b, :, P + d, :] = kv.v_bits[:, b, :, P + j, :]
         kv.seq_len[b] = P + 1 + n
+
+
+# --------------------------------------------------------------------------
+# Stochastic acceptance (Section 3.1 Eq. 2-3; Section 3.3 "Lossless Rejection Sampling")
+# --------------------------------------------------------------------------
+# Readings where the paper is silent: the target distribution is softmax(logits / T) of the row that
+# predicts the drafted token; when every draft is accepted one more token is drawn from the target
+# distribution of the last row (the usual completion of the scheme; the paper stops at "concludes the
+# current decoding step"); a draft distribution that is not given is the point mass on the drafted token
+# (a retrieval drafter such as the paper's n-gram lookup proposes one token with certainty); random
+# numbers are INPUTS (r_accept per draft position, r_sample per sequence, all in [0, 1)); a token is drawn
+# from unnormalised weights w by inversion: the smallest v with w_0 + ... + w_v > r_sample * sum(w).
+
+
+def softmax_t(logits_row: np.ndarray, temperature: float) -> np.ndarray:
+    z = np.asarray(logits_row, dtype=np.float64) / float(temperature)
+    z = z - np.max(z)
+    e = np.exp(z)
+    return e / np.sum(e)
+
+
+def sample_by_inversion(weights: np.ndarray, u: float) -> int:
+    """Smallest index v with w_0 + ... + w_v > u * sum(w) (so w_v > 0); if u is so close to 1 that rounding
+    leaves none, the last index with a positive weight."""
+    w = np.asarray(weights, dtype=np.float64)
+    c = np.cumsum(w)
+    v = int(np.searchsorted(c, u * c[-1], side="right"))
+    if v >= len(w):
+        v = int(np.nonzero(w > 0)[0][-1])
+    return v
+
+
+def accept_stochastic(logits: np.ndarray, tokens: List[int], q_probs: Optional[np.ndarray], temperature: float,
+                      r_accept: np.ndarray, r_sample: float):
+    """Chain block.  logits: [T][V] (row i predicts the token after block row i); tokens: T block tokens
+    (row 0 the last emitted token, rows 1.. the drafts); q_probs: [T][V] draft distributions (row i the
+    one draft i+1 was drawn from) or None.  Returns (accept_len, next_token)."""
+    t = len(tokens)
+    n = 0
+    for i in range(t - 1):                                   # draft i+1 against row i (Eq. 2)
+        p = softmax_t(logits[i], temperature)
+        tok = int(tokens[i + 1])
+        q_tok = 1.0 if q_probs is None else float(q_probs[i][tok])
+        ratio = 1.0 if q_tok <= 0 else min(1.0, p[tok] / q_tok)
+        if q_tok <= 0 or not (float(r_accept[i]) < ratio):
+            if q_probs is None:
+                resid = p.copy()
+                resid[tok] = 0.0                             # max(0, p - q) with q the point mass on tok
+            else:
+                resid = np.maximum(0.0, p - np.asarray(q_probs[i], dtype=np.float64))   # Eq. 3
+            if resid.sum() <= 0:                             # p == q exactly: nothing left to correct with
+                resid = p
+            return n, sample_by_inversion(resid, r_sample)
+        n += 1
+    return n, sample_by_inversion(softmax_t(logits[t - 1], temperature), r_sample)
