@@ -258,6 +258,28 @@ int quasar_verify(quasar_model* m, const quasar_kv* kv /* host struct */, const 
                   size_t workspace_bytes, int32_t* status, void* stream);
 
 /* ------------------------------------------------------------------------
+ * Stochastic acceptance of drafted CHAINS (Section 3.1 Eq. 2-3; Section 3.3 "Lossless Rejection
+ * Sampling"), applied to the logits quasar_verify wrote.  With p = softmax(logits / temperature):
+ * draft i+1 (block row i+1) is accepted while r_accept[b][i] < min(1, p_i(token) / q_i(token))
+ * (Eq. 2); at the first rejection next_token is drawn from norm(max(0, p_i - q_i)) (Eq. 3); if all
+ * drafts are accepted it is drawn from p of the last row.  A draw is by inversion with r_sample[b]:
+ * the smallest v with w_0 + ... + w_v > r_sample * sum(w).
+ * logits fp32 [B][T_max][V]; tokens, block_len as in quasar_verify; q_probs fp32 [B][T_max][V] (row i:
+ * the distribution draft i+1 came from) or NULL for a drafter that proposes its token with
+ * certainty (q = point mass: accepted with probability p(token), residual = p without that token);
+ * temperature > 0; r_accept fp32 [B][T_max] and r_sample fp32 [B], uniform in [0, 1), supplied by
+ * the caller; accept_len, next_token int32 [B].  fp32 arithmetic with fixed reduction orders (bit
+ * for bit repeatable); a decision that sits within rounding of its threshold may differ from an
+ * fp64 evaluation.  workspace: quasar_accept_stochastic_workspace_bytes(B, T_max) bytes.
+ * quasar_kv_commit takes the resulting accept_len like the greedy one.
+ * ---------------------------------------------------------------------- */
+int quasar_accept_stochastic_workspace_bytes(int32_t B, int32_t T_max, size_t* bytes_out /* host */);
+int quasar_accept_stochastic(const float* logits, const int32_t* tokens, const int32_t* block_len, const float* q_probs,
+                             int32_t B, int32_t T_max, int32_t V, float temperature, const float* r_accept,
+                             const float* r_sample, int32_t* accept_len, int32_t* next_token, void* workspace,
+                             size_t workspace_bytes, void* stream);
+
+/* ------------------------------------------------------------------------
  * Commit the accepted tokens (the cache reuse Section 3.1 implies between
  * iterations).  Chain (accept_path NULL): seq_len[b] += 1 + accept_len[b].
  * Tree: K,V of the accepted row at depth d move to slot seq_len[b] + d for

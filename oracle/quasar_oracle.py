@@ -512,3 +512,26 @@ def accept_stochastic(logits: np.ndarray, tokens: List[int], q_probs: Optional[n
             return n, sample_by_inversion(resid, r_sample)
         n += 1
     return n, sample_by_inversion(softmax_t(logits[t - 1], temperature), r_sample)
+
+
+# --------------------------------------------------------------------------
+# Drafting by prompt lookup (Section 4.1: the n-gram drafter of all experiments; lookup range
+# K = (K_min, K_max), Section 4.4 / Table 3)
+# --------------------------------------------------------------------------
+# The paper names the method and its two parameters only.  Reading: for n = K_max down to K_min the last n
+# tokens of the sequence are searched for in the tokens before them; the most recent earlier occurrence
+# that is followed by at least one token wins, and the up to gamma tokens that followed it are the draft;
+# the longest n that has such an occurrence is used; no occurrence for any n -> no draft.
+
+
+def ngram_draft(history: List[int], gamma: int, k_min: int, k_max: int) -> List[int]:
+    h = [int(t) for t in history]
+    n_hist = len(h)
+    for n in range(min(k_max, n_hist - 1), k_min - 1, -1):
+        if n < 1:
+            break
+        pattern = h[n_hist - n:]
+        for start in range(n_hist - n - 1, -1, -1):          # most recent first; start + n <= n_hist - 1
+            if h[start:start + n] == pattern:
+                return h[start + n:start + n + gamma]
+    return []

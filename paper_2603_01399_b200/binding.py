@@ -75,6 +75,8 @@ SIGNATURES = {
     "quasar_model_destroy": (C.c_int, [_vp]),
     "quasar_workspace_bytes": (C.c_int, [_vp, _i32, _i32, C.POINTER(_sz)]),
     "quasar_verify": (C.c_int, _verify_args + [_vp]),
+    "quasar_accept_stochastic_workspace_bytes": (C.c_int, [_i32, _i32, C.POINTER(_sz)]),
+    "quasar_accept_stochastic": (C.c_int, [_vp, _vp, _vp, _vp, _i32, _i32, _i32, C.c_float, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "quasar_kv_commit": (C.c_int, [_vp, C.POINTER(KV), _vp, _vp, _i32, _i32, _vp]),
     "quasar_plan_create": (C.c_int, _verify_args + [C.POINTER(_vp)]),
     "quasar_plan_launch": (C.c_int, [_vp, _vp]),
@@ -373,6 +375,22 @@ def quasar_verify(model: Model, kv: KVCache, buf: VerifyBuffers) -> None:
 def quasar_kv_commit(model: Model, kv: KVCache, buf: VerifyBuffers, tree: bool = False) -> None:
     _check(lib().quasar_kv_commit(model.handle, C.byref(kv.c), _ptr(buf.accept_len),
                                   _ptr(buf.accept_path) if tree else None, buf.batch, buf.t_max, _stream()))
+
+
+def quasar_accept_stochastic(logits: torch.Tensor, tokens: torch.Tensor, block_len: torch.Tensor, q_probs, temperature: float,
+                             r_accept: torch.Tensor, r_sample: torch.Tensor):
+    """logits fp32 [B][T][V]; tokens int32 [B][T]; block_len int32 [B]; q_probs fp32 [B][T][V] or None;
+    r_accept fp32 [B][T]; r_sample fp32 [B].  Returns (accept_len, next_token), int32 [B]."""
+    b, t, v = logits.shape
+    accept_len = torch.empty(b, dtype=torch.int32, device=logits.device)
+    nxt = torch.empty(b, dtype=torch.int32, device=logits.device)
+    nbytes = _sz(0)
+    _check(lib().quasar_accept_stochastic_workspace_bytes(b, t, C.byref(nbytes)))
+    ws = torch.empty(int(nbytes.value), dtype=torch.uint8, device=logits.device)
+    _check(lib().quasar_accept_stochastic(_ptr(logits), _ptr(tokens), _ptr(block_len), _ptr(q_probs), b, t, v, temperature,
+                                          _ptr(r_accept), _ptr(r_sample), _ptr(accept_len), _ptr(nxt), _ptr(ws), ws.numel(),
+                                          _stream()))
+    return accept_len, nxt
 
 
 class Plan:

@@ -643,6 +643,32 @@ int quasar_verify(quasar_model* m, const quasar_kv* kv, const int32_t* tokens, c
                      workspace_bytes, status, (cudaStream_t)stream);
 }
 
+int quasar_accept_stochastic_workspace_bytes(int32_t B, int32_t T_max, size_t* bytes_out) {
+  if (bytes_out == nullptr || B < 1 || T_max < 1) { set_error("accept_stochastic_workspace_bytes: bad argument"); return QUASAR_ERR_INVALID_ARG; }
+  *bytes_out = accept_stochastic_workspace_bytes(B, T_max);
+  return QUASAR_OK;
+}
+
+int quasar_accept_stochastic(const float* logits, const int32_t* tokens, const int32_t* block_len, const float* q_probs,
+                             int32_t B, int32_t T_max, int32_t V, float temperature, const float* r_accept,
+                             const float* r_sample, int32_t* accept_len, int32_t* next_token, void* workspace,
+                             size_t workspace_bytes, void* stream) {
+  if (B < 1 || T_max < 1 || T_max > QUASAR_MAX_BLOCK || V < 1 || B > 65535) { set_error("accept_stochastic: B=%d T_max=%d V=%d", B, T_max, V); return QUASAR_ERR_SHAPE; }
+  if (!(temperature > 0.f)) { set_error("accept_stochastic: temperature must be positive (use the greedy acceptance of quasar_verify at 0)"); return QUASAR_ERR_INVALID_ARG; }
+  REQUIRE_PTR(logits, "logits");
+  REQUIRE_PTR(tokens, "tokens");
+  REQUIRE_PTR(block_len, "block_len");
+  REQUIRE_PTR(r_accept, "r_accept");
+  REQUIRE_PTR(r_sample, "r_sample");
+  REQUIRE_PTR(accept_len, "accept_len");
+  REQUIRE_PTR(next_token, "next_token");
+  REQUIRE_PTR(workspace, "workspace");
+  if (q_probs && !aligned16(q_probs)) { set_error("q_probs is not 16-byte aligned"); return QUASAR_ERR_ALIGN; }
+  if (workspace_bytes < accept_stochastic_workspace_bytes(B, T_max)) { set_error("accept_stochastic: workspace too small"); return QUASAR_ERR_CAPACITY; }
+  return launch_accept_stochastic(logits, tokens, block_len, q_probs, B, T_max, V, temperature, r_accept, r_sample, accept_len,
+                                  next_token, workspace, (cudaStream_t)stream);
+}
+
 int quasar_kv_commit(quasar_model* m, const quasar_kv* kv, const int32_t* accept_len, const int32_t* accept_path,
                      int32_t B, int32_t T_max, void* stream) {
   if (m == nullptr || kv == nullptr) { set_error("kv_commit: NULL argument"); return QUASAR_ERR_INVALID_ARG; }
