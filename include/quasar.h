@@ -258,6 +258,19 @@ int quasar_verify(quasar_model* m, const quasar_kv* kv /* host struct */, const 
                   size_t workspace_bytes, int32_t* status, void* stream);
 
 /* ------------------------------------------------------------------------
+ * Drafting by prompt lookup (Section 4.1: the n-gram drafter of the paper's experiments; lookup
+ * range K = (k_min, k_max) of Section 4.4 / Table 3).  Per sequence: for n = k_max down to k_min
+ * the last n of its hist_len[b] tokens are searched for among the tokens before them; the most
+ * recent earlier occurrence that is followed by at least one token wins, and the up to gamma
+ * tokens after it are the draft (the longest n with such an occurrence is used).
+ * history int32 [B][S] (the sequence so far, prompt included); hist_len int32 [B] (<= S);
+ * draft int32 [B][gamma] (entries past draft_len are -1); draft_len int32 [B] in [0, gamma]
+ * (0: nothing to look up - verify with block_len 1, a plain decode step).  1 <= k_min <= k_max.
+ * ---------------------------------------------------------------------- */
+int quasar_ngram_draft(const int32_t* history, const int32_t* hist_len, int32_t B, int32_t S, int32_t gamma,
+                       int32_t k_min, int32_t k_max, int32_t* draft, int32_t* draft_len, void* stream);
+
+/* ------------------------------------------------------------------------
  * Stochastic acceptance of drafted CHAINS (Section 3.1 Eq. 2-3; Section 3.3 "Lossless Rejection
  * Sampling"), applied to the logits quasar_verify wrote.  With p = softmax(logits / temperature):
  * draft i+1 (block row i+1) is accepted while r_accept[b][i] < min(1, p_i(token) / q_i(token))

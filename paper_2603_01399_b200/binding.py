@@ -75,6 +75,7 @@ SIGNATURES = {
     "quasar_model_destroy": (C.c_int, [_vp]),
     "quasar_workspace_bytes": (C.c_int, [_vp, _i32, _i32, C.POINTER(_sz)]),
     "quasar_verify": (C.c_int, _verify_args + [_vp]),
+    "quasar_ngram_draft": (C.c_int, [_vp, _vp, _i32, _i32, _i32, _i32, _i32, _vp, _vp, _vp]),
     "quasar_accept_stochastic_workspace_bytes": (C.c_int, [_i32, _i32, C.POINTER(_sz)]),
     "quasar_accept_stochastic": (C.c_int, [_vp, _vp, _vp, _vp, _i32, _i32, _i32, C.c_float, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "quasar_kv_commit": (C.c_int, [_vp, C.POINTER(KV), _vp, _vp, _i32, _i32, _vp]),
@@ -375,6 +376,15 @@ def quasar_verify(model: Model, kv: KVCache, buf: VerifyBuffers) -> None:
 def quasar_kv_commit(model: Model, kv: KVCache, buf: VerifyBuffers, tree: bool = False) -> None:
     _check(lib().quasar_kv_commit(model.handle, C.byref(kv.c), _ptr(buf.accept_len),
                                   _ptr(buf.accept_path) if tree else None, buf.batch, buf.t_max, _stream()))
+
+
+def quasar_ngram_draft(history: torch.Tensor, hist_len: torch.Tensor, gamma: int, k_min: int, k_max: int):
+    """history int32 [B][S], hist_len int32 [B] -> (draft int32 [B][gamma], draft_len int32 [B])."""
+    b, s = history.shape
+    draft = torch.empty((b, gamma), dtype=torch.int32, device=history.device)
+    dlen = torch.empty(b, dtype=torch.int32, device=history.device)
+    _check(lib().quasar_ngram_draft(_ptr(history), _ptr(hist_len), b, s, gamma, k_min, k_max, _ptr(draft), _ptr(dlen), _stream()))
+    return draft, dlen
 
 
 def quasar_accept_stochastic(logits: torch.Tensor, tokens: torch.Tensor, block_len: torch.Tensor, q_probs, temperature: float,

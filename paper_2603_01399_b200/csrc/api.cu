@@ -643,6 +643,19 @@ int quasar_verify(quasar_model* m, const quasar_kv* kv, const int32_t* tokens, c
                      workspace_bytes, status, (cudaStream_t)stream);
 }
 
+int quasar_ngram_draft(const int32_t* history, const int32_t* hist_len, int32_t B, int32_t S, int32_t gamma,
+                       int32_t k_min, int32_t k_max, int32_t* draft, int32_t* draft_len, void* stream) {
+  if (B < 1 || S < 1 || gamma < 1 || gamma > QUASAR_MAX_BLOCK - 1 || k_min < 1 || k_max < k_min) {
+    set_error("ngram_draft: B=%d S=%d gamma=%d K=(%d,%d)", B, S, gamma, k_min, k_max);
+    return QUASAR_ERR_INVALID_ARG;
+  }
+  REQUIRE_PTR(history, "history");
+  REQUIRE_PTR(hist_len, "hist_len");
+  REQUIRE_PTR(draft, "draft");
+  REQUIRE_PTR(draft_len, "draft_len");
+  return launch_ngram_draft(history, hist_len, B, S, gamma, k_min, k_max, draft, draft_len, (cudaStream_t)stream);
+}
+
 int quasar_accept_stochastic_workspace_bytes(int32_t B, int32_t T_max, size_t* bytes_out) {
   if (bytes_out == nullptr || B < 1 || T_max < 1) { set_error("accept_stochastic_workspace_bytes: bad argument"); return QUASAR_ERR_INVALID_ARG; }
   *bytes_out = accept_stochastic_workspace_bytes(B, T_max);

@@ -79,6 +79,10 @@ int launch_accept_stochastic(const float* logits, const int32_t* tokens, const i
                              int T_max, int V, float temperature, const float* r_accept, const float* r_sample,
                              int32_t* accept_len, int32_t* next_token, void* workspace, cudaStream_t stream);
 
+// prompt-lookup drafter (Section 4.1)
+int launch_ngram_draft(const int32_t* history, const int32_t* hist_len, int B, int S, int gamma, int k_min, int k_max,
+                       int32_t* draft, int32_t* draft_len, cudaStream_t stream);
+
 // Per-call description of the draft blocks, derived on the device from tokens / parents / block_len.
 struct BlockInfo {
   uint64_t* anc;    // [B*T_max] bit j set: block row j is row i itself or an ancestor of it

@@ -75,9 +75,16 @@ def test_stochastic_acceptance_matches_the_oracle(V, with_q, temp):
         if m_acc > 1e-4:                             # every accept / reject comparison is clear of its threshold
             assert acc[b] == n, (b, acc[b], n)
             assert w[nxt[b]] > 0, "a token of zero weight was drawn"
+            # inversion: the drawn token's interval of the cumulative weights must hold r_sample * total, up to the
+            # rounding of an fp32 running sum over V terms; where the target is clear of every edge the token is
+            # the oracle's
+            c = np.cumsum(w)
+            tgt, tol = float(r_sample[b]) * c[-1], 3e-5 * c[-1]
+            lo = c[nxt[b] - 1] if nxt[b] > 0 else 0.0
+            assert lo - tol <= tgt <= c[nxt[b]] + tol, (b, nxt[b], tok, lo, tgt, c[nxt[b]])
             if m_draw > 1e-4:
                 assert nxt[b] == tok, (b, nxt[b], tok)
-                checked += 1
+            checked += 1
     assert checked >= B // 2
 
 
