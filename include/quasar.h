@@ -140,8 +140,12 @@ int quasar_linear_w8a8(const void* x, const float* s, const int8_t* w, const flo
  * process exits.  The call itself allocates and frees nothing.
  *  - Shapes whose scratch would exceed the array are refused with QUASAR_ERR_CAPACITY
  *    (the message gives both sizes); use quasar_linear for those.
- *  - The first call on a device looks up the array's device address (with that device
- *    current); make that first call outside any stream capture.
+ *  - The array is the one of the CURRENT device: on every call the current device must be the
+ *    device `stream` belongs to (the library cannot check this; a mismatch hands the kernel
+ *    another GPU's address).  The first call on a device looks up the array's device address;
+ *    that lookup may make the runtime load the library's device code and is the only step
+ *    that can allocate, so make that first call outside any stream capture.  Argument errors
+ *    are reported before the lookup.
  *  - All calls on a device share the one array, and it keeps the previous call's contents
  *    (the part that must start at zero is cleared on `stream` by every call).  Two calls
  *    that may overlap on the GPU - different streams without an ordering between them -

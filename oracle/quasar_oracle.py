@@ -535,3 +535,53 @@ def ngram_draft(history: List[int], gamma: int, k_min: int, k_max: int) -> List[
             if h[start:start + n] == pattern:
                 return h[start + n:start + n + gamma]
     return []
+
+
+# --------------------------------------------------------------------------
+# 4-bit weights (Section 6, "Ultra-low Bit Verification": the first item of the paper's outlook)
+# --------------------------------------------------------------------------
+# The paper only names the direction (weights of 4 bits or fewer).  Reading: the operator Q of Eq. 6 with a
+# range of [-7, 7] and one step size per output channel AND group of 128 consecutive input channels
+# (per-channel steps alone are too coarse at 4 bits); two codes per byte, the even input channel in the low
+# nibble, two's complement.
+
+
+INT4_GROUP = 128
+
+
+def quantize_int4(w_f32: np.ndarray, group: int = INT4_GROUP):
+    """w_f32: [N][K] fp32 holding bf16 values, K a multiple of `group`.
+    Returns (codes int8 [N][K] in [-7, 7], delta fp32 [N][K / group])."""
+    w = np.asarray(w_f32, dtype=np.float32)
+    n, k = w.shape
+    assert k % group == 0
+    wg = w.reshape(n, k // group, group)
+    absmax = np.max(np.abs(wg), axis=2)
+    delta = (absmax / np.float32(7.0)).astype(np.float32)
+    delta = np.where(absmax == 0, np.float32(1.0), delta).astype(np.float32)
+    q = np.clip(np.rint(wg / delta[:, :, None]), -7.0, 7.0).astype(np.int8)
+    return q.reshape(n, k), delta
+
+
+def pack_int4(codes: np.ndarray) -> np.ndarray:
+    """int8 [N][K] in [-8, 7] -> uint8 [N][K / 2]: channel 2j in the low nibble, 2j + 1 in the high one."""
+    c = codes.astype(np.int16) & 0xF
+    return (c[:, 0::2] | (c[:, 1::2] << 4)).astype(np.uint8)
+
+
+def unpack_int4(packed: np.ndarray) -> np.ndarray:
+    p = packed.astype(np.int16)
+    lo, hi = p & 0xF, (p >> 4) & 0xF
+    out = np.empty((packed.shape[0], packed.shape[1] * 2), np.int16)
+    out[:, 0::2], out[:, 1::2] = lo, hi
+    return np.where(out >= 8, out - 16, out).astype(np.int8)
+
+
+def linear_int4(x: np.ndarray, codes: np.ndarray, delta: np.ndarray, group: int = INT4_GROUP) -> np.ndarray:
+    """Y[m][n] = sum_g delta[n][g] * sum_{k in g} X[m][k] * codes[n][k]  (Eq. 8 with one step per group), fp64."""
+    m, k = x.shape
+    n = codes.shape[0]
+    xg = np.asarray(x, np.float64).reshape(m, k // group, group)
+    cg = codes.astype(np.float64).reshape(n, k // group, group)
+    part = np.einsum("mgk,ngk->mng", xg, cg)
+    return np.einsum("mng,ng->mn", part, delta.astype(np.float64))

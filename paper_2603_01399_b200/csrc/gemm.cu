@@ -368,8 +368,22 @@ size_t linear_static_scratch_bytes() { return kStaticScratchBytes; }
 int launch_linear_static(const __nv_bfloat16* x, const void* w, const float* delta, int weight_dtype, int64_t M,
                          int64_t N, int64_t K, void* y, bool y_is_f32, const __nv_bfloat16* residual,
                          cudaStream_t stream) {
+  if (M <= 0 || N <= 0 || K <= 0 || (K % 16) != 0 || N > kMaxChannels || K > 0x7fffffff) {
+    set_error("linear_static: unsupported sizes M=%lld N=%lld K=%lld (K must be a multiple of 16, N at most %lld)",
+              (long long)M, (long long)N, (long long)K, (long long)kMaxChannels);
+    return QUASAR_ERR_SHAPE;
+  }
+  const size_t need = linear_workspace_bytes(M, N, K);
+  if (need > kStaticScratchBytes) {
+    set_error("linear_static: M=%lld N=%lld K=%lld needs %zu bytes of scratch, the built-in array holds %zu; "
+              "use quasar_linear with a workspace",
+              (long long)M, (long long)N, (long long)K, need, kStaticScratchBytes);
+    return QUASAR_ERR_CAPACITY;
+  }
   // In host code the array's name only stands for the symbol; its device address is looked up once per
-  // device (with that device current) and kept.
+  // device (with that device current) and kept.  The lookup comes after the argument checks, so a refused
+  // call touches nothing; it is the only step that may make the runtime load the module (and with it
+  // materialise the array) - hence "first call outside any capture".
   constexpr int kMaxDevices = 64;
   static void* scratch_of_device[kMaxDevices] = {};
   static std::mutex mu;
@@ -389,20 +403,10 @@ int launch_linear_static(const __nv_bfloat16* x, const void* w, const float* del
     }
     scratch = scratch_of_device[dev];
   }
-  if (M <= 0 || N <= 0 || K <= 0 || (K % 16) != 0 || N > kMaxChannels || K > 0x7fffffff) {
-    set_error("linear_static: unsupported sizes M=%lld N=%lld K=%lld (K must be a multiple of 16, N at most %lld)",
-              (long long)M, (long long)N, (long long)K, (long long)kMaxChannels);
-    return QUASAR_ERR_SHAPE;
-  }
-  const size_t need = linear_workspace_bytes(M, N, K);
-  if (need > kStaticScratchBytes) {
-    set_error("linear_static: M=%lld N=%lld K=%lld needs %zu bytes of scratch, the built-in array holds %zu; "
-              "use quasar_linear with a workspace",
-              (long long)M, (long long)N, (long long)K, need, kStaticScratchBytes);
-    return QUASAR_ERR_CAPACITY;
-  }
-  // The arrival counters must start at zero; the array keeps whatever the last call left in it.
-  QUASAR_CUDA_CHECK(cudaMemsetAsync(scratch, 0, kCounterBytes, stream));
+  // The arrival counters must start at zero; the array keeps whatever the last call left in it.  (Only the
+  // split-K form of the warp-level kernel counts arrivals.)
+  const bool counts = plan_split(N, K).nsplit > 1 && !(weight_dtype == QUASAR_W_INT8 && M > 8 && umma_w8a16_usable(M < 80 ? M : 80, N, K));
+  if (counts) QUASAR_CUDA_CHECK(cudaMemsetAsync(scratch, 0, kCounterBytes, stream));
   return launch_linear(x, w, delta, weight_dtype, M, N, K, y, y_is_f32, residual, scratch, kStaticScratchBytes, stream, nullptr);
 }
 

@@ -47,6 +47,22 @@ def test_two_calls_in_a_row_match_the_workspace_version():
         assert torch.equal(out, want)
 
 
+def test_a_warmed_up_call_allocates_nothing_and_blocks_of_more_than_72_rows_work():
+    """The point of the entry: after its first call on the device (which looks the array up) a call leaves
+    the device's free memory exactly as it found it; and a block of 80 rows takes the same route."""
+    x, w, d, res, want, out = _case(80, 256, 512, 31)
+    binding.quasar_linear_static(x, w, d, out)                      # first call: address lookup
+    torch.cuda.synchronize()
+    assert torch.equal(out, want)
+    free_before, _ = torch.cuda.mem_get_info()
+    for _ in range(3):
+        binding.quasar_linear_static(x, w, d, out)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before
+    assert torch.equal(out, want)
+
+
 def test_refuses_shapes_beyond_the_built_in_scratch():
     cap = binding.quasar_linear_static_scratch_bytes()
     assert cap == 4 << 20
