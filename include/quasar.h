@@ -126,6 +126,22 @@ int quasar_linear_w8a8(const void* x, const float* s, const int8_t* w, const flo
                        size_t workspace_bytes, void* stream);
 
 /* ------------------------------------------------------------------------
+ * 4-bit weights (Section 6, "Ultra-low Bit Verification", the first item of the paper's outlook;
+ * the weight term of Section 3.4 drops to a quarter of the bf16 one).  The quantiser is Q of Eq. 6
+ * with the range [-7, 7] and one step size per output channel and group of 128 consecutive input
+ * channels; two codes per byte, the even input channel in the low nibble, two's complement.
+ * quasar_quantize_int4: w_bf16 [N][K], K % 128 == 0 -> packed uint8 [N][K/2], delta fp32 [N][K/128];
+ *   bit-exact with the definition (fp32 IEEE division, round-half-even, all-zero group -> delta 1).
+ * quasar_linear_w4:  Y[m][n] = sum_g delta[n][g] * sum_{k in g} X[m][k] * code[n][k]  (+ residual as
+ *   in quasar_linear); x bf16 [M][K]; fp32 accumulation inside a group and across groups; y bf16 or
+ *   fp32; workspace from quasar_linear_w4_workspace_bytes (no zero-filling needed).
+ * ---------------------------------------------------------------------- */
+int quasar_quantize_int4(const void* w_bf16, int64_t N, int64_t K, uint8_t* packed_out, float* delta_out, void* stream);
+int quasar_linear_w4_workspace_bytes(int64_t M, int64_t N, int64_t K, size_t* bytes_out /* host */);
+int quasar_linear_w4(const void* x, const uint8_t* packed, const float* delta, int64_t M, int64_t N, int64_t K, void* y,
+                     int32_t y_is_f32, const void* residual, void* workspace, size_t workspace_bytes, void* stream);
+
+/* ------------------------------------------------------------------------
  * quasar_linear for callers that may not allocate device memory.  (The paper has no
  * counterpart: this is a convenience of the library, not a step of the method.)
  *

@@ -69,6 +69,9 @@ SIGNATURES = {
     "quasar_quantize_activations": (C.c_int, [_vp, _vp, _i64, _i64, _vp, _vp, _vp]),
     "quasar_linear_w8a8_workspace_bytes": (C.c_int, [_i64, _i64, _i64, C.POINTER(_sz)]),
     "quasar_linear_w8a8": (C.c_int, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _vp, _i32, _vp, _vp, _vp, _sz, _vp]),
+    "quasar_quantize_int4": (C.c_int, [_vp, _i64, _i64, _vp, _vp, _vp]),
+    "quasar_linear_w4_workspace_bytes": (C.c_int, [_i64, _i64, _i64, C.POINTER(_sz)]),
+    "quasar_linear_w4": (C.c_int, [_vp, _vp, _vp, _i64, _i64, _i64, _vp, _i32, _vp, _vp, _sz, _vp]),
     "quasar_linear_static_scratch_bytes": (_sz, []),
     "quasar_linear_static": (C.c_int, [_vp, _vp, _vp, _i32, _i64, _i64, _i64, _vp, _i32, _vp, _vp]),
     "quasar_model_create": (C.c_int, [C.POINTER(Config), C.POINTER(Weights), C.POINTER(_vp)]),
@@ -197,6 +200,30 @@ def quasar_linear_w8a8(x: torch.Tensor, s: Optional[torch.Tensor], w: torch.Tens
     _check(lib().quasar_linear_w8a8(_ptr(x), _ptr(s), _ptr(w), _ptr(delta_w), m, n, k, _ptr(y), 1 if out_f32 else 0,
                                     _ptr(residual), _ptr(acc), _ptr(ws), ws.numel(), _stream()))
     return (y, acc) if want_acc else y
+
+
+def quasar_quantize_int4(w_bf16: torch.Tensor):
+    """bf16 [N][K] (K a multiple of 128) -> (packed uint8 [N][K/2], delta fp32 [N][K/128])."""
+    n, k = w_bf16.shape
+    packed = torch.empty((n, k // 2), dtype=torch.uint8, device=w_bf16.device)
+    delta = torch.empty((n, k // 128), dtype=torch.float32, device=w_bf16.device)
+    _check(lib().quasar_quantize_int4(_ptr(w_bf16), n, k, _ptr(packed), _ptr(delta), _stream()))
+    return packed, delta
+
+
+def quasar_linear_w4(x: torch.Tensor, packed: torch.Tensor, delta: torch.Tensor, residual=None, out_f32=False,
+                     workspace=None, out=None) -> torch.Tensor:
+    m, k = x.shape
+    n = packed.shape[0]
+    if out is None:
+        out = torch.empty((m, n), dtype=torch.float32 if out_f32 else torch.bfloat16, device=x.device)
+    if workspace is None:
+        nbytes = _sz(0)
+        _check(lib().quasar_linear_w4_workspace_bytes(m, n, k, C.byref(nbytes)))
+        workspace = torch.empty(max(int(nbytes.value), 16), dtype=torch.uint8, device=x.device)
+    _check(lib().quasar_linear_w4(_ptr(x), _ptr(packed), _ptr(delta), m, n, k, _ptr(out), 1 if out.dtype == torch.float32 else 0,
+                                  _ptr(residual), _ptr(workspace), workspace.numel(), _stream()))
+    return out
 
 
 def quasar_linear_static_scratch_bytes() -> int:

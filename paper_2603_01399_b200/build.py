@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libquasar.so")
-SOURCES = ["api.cu", "quantize.cu", "gemm.cu", "layer_ops.cu", "attention.cu", "megakernel.cu", "w8a8.cu", "umma_gemm.cu", "sampling.cu", "drafter.cu"]
+SOURCES = ["api.cu", "quantize.cu", "gemm.cu", "layer_ops.cu", "attention.cu", "megakernel.cu", "w8a8.cu", "umma_gemm.cu", "sampling.cu", "drafter.cu", "int4.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC",

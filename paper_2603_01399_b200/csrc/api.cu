@@ -431,6 +431,34 @@ int quasar_linear_w8a8(const void* x, const float* s, const int8_t* w, const flo
                             (cudaStream_t)stream);
 }
 
+int quasar_quantize_int4(const void* w_bf16, int64_t N, int64_t K, uint8_t* packed_out, float* delta_out, void* stream) {
+  if (N < 0 || K < 0) { set_error("quantize_int4: negative size"); return QUASAR_ERR_INVALID_ARG; }
+  if (N == 0 || K == 0) return QUASAR_OK;
+  if (K % 128 != 0 || N > 0x7fffffffLL) { set_error("quantize_int4: K=%lld must be a multiple of 128", (long long)K); return QUASAR_ERR_SHAPE; }
+  REQUIRE_PTR(w_bf16, "w_bf16");
+  REQUIRE_PTR(packed_out, "packed_out");
+  REQUIRE_PTR(delta_out, "delta_out");
+  return launch_quantize_int4(reinterpret_cast<const __nv_bfloat16*>(w_bf16), N, K, packed_out, delta_out, (cudaStream_t)stream);
+}
+
+int quasar_linear_w4_workspace_bytes(int64_t M, int64_t N, int64_t K, size_t* bytes_out) {
+  if (bytes_out == nullptr || M <= 0 || N <= 0 || K <= 0 || K % 128 != 0) { set_error("linear_w4_workspace_bytes: bad argument"); return QUASAR_ERR_INVALID_ARG; }
+  *bytes_out = linear_w4_workspace_bytes(M, N, K);
+  return QUASAR_OK;
+}
+
+int quasar_linear_w4(const void* x, const uint8_t* packed, const float* delta, int64_t M, int64_t N, int64_t K, void* y,
+                     int32_t y_is_f32, const void* residual, void* workspace, size_t workspace_bytes, void* stream) {
+  REQUIRE_PTR(x, "x");
+  REQUIRE_PTR(packed, "packed");
+  REQUIRE_PTR(delta, "delta");
+  REQUIRE_PTR(y, "y");
+  REQUIRE_PTR(workspace, "workspace");
+  if (residual && !aligned16(residual)) { set_error("residual is not 16-byte aligned"); return QUASAR_ERR_ALIGN; }
+  return launch_linear_w4(reinterpret_cast<const __nv_bfloat16*>(x), packed, delta, M, N, K, y, y_is_f32 != 0,
+                          reinterpret_cast<const __nv_bfloat16*>(residual), workspace, workspace_bytes, (cudaStream_t)stream);
+}
+
 int quasar_linear_static(const void* x, const void* w, const float* delta, int32_t weight_dtype, int64_t M, int64_t N,
                          int64_t K, void* y, int32_t y_is_f32, const void* residual, void* stream) {
   if (weight_dtype != QUASAR_W_INT8 && weight_dtype != QUASAR_W_BF16) { set_error("linear_static: weight_dtype %d", weight_dtype); return QUASAR_ERR_INVALID_ARG; }

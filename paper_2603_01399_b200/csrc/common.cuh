@@ -83,6 +83,13 @@ int launch_accept_stochastic(const float* logits, const int32_t* tokens, const i
 int launch_ngram_draft(const int32_t* history, const int32_t* hist_len, int B, int S, int gamma, int k_min, int k_max,
                        int32_t* draft, int32_t* draft_len, cudaStream_t stream);
 
+// 4-bit group-wise weights (Section 6 outlook)
+int launch_quantize_int4(const __nv_bfloat16* w, int64_t N, int64_t K, uint8_t* packed, float* delta, cudaStream_t stream);
+size_t linear_w4_workspace_bytes(int64_t M, int64_t N, int64_t K);
+int launch_linear_w4(const __nv_bfloat16* x, const uint8_t* w, const float* delta, int64_t M, int64_t N, int64_t K, void* y,
+                     bool y_is_f32, const __nv_bfloat16* residual, void* workspace, size_t workspace_bytes,
+                     cudaStream_t stream);
+
 // Per-call description of the draft blocks, derived on the device from tokens / parents / block_len.
 struct BlockInfo {
   uint64_t* anc;    // [B*T_max] bit j set: block row j is row i itself or an ancestor of it
