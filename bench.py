@@ -277,6 +277,8 @@ def run_ours(args):
     torch.cuda.empty_cache()
     extra = {}
     if rank == 0 and not args.headline_only:
+        extra["gamma_sweep"] = gamma_sweep(binding, m_int8, shape, kv, root, hbm_peak)
+        extra["int4_linear"] = int4_linear_line(binding, hbm_peak)
         extra["w8a8"] = time_w8a8(binding, shape, kv, tokens_host, max(3, args.steps // 4), hbm_peak)
         extra["linear_sweep"] = linear_sweep_summary(binding, hbm_peak)
         extra["tree14b"] = time_tree14b(binding, max(3, args.steps // 5), hbm_peak)
@@ -460,6 +462,63 @@ def linear_sweep_summary(binding, hbm_peak):
         torch.cuda.empty_cache()
     return {"what": "quantised linear layer alone (quasar_linear, int8 weights), fraction of the measured copy bandwidth",
             "shapes": out}
+
+
+def gamma_sweep(binding, model, shape, kv, root, hbm_peak):
+    """Section 4.4 / Table 3 and Eq. 13 in miniature: verify latency and accepted tokens per second against the
+    draft length gamma, on the model's own greedy continuation with each token replaced w.p. 0.3, plus the cost
+    of the prompt-lookup drafter on a 4096-token history (T_draft of Eq. 13)."""
+    out = {}
+    greedy = greedy_continuation(binding, model, kv, root, 9)
+    for gamma in (3, 5, 7, 9):
+        draft = synth.corrupt_draft(greedy[:, :gamma], 0.3, shape.vocab, seed=2)
+        buf = binding.VerifyBuffers(model, BATCH, gamma + 1, want_logits=False)
+        buf.tokens.copy_(torch.cat([root.cpu().view(-1, 1), draft], dim=1).to(torch.int32))
+        plan = binding.Plan(model, kv, buf)
+        ms = _time_plan(plan, 10)
+        acc = int((buf.accept_len + 1).sum())
+        out[str(gamma)] = {"verify_latency_ms": ms, "accepted_per_pass": acc, "accepted_tok_s": acc / (ms * 1e-3),
+                           "launch": model.launch_kind(BATCH, gamma + 1)}
+        plan.close()
+        del buf
+    hist = synth.uniform_tokens((BATCH, 4096), 50, synth.sub_seed(3, "tokens")).cuda()
+    hlen = torch.full((BATCH,), 4096, dtype=torch.int32, device="cuda")
+    binding.quasar_ngram_draft(hist, hlen, 5, 1, 4)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(20):
+        binding.quasar_ngram_draft(hist, hlen, 5, 1, 4)
+    e1.record()
+    torch.cuda.synchronize()
+    out["ngram_draft_us"] = e0.elapsed_time(e1) * 1e3 / 20
+    return out
+
+
+def int4_linear_line(binding, hbm_peak):
+    """The 4-bit group-wise linear layer alone on the gate+up shape at 6 rows, distinct weight copies per launch."""
+    k, n, m = 4096, 24576, 6
+    master = synth.normal_bf16((n, k), 0.02, seed=k + n, device="cuda")
+    packed, delta = binding.quasar_quantize_int4(master)
+    copies = 24
+    plist = [packed] + [packed.clone() for _ in range(copies - 1)]
+    x = synth.normal_bf16((m, k), 1.0, seed=m, device="cuda")
+    y = torch.empty((m, n), dtype=torch.bfloat16, device="cuda")
+    ws = torch.empty(1 << 26, dtype=torch.uint8, device="cuda")
+    for p in plist:
+        binding.quasar_linear_w4(x, p, delta, workspace=ws, out=y)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(3):
+        for p in plist:
+            binding.quasar_linear_w4(x, p, delta, workspace=ws, out=y)
+    e1.record()
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / (3 * copies)
+    nbytes = n * k // 2 + n * (k // 128) * 4
+    return {"what": "quasar_linear_w4, gate+up shape (K 4096, N 24576), 6 rows", "us_per_launch": us, "bytes": nbytes,
+            "gbs": nbytes / (us * 1e-6) / 1e9, "frac": nbytes / (us * 1e-6) / 1e9 / hbm_peak}
 
 
 def run_linear_sweep(args):
@@ -661,6 +720,64 @@ def run_profile_pass(args):
     print(json.dumps({"profile_pass": "done", "layers": shape.n_layers, "status": int(buf.status[0])}))
 
 
+def run_profile_linear(args):
+    """For `ncu --profile-from-start off`: ONE quantised linear layer of a named Qwen3-8B shape at --rows rows
+    (int8 weights; --a8: the W8A8 form) between cudaProfilerStart/Stop, after two warm-up calls."""
+    from paper_2603_01399_b200 import binding, build
+    build.build()
+    torch.cuda.set_device(0)
+    shapes = {"qkv": (4096, 6144), "o": (4096, 4096), "gateup": (4096, 24576), "down": (12288, 4096), "lm_head": (4096, 151936)}
+    k, n = shapes[args.profile_linear]
+    m = args.rows
+    master = synth.normal_bf16((n, k), 0.02, seed=k + n, device="cuda")
+    x = synth.normal_bf16((m, k), 1.0, seed=m, device="cuda")
+    if args.a8:
+        q, d = binding.quasar_quantize_weights_smoothed(master, None)
+        call = lambda: binding.quasar_linear_w8a8(x, None, q, d)
+    else:
+        q, d = binding.quasar_quantize(master)
+        ws = torch.zeros(binding.quasar_linear_workspace_bytes(m, n, k), dtype=torch.uint8, device="cuda")
+        y = torch.empty((m, n), dtype=torch.bfloat16, device="cuda")
+        call = lambda: binding.quasar_linear(x, q, d, workspace=ws, out=y)
+    del master
+    for _ in range(2):
+        call()
+    torch.cuda.synchronize()
+    torch.cuda.profiler.start()
+    call()
+    torch.cuda.synchronize()
+    torch.cuda.profiler.stop()
+    print(json.dumps({"profile_linear": args.profile_linear, "rows": m, "a8": bool(args.a8), "weight_bytes": n * k}))
+
+
+def run_profile_batch8(args):
+    """For `ncu --profile-from-start off`: one eager pass of the batch-of-eight workload (prefixes U(512,4096),
+    chains of 8 drafts, 72 block rows) on a model cut to --profile-layers layers."""
+    from paper_2603_01399_b200 import binding, build
+    build.build()
+    torch.cuda.set_device(0)
+    full = synth.SHAPES["qwen3_8b"]
+    shape = synth.ModelShape("qwen3_8b_cut", args.profile_layers or 2, full.hidden, full.n_q_heads, full.n_kv_heads, full.head_dim,
+                             full.ffn, full.vocab, full.qk_norm, full.rope_theta, full.rms_eps)
+    absmax = (lambda kind, layer: synth.activation_absmax(shape, kind, layer, 0, "cuda")) if args.a8 else None
+    model = binding.Model.from_master(shape, master_getter(shape, 0, "cuda"), 4096 + 16, int8=True, act_int8=bool(args.a8),
+                                      get_act_absmax=absmax)
+    rng = np.random.default_rng(4)
+    prefix = [int(v) for v in rng.integers(512, 4097, 8)]
+    kk, vv = synth.kv_prefix(shape, 8, 4096 + 16, seed=1, device="cuda")
+    kv = binding.KVCache(shape, 8, 4096 + 16, k=kk, v=vv, seq_len=torch.tensor(prefix, dtype=torch.int32, device="cuda"))
+    buf = binding.VerifyBuffers(model, 8, 9, want_logits=False)
+    buf.tokens.copy_(synth.uniform_tokens((8, 9), shape.vocab, synth.sub_seed(2, "tokens")))
+    for _ in range(2):
+        binding.quasar_verify(model, kv, buf)
+    torch.cuda.synchronize()
+    torch.cuda.profiler.start()
+    binding.quasar_verify(model, kv, buf)
+    torch.cuda.synchronize()
+    torch.cuda.profiler.stop()
+    print(json.dumps({"profile_batch8": "done", "layers": shape.n_layers, "a8": bool(args.a8), "status": int(buf.status[0])}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -671,10 +788,18 @@ def main():
                     help="run one eager verify pass inside cudaProfilerStart/Stop (for ncu), no timing")
     ap.add_argument("--profile-layers", type=int, default=0, help="with --profile-pass: cut the model to this many layers")
     ap.add_argument("--linear-sweep", action="store_true", help="time the quantised linear layer alone over shapes and row counts")
+    ap.add_argument("--profile-linear", default="", help="one quantised linear layer of this Qwen3-8B shape inside cudaProfilerStart/Stop (for ncu)")
+    ap.add_argument("--profile-batch8", action="store_true", help="one eager batch-of-eight pass inside cudaProfilerStart/Stop (for ncu)")
+    ap.add_argument("--rows", type=int, default=72, help="with --profile-linear: activation rows")
+    ap.add_argument("--a8", action="store_true", help="with --profile-linear / --profile-batch8: the W8A8 form")
     ap.add_argument("--headline-only", action="store_true", help="skip the side workloads (W8A8, linear sweep, 14B tree)")
     args = ap.parse_args()
     if args.profile_pass:
         return run_profile_pass(args)
+    if args.profile_linear:
+        return run_profile_linear(args)
+    if args.profile_batch8:
+        return run_profile_batch8(args)
     if args.linear_sweep:
         return run_linear_sweep(args)
     # --gpus N: N independent replicas (the pass has no exchange step), one process per GPU.  Launched
