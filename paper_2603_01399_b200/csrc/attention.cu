@@ -76,8 +76,10 @@ template <int D>
 __global__ void __launch_bounds__(kMaxWarps * 32) verify_attention_kernel(AttnArgs a) {
   constexpr int kStride = D + 8;  // padded row of the staged K / V tiles (bf16 elements)
   constexpr int kDSteps = D / 16;
-  __shared__ __align__(16) __nv_bfloat16 k_s[kKeyTile * kStride];
-  __shared__ __align__(16) __nv_bfloat16 v_s[kKeyTile * kStride];
+  // two K tiles and two V tiles: the next tile of the chunk lands (cp.async) while the current one is multiplied
+  extern __shared__ __align__(16) unsigned char attn_smem[];
+  __nv_bfloat16* const tiles = reinterpret_cast<__nv_bfloat16*>(attn_smem);
+  constexpr int kTileElems = kKeyTile * kStride;
 
   const int c = blockIdx.x / a.ngroups, group = blockIdx.x % a.ngroups;
   const int hk = blockIdx.y, b = blockIdx.z;
@@ -125,19 +127,35 @@ __global__ void __launch_bounds__(kMaxWarps * 32) verify_attention_kernel(AttnAr
   const __nv_bfloat16* kbase = a.kc + ((size_t)b * a.Hkv + hk) * (size_t)a.s_max * D;
   const __nv_bfloat16* vbase = a.vc + ((size_t)b * a.Hkv + hk) * (size_t)a.s_max * D;
 
-  for (int k0 = key_begin; k0 < key_end; k0 += kKeyTile) {
-    __syncthreads();
+  auto stage_tile = [&](int buf, int k0) {
+    __nv_bfloat16* kd = tiles + buf * 2 * kTileElems;
+    __nv_bfloat16* vd = kd + kTileElems;
     for (int i = threadIdx.x; i < kKeyTile * (D / 8); i += blockDim.x) {
       const int key = i / (D / 8), ch = i % (D / 8);
-      uint4 kv4 = make_uint4(0, 0, 0, 0), vv4 = make_uint4(0, 0, 0, 0);
       if (k0 + key < key_end) {
-        kv4 = __ldg(reinterpret_cast<const uint4*>(kbase + (size_t)(k0 + key) * D) + ch);
-        vv4 = __ldg(reinterpret_cast<const uint4*>(vbase + (size_t)(k0 + key) * D) + ch);
+        const uint32_t ks = (uint32_t)__cvta_generic_to_shared(kd + key * kStride + ch * 8);
+        const uint32_t vs = (uint32_t)__cvta_generic_to_shared(vd + key * kStride + ch * 8);
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(ks), "l"(kbase + (size_t)(k0 + key) * D + ch * 8) : "memory");
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(vs), "l"(vbase + (size_t)(k0 + key) * D + ch * 8) : "memory");
+      } else {
+        *reinterpret_cast<uint4*>(kd + key * kStride + ch * 8) = make_uint4(0, 0, 0, 0);
+        *reinterpret_cast<uint4*>(vd + key * kStride + ch * 8) = make_uint4(0, 0, 0, 0);
       }
-      *reinterpret_cast<uint4*>(k_s + key * kStride + ch * 8) = kv4;
-      *reinterpret_cast<uint4*>(v_s + key * kStride + ch * 8) = vv4;
+    }
+    asm volatile("cp.async.commit_group;\n" ::: "memory");
+  };
+  stage_tile(0, key_begin);
+  int buf = 0;
+  for (int k0 = key_begin; k0 < key_end; k0 += kKeyTile, buf ^= 1) {
+    if (k0 + kKeyTile < key_end) {
+      stage_tile(buf ^ 1, k0 + kKeyTile);           // (its last readers passed the barrier that ended the tile before)
+      asm volatile("cp.async.wait_group 1;\n" ::: "memory");
+    } else {
+      asm volatile("cp.async.wait_group 0;\n" ::: "memory");
     }
     __syncthreads();
+    const __nv_bfloat16* k_s = tiles + buf * 2 * kTileElems;
+    const __nv_bfloat16* v_s = k_s + kTileElems;
 
     // S = Q K^T for 16 rows x 64 keys
     float s[kKeyTile / 8][4];
@@ -215,6 +233,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32) verify_attention_kernel(AttnAr
         mma16816(o[2 * dt + 1], al[0], al[1], al[2], al[3], b2, b3);
       }
     }
+    __syncthreads();   // every warp is done with this tile before the copy of the tile after next overwrites it
   }
 
   // ---- partial results ----------------------------------------------------------------------
@@ -333,12 +352,19 @@ int launch_attention(const __nv_bfloat16* qkv, const __nv_bfloat16* k_cache_laye
   dim3 grid(p.nchunk * p.ngroups, Hkv, B);
   const int items = B * T_max * Hq;
   if (D == 128) {
-    verify_attention_kernel<128><<<grid, p.warps * 32, 0, stream>>>(a);
+    constexpr size_t smem128 = 4u * kKeyTile * (128 + 8) * sizeof(__nv_bfloat16);
+    static bool configured128 = false;
+    if (!configured128) {
+      QUASAR_CUDA_CHECK(cudaFuncSetAttribute(verify_attention_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem128));
+      configured128 = true;
+    }
+    verify_attention_kernel<128><<<grid, p.warps * 32, smem128, stream>>>(a);
     QUASAR_LAUNCH_CHECK();
     attention_merge_kernel<128><<<(items + 3) / 4, 128, 0, stream>>>(a);
     QUASAR_LAUNCH_CHECK();
   } else if (D == 64) {
-    verify_attention_kernel<64><<<grid, p.warps * 32, 0, stream>>>(a);
+    constexpr size_t smem64 = 4u * kKeyTile * (64 + 8) * sizeof(__nv_bfloat16);
+    verify_attention_kernel<64><<<grid, p.warps * 32, smem64, stream>>>(a);
     QUASAR_LAUNCH_CHECK();
     attention_merge_kernel<64><<<(items + 3) / 4, 128, 0, stream>>>(a);
     QUASAR_LAUNCH_CHECK();
