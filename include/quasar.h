@@ -194,6 +194,13 @@ typedef struct quasar_config {
   int32_t max_seq;      /* cache capacity S_max (positions) the RoPE table covers */
   int32_t act_dtype;    /* QUASAR_A_BF16, or QUASAR_A_INT8 (needs weight_dtype QUASAR_W_INT8; the
                            weights must then be Q(W diag(s)^-1) for the smoothing vectors below) */
+  int32_t weights_in_place; /* 0: the model borrows the weight matrices and keeps a second, permuted copy for
+                           the persistent single-kernel pass (twice the weight bytes).  1: the caller hands
+                           the matrices over: quasar_model_create permutes each of them WHERE IT LIES into the
+                           order the persistent kernel streams it (their contents are no longer row-major
+                           afterwards) and keeps no copy, so the model occupies the weight bytes once - the
+                           footprint Section 3.3 ("Offline Weight Preparation") promises.  Such a model
+                           runs the persistent kernel only: blocks of at most 8 rows in total, no trace. */
 } quasar_config;
 
 typedef struct quasar_layer_weights {

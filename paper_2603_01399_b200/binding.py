@@ -35,7 +35,7 @@ class Config(C.Structure):
     _fields_ = [("n_layers", C.c_int32), ("hidden", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
                 ("head_dim", C.c_int32), ("ffn", C.c_int32), ("vocab", C.c_int32), ("qk_norm", C.c_int32),
                 ("rope_theta", C.c_float), ("rms_eps", C.c_float), ("weight_dtype", C.c_int32),
-                ("max_seq", C.c_int32), ("act_dtype", C.c_int32)]
+                ("max_seq", C.c_int32), ("act_dtype", C.c_int32), ("weights_in_place", C.c_int32)]
 
 
 class LayerWeights(C.Structure):
@@ -253,7 +253,7 @@ class Model:
     `.gateup_w`, `.gateup_delta`, `.down_w`, `.down_delta` (deltas absent for bf16 weights)."""
 
     def __init__(self, shape, tensors: Dict[str, torch.Tensor], max_seq: int, weight_dtype: int = QUASAR_W_INT8,
-                 act_dtype: int = QUASAR_A_BF16):
+                 act_dtype: int = QUASAR_A_BF16, weights_in_place: bool = False):
         self.shape = shape
         self.tensors = tensors
         self.weight_dtype = weight_dtype
@@ -261,7 +261,7 @@ class Model:
         self.max_seq = max_seq
         self.cfg = Config(shape.n_layers, shape.hidden, shape.n_q_heads, shape.n_kv_heads, shape.head_dim, shape.ffn,
                           shape.vocab, 1 if shape.qk_norm else 0, shape.rope_theta, shape.rms_eps, weight_dtype,
-                          max_seq, act_dtype)
+                          max_seq, act_dtype, 1 if weights_in_place else 0)
         layers = (LayerWeights * max(shape.n_layers, 1))()
         for l in range(shape.n_layers):
             for name, _ in LayerWeights._fields_:
@@ -276,7 +276,7 @@ class Model:
 
     @classmethod
     def from_master(cls, shape, get_master, max_seq: int, int8: bool = True, device="cuda", act_int8: bool = False,
-                    get_act_absmax=None, alpha: float = 0.5):
+                    get_act_absmax=None, alpha: float = 0.5, weights_in_place: bool = False):
         """get_master(kind, layer) -> bf16 master tensor (any device).  int8=True quantises every
         matrix on the GPU with quasar_quantize (the offline weight preparation).  act_int8=True builds the
         W8A8 verifier: get_act_absmax(kind, layer) -> fp32 [K] calibration maxima of the layer's input give
@@ -314,7 +314,7 @@ class Model:
             put_linear(f"l{l}.down", "down", l)
         torch.cuda.synchronize()
         return cls(shape, t, max_seq, QUASAR_W_INT8 if int8 else QUASAR_W_BF16,
-                   QUASAR_A_INT8 if act_int8 else QUASAR_A_BF16)
+                   QUASAR_A_INT8 if act_int8 else QUASAR_A_BF16, weights_in_place)
 
     def workspace_bytes(self, batch: int, t_max: int) -> int:
         out = _sz(0)

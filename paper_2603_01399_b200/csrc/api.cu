@@ -5,6 +5,7 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <algorithm>
 #include <atomic>
 #include <new>
 #include <vector>
@@ -132,6 +133,10 @@ int check_cfg(const quasar_config& c) {
   }
   if (c.weight_dtype != QUASAR_W_INT8 && c.weight_dtype != QUASAR_W_BF16) {
     set_error("config: weight_dtype %d", c.weight_dtype);
+    return QUASAR_ERR_INVALID_ARG;
+  }
+  if (c.weights_in_place && c.act_dtype != QUASAR_A_BF16) {
+    set_error("config: weights_in_place needs the persistent kernel, which handles bf16 activations only");
     return QUASAR_ERR_INVALID_ARG;
   }
   if (c.act_dtype != QUASAR_A_BF16 && !(c.act_dtype == QUASAR_A_INT8 && c.weight_dtype == QUASAR_W_INT8)) {
@@ -585,19 +590,42 @@ int quasar_model_create(const quasar_config* cfg, const quasar_weights* w, quasa
       offs.push_back(total);
       total += align_up((size_t)j.N * j.K * esz);
     }
-    cudaError_t e2 = cudaMalloc(&m->mega_weights, total);
+    // weights_in_place: the caller hands the weight buffers over to the persistent kernel - every matrix is
+    // permuted where it lies (through one scratch buffer of the largest matrix, freed again), no second copy is
+    // kept, and the kernel-per-step form, which reads the row-major layout, is switched off for this model.
+    const bool in_place = cfg->weights_in_place != 0;
+    cudaError_t e2 = cudaSuccess;
+    unsigned char* scratch = nullptr;
+    if (in_place) {
+      size_t largest = 0;
+      for (auto& j : jobs) largest = std::max(largest, align_up((size_t)j.N * j.K * esz));
+      e2 = cudaMalloc(&scratch, largest);
+    } else {
+      e2 = cudaMalloc(&m->mega_weights, total);
+    }
     if (e2 == cudaSuccess) e2 = cudaMalloc(&m->mega_jobs, jobs.size() * sizeof(MegaJob));
     if (e2 == cudaSuccess) e2 = cudaMalloc(&m->mega_layers, mls.size() * sizeof(MegaLayer));
     int rc2 = QUASAR_OK;
     if (e2 == cudaSuccess) {
       for (size_t i = 0; i < jobs.size() && rc2 == QUASAR_OK; ++i) {
-        jobs[i].wp = m->mega_weights + offs[i];
-        rc2 = launch_repack(src[i], m->mega_weights + offs[i], jobs[i].N, jobs[i].K, jobs[i].kind, cfg->weight_dtype, ncta, 0);
+        if (in_place) {
+          void* w = const_cast<void*>(src[i]);
+          jobs[i].wp = w;
+          rc2 = launch_repack(src[i], scratch, jobs[i].N, jobs[i].K, jobs[i].kind, cfg->weight_dtype, ncta, 0);
+          if (rc2 == QUASAR_OK)
+            e2 = cudaMemcpyAsync(w, scratch, (size_t)jobs[i].N * jobs[i].K * esz, cudaMemcpyDeviceToDevice, 0);
+          if (e2 != cudaSuccess) break;
+        } else {
+          jobs[i].wp = m->mega_weights + offs[i];
+          rc2 = launch_repack(src[i], m->mega_weights + offs[i], jobs[i].N, jobs[i].K, jobs[i].kind, cfg->weight_dtype, ncta, 0);
+        }
       }
-      if (rc2 == QUASAR_OK) e2 = cudaMemcpy(m->mega_jobs, jobs.data(), jobs.size() * sizeof(MegaJob), cudaMemcpyHostToDevice);
+      if (rc2 == QUASAR_OK && e2 == cudaSuccess) e2 = cudaMemcpy(m->mega_jobs, jobs.data(), jobs.size() * sizeof(MegaJob), cudaMemcpyHostToDevice);
       if (rc2 == QUASAR_OK && e2 == cudaSuccess) e2 = cudaMemcpy(m->mega_layers, mls.data(), mls.size() * sizeof(MegaLayer), cudaMemcpyHostToDevice);
       if (rc2 == QUASAR_OK && e2 == cudaSuccess) e2 = cudaStreamSynchronize(0);
     }
+    if (scratch) cudaFree(scratch);
+    if (in_place && e2 == cudaSuccess && rc2 == QUASAR_OK) m->path = 2;
     if (e2 != cudaSuccess || rc2 != QUASAR_OK) {
       if (e2 != cudaSuccess) set_error("model_create: tables of the persistent kernel (%zu bytes): %s", total, cudaGetErrorString(e2));
       quasar_model_destroy(m);
@@ -611,6 +639,10 @@ int quasar_model_create(const quasar_config* cfg, const quasar_weights* w, quasa
 
 int quasar_set_path(quasar_model* m, int32_t path) {
   if (m == nullptr || path < 0 || path > 2) { set_error("set_path: bad argument"); return QUASAR_ERR_INVALID_ARG; }
+  if (m->cfg.weights_in_place && path != 2) {
+    set_error("set_path: this model's weights were permuted in place for the persistent kernel; only path 2 exists");
+    return QUASAR_ERR_INVALID_ARG;
+  }
   m->path = path;
   return QUASAR_OK;
 }

@@ -39,7 +39,7 @@ def test_host_side_argument_errors_need_no_gpu():
     assert lib.quasar_linear_workspace_bytes(6, 4096, 4096, ctypes.byref(out)) == 0 and out.value > 0
     assert lib.quasar_linear(16, 16, 16, 0, 4, 64, 24, 16, 0, None, 16, 1 << 30, None) == -2   # K % 16 != 0
     assert lib.quasar_verify(None, None, None, None, None, 1, 1, None, None, None, None, None, 0, None, None) == -1
-    cfg = binding.Config(1, 256, 4, 2, 48, 688, 1024, 0, 1e6, 1e-6, 0, 128)  # head_dim 48 unsupported
+    cfg = binding.Config(1, 256, 4, 2, 48, 688, 1024, 0, 1e6, 1e-6, 0, 128, 0, 0)  # head_dim 48 unsupported
     w = binding.Weights()
     h = ctypes.c_void_p()
     assert lib.quasar_model_create(ctypes.byref(cfg), ctypes.byref(w), ctypes.byref(h)) == -2

@@ -365,3 +365,44 @@ def test_full_depth_qwen3_8b_both_gpu_paths_against_the_oracle(monkeypatch):
         if all(safe[q] for q in path_rows):
             assert int(buf.accept_len[0]) == int(r.accept_len[0]) and int(buf.bonus[0]) == int(r.bonus[0])
         assert 0 <= int(buf.accept_len[0]) <= 5
+
+
+def test_weights_in_place_model_occupies_the_weight_bytes_once_and_gives_the_same_pass():
+    """The offline preparation promises half the footprint of bf16 (Section 3.3).  A model created with
+    weights_in_place permutes the caller's matrices where they lie and keeps no second copy: device memory
+    grows by less than a tenth of the int8 weight bytes on creation (scratch of one matrix comes and goes),
+    the pass through the persistent kernel is bit-identical to the ordinary model's, and the kernel-per-step
+    form is refused."""
+    shape = _cut(synth.SHAPES["qwen3_8b"], 2, "qwen3_8b_2l")
+    s_max = 1040
+    get = master_getter(shape, 0, "cuda")
+    ref = binding.Model.from_master(shape, get, s_max, int8=True)
+    kk, vv = synth.kv_prefix(shape, 1, s_max, seed=1, device="cuda")
+    kv = binding.KVCache(shape, 1, s_max, k=kk, v=vv, seq_len=torch.full((1,), 1024, dtype=torch.int32, device="cuda"))
+    tokens = synth.uniform_tokens((1, 6), shape.vocab, synth.sub_seed(2, "tokens")).numpy()
+    bl = np.array([6], np.int32)
+    want, _ = _run(ref, kv, tokens, None, bl, path=2)
+    want_logits = want.logits.clone()
+    ref.close()
+    del ref
+    torch.cuda.empty_cache()
+    torch.cuda.synchronize()
+    tensors = {}
+    free0, _ = torch.cuda.mem_get_info()
+    m = binding.Model.from_master(shape, get, s_max, int8=True, weights_in_place=True)
+    torch.cuda.synchronize()
+    torch.cuda.empty_cache()
+    free1, _ = torch.cuda.mem_get_info()
+    weight_bytes = m.weight_bytes()
+    other = sum(v.numel() * v.element_size() for k, v in m.tensors.items() if not (k.endswith("_w") or k.endswith("_delta")))
+    assert free0 - free1 <= 1.1 * weight_bytes + other + (64 << 20), (free0 - free1, weight_bytes, other)
+    buf = binding.VerifyBuffers(m, 1, 6)
+    buf.tokens.copy_(torch.from_numpy(tokens))
+    binding.quasar_verify(m, kv, buf)
+    torch.cuda.synchronize()
+    assert int(buf.status[0]) == 0 and torch.equal(buf.logits, want_logits)
+    with pytest.raises(binding.QuasarError):
+        m.set_path(1)
+    big = binding.VerifyBuffers(m, 2, 6)                 # 12 rows: beyond the persistent kernel
+    with pytest.raises(binding.QuasarError):
+        binding.quasar_verify(m, binding.KVCache(shape, 2, s_max), big)
