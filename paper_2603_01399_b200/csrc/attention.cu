@@ -24,7 +24,7 @@ namespace quasar {
 namespace {
 
 constexpr int kKeyTile = 64;   // keys staged in shared memory at a time
-constexpr int kMaxWarps = 8;
+constexpr int kMaxWarps = 4;   // per CTA; three CTAs share an SM (168 registers per thread)
 constexpr float kLog2e = 1.4426950408889634f;
 
 struct AttnArgs {
@@ -42,8 +42,7 @@ struct AttnArgs {
 
 __device__ __forceinline__ void mma16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                          uint32_t b0, uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
@@ -52,6 +51,13 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t& r0, uint32_t& r1, ui
                                                   const void* smem_ptr) {
   const uint32_t addr = (uint32_t)__cvta_generic_to_shared(smem_ptr);
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"(addr));
+}
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3, const void* smem_ptr) {
+  const uint32_t addr = (uint32_t)__cvta_generic_to_shared(smem_ptr);
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
                : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
                : "r"(addr));
 }
@@ -73,7 +79,7 @@ __device__ __forceinline__ void split_bf16(float a, float b, uint32_t& hi, uint3
 }
 
 template <int D>
-__global__ void __launch_bounds__(kMaxWarps * 32) verify_attention_kernel(AttnArgs a) {
+__global__ void __launch_bounds__(kMaxWarps * 32, 3) verify_attention_kernel(AttnArgs a) {
   constexpr int kStride = D + 8;  // padded row of the staged K / V tiles (bf16 elements)
   constexpr int kDSteps = D / 16;
   // two K tiles and two V tiles: the next tile of the chunk lands (cp.async) while the current one is multiplied
@@ -157,17 +163,25 @@ __global__ void __launch_bounds__(kMaxWarps * 32) verify_attention_kernel(AttnAr
     const __nv_bfloat16* k_s = tiles + buf * 2 * kTileElems;
     const __nv_bfloat16* v_s = k_s + kTileElems;
 
-    // S = Q K^T for 16 rows x 64 keys
+    // S = Q K^T for 16 rows x 64 keys.  One ldmatrix brings the K fragments of 8 keys x 32 head dimensions;
+    // MMAs on the same accumulator are kept apart (a dependent MMA waits ~20 cycles).
     float s[kKeyTile / 8][4];
 #pragma unroll
-    for (int j = 0; j < kKeyTile / 8; ++j) {
-      s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f;
+    for (int j = 0; j < kKeyTile / 8; ++j) s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f;
+    {
+      const __nv_bfloat16* k_lane = k_s + (lane & 7) * kStride + (lane >> 3) * 8;
 #pragma unroll
-      for (int kd = 0; kd < kDSteps; ++kd) {
-        const __nv_bfloat16* kr = k_s + (8 * j + g) * kStride + kd * 16 + 2 * t;
-        const uint32_t b0 = *reinterpret_cast<const uint32_t*>(kr);
-        const uint32_t b1 = *reinterpret_cast<const uint32_t*>(kr + 8);
-        mma16816(s[j], qf[kd][0], qf[kd][1], qf[kd][2], qf[kd][3], b0, b1);
+      for (int kd2 = 0; kd2 < kDSteps / 2; ++kd2) {
+#pragma unroll
+        for (int jp = 0; jp < kKeyTile / 16; ++jp) {
+          uint32_t ka[4], kb[4];
+          ldmatrix_x4(ka[0], ka[1], ka[2], ka[3], k_lane + (16 * jp) * kStride + kd2 * 32);
+          ldmatrix_x4(kb[0], kb[1], kb[2], kb[3], k_lane + (16 * jp + 8) * kStride + kd2 * 32);
+          mma16816(s[2 * jp], qf[2 * kd2][0], qf[2 * kd2][1], qf[2 * kd2][2], qf[2 * kd2][3], ka[0], ka[1]);
+          mma16816(s[2 * jp + 1], qf[2 * kd2][0], qf[2 * kd2][1], qf[2 * kd2][2], qf[2 * kd2][3], kb[0], kb[1]);
+          mma16816(s[2 * jp], qf[2 * kd2 + 1][0], qf[2 * kd2 + 1][1], qf[2 * kd2 + 1][2], qf[2 * kd2 + 1][3], ka[2], ka[3]);
+          mma16816(s[2 * jp + 1], qf[2 * kd2 + 1][0], qf[2 * kd2 + 1][1], qf[2 * kd2 + 1][2], qf[2 * kd2 + 1][3], kb[2], kb[3]);
+        }
       }
     }
 
@@ -223,14 +237,20 @@ __global__ void __launch_bounds__(kMaxWarps * 32) verify_attention_kernel(AttnAr
       split_bf16(s[2 * kk + 1][0], s[2 * kk + 1][1], ah[2], al[2]);
       split_bf16(s[2 * kk + 1][2], s[2 * kk + 1][3], ah[3], al[3]);
 #pragma unroll
-      for (int dt = 0; dt < D / 16; ++dt) {
-        uint32_t b0, b1, b2, b3;
+      for (int dt = 0; dt < D / 16; dt += 2) {
+        uint32_t b[2][4];
         const int mat = lane >> 3, r = lane & 7;
-        ldmatrix_x4_trans(b0, b1, b2, b3, v_s + (kk * 16 + (mat & 1) * 8 + r) * kStride + dt * 16 + (mat >> 1) * 8);
-        mma16816(o[2 * dt], ah[0], ah[1], ah[2], ah[3], b0, b1);
-        mma16816(o[2 * dt], al[0], al[1], al[2], al[3], b0, b1);
-        mma16816(o[2 * dt + 1], ah[0], ah[1], ah[2], ah[3], b2, b3);
-        mma16816(o[2 * dt + 1], al[0], al[1], al[2], al[3], b2, b3);
+        const __nv_bfloat16* v_lane = v_s + (kk * 16 + (mat & 1) * 8 + r) * kStride + (mat >> 1) * 8;
+        ldmatrix_x4_trans(b[0][0], b[0][1], b[0][2], b[0][3], v_lane + dt * 16);
+        ldmatrix_x4_trans(b[1][0], b[1][1], b[1][2], b[1][3], v_lane + dt * 16 + 16);
+        mma16816(o[2 * dt], ah[0], ah[1], ah[2], ah[3], b[0][0], b[0][1]);
+        mma16816(o[2 * dt + 1], ah[0], ah[1], ah[2], ah[3], b[0][2], b[0][3]);
+        mma16816(o[2 * dt + 2], ah[0], ah[1], ah[2], ah[3], b[1][0], b[1][1]);
+        mma16816(o[2 * dt + 3], ah[0], ah[1], ah[2], ah[3], b[1][2], b[1][3]);
+        mma16816(o[2 * dt], al[0], al[1], al[2], al[3], b[0][0], b[0][1]);
+        mma16816(o[2 * dt + 1], al[0], al[1], al[2], al[3], b[0][2], b[0][3]);
+        mma16816(o[2 * dt + 2], al[0], al[1], al[2], al[3], b[1][0], b[1][1]);
+        mma16816(o[2 * dt + 3], al[0], al[1], al[2], al[3], b[1][2], b[1][3]);
       }
     }
     __syncthreads();   // every warp is done with this tile before the copy of the tile after next overwrites it
@@ -318,8 +338,8 @@ AttnPlan plan_attention(int B, int T_max, int Hq, int Hkv, int s_max) {
   p.nchunk = (s_max + chunk - 1) / chunk;
   const int R = (Hq / Hkv) * T_max;
   const int tiles = (R + 15) / 16;
-  p.warps = tiles < kMaxWarps ? tiles : kMaxWarps;
-  p.ngroups = (tiles + p.warps - 1) / p.warps;
+  p.ngroups = (tiles + kMaxWarps - 1) / kMaxWarps;
+  p.warps = (tiles + p.ngroups - 1) / p.ngroups;
   p.Rpad = p.ngroups * p.warps * 16;
   return p;
 }
@@ -356,6 +376,7 @@ int launch_attention(const __nv_bfloat16* qkv, const __nv_bfloat16* k_cache_laye
     static bool configured128 = false;
     if (!configured128) {
       QUASAR_CUDA_CHECK(cudaFuncSetAttribute(verify_attention_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem128));
+      QUASAR_CUDA_CHECK(cudaFuncSetAttribute(verify_attention_kernel<128>, cudaFuncAttributePreferredSharedMemoryCarveout, 100));
       configured128 = true;
     }
     verify_attention_kernel<128><<<grid, p.warps * 32, smem128, stream>>>(a);

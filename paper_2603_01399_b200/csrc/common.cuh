@@ -73,6 +73,12 @@ size_t umma_w8a16_scratch_bytes(int64_t M, int64_t N, int64_t K);
 int launch_umma_w8a16(const __nv_bfloat16* x, const int8_t* w, const float* dw, int64_t M, int64_t N, int64_t K, void* y,
                       bool y_is_f32, const __nv_bfloat16* residual, void* scratch, int32_t* error_word, cudaStream_t stream);
 
+// the weight-only linear layer for at most 8 rows as an exact integer contraction on tcgen05 (umma_gemm.cu)
+bool umma_rows8_usable(int64_t M, int64_t N, int64_t K);
+size_t umma_rows8_scratch_bytes(int64_t M, int64_t N, int64_t K);
+int launch_umma_rows8(const __nv_bfloat16* x, const int8_t* w, const float* dw, int64_t M, int64_t N, int64_t K, void* y,
+                      bool y_is_f32, const __nv_bfloat16* residual, void* scratch, int32_t* error_word, cudaStream_t stream);
+
 // stochastic acceptance of a chain (Section 3.1 Eq. 2-3)
 size_t accept_stochastic_workspace_bytes(int B, int T_max);
 int launch_accept_stochastic(const float* logits, const int32_t* tokens, const int32_t* block_len, const float* q_probs, int B,

@@ -22,6 +22,8 @@ namespace quasar {
 
 namespace {
 
+constexpr int64_t kRows8UmmaMinBytes = (int64_t)1 << 27;   // weight bytes from which blocks of <= 8 rows take the tcgen05 stream kernel
+
 constexpr int kWarps = 4;
 constexpr int kThreads = kWarps * 32;
 constexpr int kBlockN = kWarps * 16;  // output channels per CTA
@@ -306,6 +308,10 @@ size_t linear_workspace_bytes(int64_t M, int64_t N, int64_t K) {
     const size_t su = umma_w8a16_scratch_bytes(rows_u, N, K);
     partial = su > partial ? su : partial;
   }
+  if (M <= 8 && N * K >= kRows8UmmaMinBytes && umma_rows8_usable(M, N, K)) {
+    const size_t su = umma_rows8_scratch_bytes(M, N, K);
+    partial = su > partial ? su : partial;
+  }
   return counters + partial;
 }
 
@@ -336,6 +342,12 @@ int launch_linear(const __nv_bfloat16* x, const void* w, const float* delta, int
     }
     return QUASAR_OK;
   }
+  // A matrix of LM-head size with at most 8 rows is a long pure stream: the persistent tcgen05 kernel that feeds
+  // the int8 tiles straight into integer MMAs (activations as base-256 digits, umma_gemm.cu) sustains a higher
+  // rate than the warp-level kernel there; below that size its two extra launches cost more than it gains.
+  if (weight_dtype == QUASAR_W_INT8 && M <= 8 && N * K >= kRows8UmmaMinBytes && umma_rows8_usable(M, N, K))
+    return launch_umma_rows8(x, reinterpret_cast<const int8_t*>(w), delta, M, N, K, y, y_is_f32, residual,
+                             reinterpret_cast<unsigned char*>(workspace) + counters, status, stream);
   for (int64_t m0 = 0; m0 < M; m0 += kMaxRowsPerGemm) {
     GemmArgs a;
     a.M = (int)((M - m0) < kMaxRowsPerGemm ? (M - m0) : kMaxRowsPerGemm);

@@ -496,6 +496,199 @@ __global__ void __launch_bounds__(256) f16_rows_kernel(const __nv_bfloat16* __re
   for (int64_t k = threadIdx.x; k < K; k += 256) x16[m * K + k] = __float2half_rn(__bfloat162float(row[k]) * scale);
 }
 
+// ---- blocks of at most 8 rows: the weight-only product as an exact integer contraction -------------------
+// With so few rows the layer is a pure weight stream, and the cheapest consumer of a weight byte is one that no
+// instruction of the SM's own pipelines ever touches: the int8 tile goes from TMA straight into the integer
+// MMA (kind::i8).  The 16-bit activations enter as integers too: a row is written as fixed point against a power of
+// two above its largest magnitude,  x = q * 2^(E-21)  with |q| <= 2^21, and q as three balanced base-256 digits
+// q = d0 + 256 d1 + 65536 d2, each an int8.  A bf16 value has 8 significant bits, so every element within 2^-14 of
+// the row's maximum is represented exactly and a smaller one to 2^-22 of that maximum - far inside what an fp32
+// accumulation of the same products loses.  The digits are rows of operand B (row 4 m + j = digit j of activation
+// row m, j = 3 a zero row), the MMA adds up exact int32 sums per digit (|sum| < 2^31 for up to 2^17 contraction
+// bytes per range), and the epilogue puts them together as one 64-bit integer:
+//      y[m][n] = delta_w[n] * 2^(E_m - 21) * sum_k w[n][k] q[m][k]        (Section 3.2 Eq. 8 with X kept at 16 bits).
+// A CTA is persistent: it keeps the digit rows of one range of the contraction index (<= 2048 bytes: 64 KB)
+// resident in shared memory and streams the weight tiles of its share of the channel blocks through an
+// eight-stage ring, with two accumulators in tensor memory so that the epilogue of one channel block overlaps the
+// MMAs of the next.
+constexpr int kStagesS = 8;
+constexpr int kDigitKRange = 2048;
+constexpr int kStreamTmemCols = 64;
+
+__global__ void __launch_bounds__(256) digit_rows_kernel(const __nv_bfloat16* __restrict__ x, int64_t K, int8_t* __restrict__ xd,
+                                                         float* __restrict__ row_scale) {
+  const int64_t m = blockIdx.x;
+  const __nv_bfloat16* row = x + m * K;
+  float amax = 0.f;
+  for (int64_t k = threadIdx.x; k < K; k += 256) amax = fmaxf(amax, fabsf(__bfloat162float(row[k])));
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+  __shared__ float s_max[8];
+  if ((threadIdx.x & 31) == 0) s_max[threadIdx.x >> 5] = amax;
+  __syncthreads();
+  amax = s_max[0];
+#pragma unroll
+  for (int i = 1; i < 8; ++i) amax = fmaxf(amax, s_max[i]);
+  float up = 1.f, down = 1.f;
+  if (amax > 0.f && amax < 3.0e38f) {
+    int e;
+    (void)frexpf(amax, &e);            // amax = f * 2^e, f in [0.5, 1): |x| < 2^e along the row
+    e = e < -100 ? -100 : e;           // keeps both factors normal numbers
+    up = ldexpf(1.f, 21 - e);
+    down = ldexpf(1.f, e - 21);
+  } else if (!(amax < 3.0e38f)) {
+    down = __int_as_float(0x7fc00000);   // a row holding inf or NaN gives NaN outputs
+  }
+  if (threadIdx.x == 0) row_scale[m] = down;
+  int8_t* d0 = xd + (m * 4 + 0) * K;
+  int8_t* d1 = xd + (m * 4 + 1) * K;
+  int8_t* d2 = xd + (m * 4 + 2) * K;
+  int8_t* d3 = xd + (m * 4 + 3) * K;
+  for (int64_t k = threadIdx.x; k < K; k += 256) {
+    float v = __bfloat162float(row[k]) * up;
+    v = fminf(fmaxf(v, -2097152.f), 2097152.f);
+    const int q = __float2int_rn(v);
+    const int a0 = (int)(int8_t)(q & 0xff);
+    const int q1 = (q - a0) >> 8;
+    const int a1 = (int)(int8_t)(q1 & 0xff);
+    const int a2 = (q1 - a1) >> 8;
+    d0[k] = (int8_t)a0;
+    d1[k] = (int8_t)a1;
+    d2[k] = (int8_t)a2;
+    d3[k] = 0;
+  }
+}
+
+__global__ void __launch_bounds__(kThreadsU, 1)
+umma_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_xd, UmmaArgs a, int nb,
+                   int ctas_per_split, int ntiles) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+  constexpr int kATile = kTileN * kTileKBytes;
+  unsigned char* ring = smem;
+  unsigned char* b_res = smem + kStagesS * kATile;                        // digit rows: per 128 contraction bytes nb x 128 B
+  uint64_t* full = reinterpret_cast<uint64_t*>(b_res + (size_t)nb * a.k_per_split);
+  uint64_t* empty = full + kStagesS;
+  uint64_t* b_full = empty + kStagesS;
+  uint64_t* acc_full = b_full + 1;     // [2] the MMAs of a channel block have finished
+  uint64_t* acc_empty = acc_full + 2;  // [2] the epilogue has read the accumulator out of tensor memory
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int split = blockIdx.x / ctas_per_split, part = blockIdx.x % ctas_per_split;
+  const int t_begin = (int)((int64_t)part * ntiles / ctas_per_split);
+  const int t_end = (int)((int64_t)(part + 1) * ntiles / ctas_per_split);
+  const int k_begin = split * a.k_per_split;
+  const int k_end = min(a.K, k_begin + a.k_per_split);
+  const int nkb = (k_end - k_begin + kTileKBytes - 1) / kTileKBytes;
+
+  if (threadIdx.x == 0) {
+    *abort_flag = 0;
+    for (int s = 0; s < kStagesS; ++s) {
+      mbar_init(full + s, 1);
+      mbar_init(empty + s, 1);
+    }
+    mbar_init(b_full, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(acc_full + i, 1);
+      mbar_init(acc_empty + i, 4);   // one arrival per epilogue warp
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(tmem_slot)),
+                 "r"((uint32_t)kStreamTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {   // ---- TMA producer: the digit rows once, then the weight tiles of every channel block ----
+      mbar_expect_tx(b_full, (uint32_t)(nkb * nb * kTileKBytes));
+      for (int kb = 0; kb < nkb; ++kb)
+        tma_load_2d(b_res + (size_t)kb * nb * kTileKBytes, &map_xd, k_begin + kb * kTileKBytes, 0, b_full);
+      int s = 0;
+      uint32_t ph = 0;
+      bool ok = true;
+      for (int t = t_begin; t < t_end && ok; ++t) {
+        for (int kb = 0; kb < nkb; ++kb) {
+          if (!(ok = mbar_wait(empty + s, ph ^ 1u, abort_flag, a.error))) break;
+          mbar_expect_tx(full + s, (uint32_t)kATile);
+          tma_load_2d(ring + s * kATile, &map_w, k_begin + kb * kTileKBytes, t * kTileN, full + s);
+          if (++s == kStagesS) { s = 0; ph ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {   // ---- MMA issuer ----
+      const uint32_t idesc = umma_idesc(/*s32*/ 2, /*signed int8*/ 1, nb);
+      int s = 0;
+      uint32_t ph = 0;
+      bool ok = mbar_wait(b_full, 0, abort_flag, a.error);
+      for (int t = t_begin, it = 0; t < t_end && ok; ++t, ++it) {
+        const int buf = it & 1;
+        if (!(ok = mbar_wait(acc_empty + buf, (((uint32_t)it >> 1) & 1u) ^ 1u, abort_flag, a.error))) break;
+        asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+        const uint32_t tmem_d = tmem_base + (uint32_t)(buf * 32);
+        for (int kb = 0; kb < nkb; ++kb) {
+          if (!(ok = mbar_wait(full + s, ph, abort_flag, a.error))) break;
+          asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+          const uint64_t da = umma_desc_sw128(ring + s * kATile);
+          const uint64_t db = umma_desc_sw128(b_res + (size_t)kb * nb * kTileKBytes);
+#pragma unroll
+          for (int j = 0; j < kTileKBytes / 32; ++j)
+            umma_ss<true>(tmem_d, da + (uint64_t)(j * 2), db + (uint64_t)(j * 2), idesc, (kb > 0 || j > 0) ? 1u : 0u);
+          umma_commit(empty + s);
+          if (++s == kStagesS) { s = 0; ph ^= 1u; }
+        }
+        if (ok) umma_commit(acc_full + buf);
+      }
+    }
+  } else {
+    // ---- epilogue: warps 2..5, one output channel per thread ----
+    const int q = warp & 3;
+    for (int t = t_begin, it = 0; t < t_end; ++t, ++it) {
+      const int buf = it & 1;
+      int got = 1;
+      if (lane == 0) got = mbar_wait(acc_full + buf, ((uint32_t)it >> 1) & 1u, abort_flag, a.error) ? 1 : 0;
+      got = __shfl_sync(0xffffffffu, got, 0);
+      if (!got) break;
+      asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+      uint32_t v0[16], v1[16];
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * 32);
+      tmem_ld16(taddr, v0);
+      if (nb > 16) tmem_ld16(taddr + 16u, v1);
+      asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+      __syncwarp();
+      if (lane == 0) mbar_arrive(acc_empty + buf);     // the next channel block but one may overwrite the accumulator
+      const int n = t * kTileN + q * 32 + lane;
+      if (n < a.N) {
+#pragma unroll
+        for (int m = 0; m < 8; ++m) {
+          if (m >= a.M) continue;
+          const uint32_t* v = m < 4 ? v0 + 4 * m : v1 + 4 * (m - 4);
+          const long long total = ((long long)(int)v[2] << 16) + ((long long)(int)v[1] << 8) + (long long)(int)v[0];
+          const uint32_t bits = __float_as_uint((float)total);
+          if (a.nsplit == 1) store_output<false>(a, bits, m, n);
+          else __stcg(reinterpret_cast<uint32_t*>(a.partial) + ((size_t)split * a.Mpad + m) * a.N + n, bits);
+        }
+      }
+    }
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+  __threadfence();
+  __syncthreads();
+  if (warp == 1) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem_base), "r"((uint32_t)kStreamTmemCols)
+                 : "memory");
+  }
+}
+
 // ---- host side ------------------------------------------------------------------------------------
 PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
   static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
@@ -636,6 +829,75 @@ int launch_umma_w8a16(const __nv_bfloat16* x, const int8_t* w, const float* dw, 
     configured = true;
   }
   umma_w8a16_kernel<<<dim3(p.nblocks, p.nsplit), kThreadsU, smem, stream>>>(map_w, map_x, a);
+  QUASAR_LAUNCH_CHECK();
+  if (p.nsplit > 1) {
+    const int64_t items = M * ((N + 3) / 4);
+    umma_reduce_kernel<false><<<(unsigned)((items + 255) / 256), 256, 0, stream>>>(a);
+    QUASAR_LAUNCH_CHECK();
+  }
+  return QUASAR_OK;
+}
+
+
+// ---- weight-only form, at most 8 rows ----
+namespace {
+struct StreamPlan {
+  int nb, nsplit, k_per_split, ntiles, ctas_per_split;
+};
+StreamPlan plan_stream(int64_t M, int64_t N, int64_t K) {
+  StreamPlan p;
+  p.nb = M <= 4 ? 16 : 32;
+  const int kbs = (int)((K + kTileKBytes - 1) / kTileKBytes);
+  const int want = (int)((K + kDigitKRange - 1) / kDigitKRange);
+  const int per = (kbs + want - 1) / want;
+  p.k_per_split = per * kTileKBytes;
+  p.nsplit = (kbs + per - 1) / per;
+  p.ntiles = (int)((N + kTileN - 1) / kTileN);
+  int cps = 148 / p.nsplit;
+  cps = cps < 1 ? 1 : cps;
+  p.ctas_per_split = cps < p.ntiles ? cps : p.ntiles;
+  return p;
+}
+}  // namespace
+
+bool umma_rows8_usable(int64_t M, int64_t N, int64_t K) {
+  return M >= 1 && M <= 8 && K % 16 == 0 && N >= 1 && K <= (int64_t)148 * kDigitKRange;
+}
+
+// bytes of scratch: the digit rows, the rows' scales, partial sums of the k-ranges
+size_t umma_rows8_scratch_bytes(int64_t M, int64_t N, int64_t K) {
+  const StreamPlan p = plan_stream(M, N, K);
+  const size_t partial = p.nsplit > 1 ? (size_t)p.nsplit * (size_t)M * (size_t)N * 4 : 0;
+  return ((size_t)4 * M * K + 255) / 256 * 256 + 256 + partial;
+}
+
+int launch_umma_rows8(const __nv_bfloat16* x, const int8_t* w, const float* dw, int64_t M, int64_t N, int64_t K, void* y,
+                      bool y_is_f32, const __nv_bfloat16* residual, void* scratch, int32_t* error_word, cudaStream_t stream) {
+  unsigned char* sc = reinterpret_cast<unsigned char*>(scratch);
+  int8_t* xd = reinterpret_cast<int8_t*>(sc);
+  float* row_scale = reinterpret_cast<float*>(sc + ((size_t)4 * M * K + 255) / 256 * 256);
+  void* partial = sc + ((size_t)4 * M * K + 255) / 256 * 256 + 256;
+  digit_rows_kernel<<<(unsigned)M, 256, 0, stream>>>(x, K, xd, row_scale);
+  QUASAR_LAUNCH_CHECK();
+  const StreamPlan p = plan_stream(M, N, K);
+  CUtensorMap map_w, map_xd;
+  int rc = make_map(&map_w, w, (uint64_t)N, (uint64_t)K, kTileN);
+  if (rc != QUASAR_OK) return rc;
+  rc = make_map(&map_xd, xd, (uint64_t)(4 * M), (uint64_t)K, (uint32_t)p.nb);
+  if (rc != QUASAR_OK) return rc;
+  UmmaArgs a;
+  a.dx = row_scale; a.dw = dw; a.y = y; a.res = residual; a.acc_out = nullptr; a.partial = partial; a.counters = nullptr;
+  a.error = error_word;
+  a.M = (int)M; a.Mpad = (int)M; a.N = (int)N; a.K = (int)K; a.k_per_split = p.k_per_split; a.nsplit = p.nsplit;
+  a.y_is_f32 = y_is_f32 ? 1 : 0;
+  const size_t smem = (size_t)kStagesS * kTileN * kTileKBytes + (size_t)p.nb * p.k_per_split + 256 + 1024;
+  static bool configured = false;
+  if (!configured) {
+    QUASAR_CUDA_CHECK(cudaFuncSetAttribute(umma_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+    configured = true;
+  }
+  umma_stream_kernel<<<(unsigned)(p.nsplit * p.ctas_per_split), kThreadsU, smem, stream>>>(map_w, map_xd, a, p.nb,
+                                                                                         p.ctas_per_split, p.ntiles);
   QUASAR_LAUNCH_CHECK();
   if (p.nsplit > 1) {
     const int64_t items = M * ((N + 3) / 4);

@@ -135,6 +135,35 @@ def test_linear_exact_integer_case():
     assert torch.equal(y.cpu().to(torch.int64), want)
 
 
+@pytest.mark.parametrize("m", [1, 4, 5, 8])
+def test_linear_long_stream_with_ragged_tails_is_an_exact_integer_contraction(m):
+    """Matrices of LM-head size with at most 8 rows run as an integer contraction on tcgen05 (the activations as
+    three base-256 digits against a power of two above the row maximum).  With integer activations and unit step
+    sizes the result must be the integer product bit for bit - on a shape whose channel count and contraction
+    length both leave a partial tile - and with ordinary inputs it must agree with the oracle to fp32 rounding."""
+    n, k = 33000, 4112                                  # 135.7 MB of weights; 33000 = 257 * 128 + 104, 4112 = 32 * 128 + 16
+    g = torch.Generator().manual_seed(7 + m)
+    x = torch.randint(-4, 5, (m, k), generator=g).to(torch.bfloat16).cuda()
+    q = torch.randint(-127, 128, (n, k), generator=g, dtype=torch.int8).cuda()
+    d = torch.ones(n, dtype=torch.float32, device="cuda")
+    y = binding.quasar_linear(x, q, d, out_f32=True)
+    rows = np.unique(np.concatenate([np.arange(0, 130), np.arange(n - 130, n), np.random.default_rng(m).integers(0, n, 256)]))
+    want = x.cpu().to(torch.int64) @ q[torch.from_numpy(rows).cuda()].cpu().to(torch.int64).T
+    assert torch.equal(y.cpu()[:, torch.from_numpy(rows)].to(torch.int64), want)
+    # ordinary inputs, one row scaled far below the others (its digits use the same 21 bits against its own maximum)
+    x = synth.normal_bf16((m, k), 1.0, seed=m, device="cuda")
+    x[m - 1] = (x[m - 1].float() * 2.0 ** -20).to(torch.bfloat16)
+    wq, wd = binding.quasar_quantize(synth.normal_bf16((n, k), 0.02, seed=3, device="cuda"))
+    y = binding.quasar_linear(x, wq, wd, out_f32=True)
+    oq = wq[torch.from_numpy(rows).cuda()].cpu().numpy()
+    od = wd.cpu().numpy()[rows]
+    xo = qo.bf16_bits_to_f64(_bits(x))
+    want = qo.linear(xo, oq, od)
+    absw = qo.linear(np.abs(xo), np.abs(oq.astype(np.int16)).astype(np.float64), od)
+    got = y.cpu().numpy()[:, rows].astype(np.float64)
+    assert np.all(np.abs(got - want) <= 1e-6 * absw + 2e-7 * np.abs(want))
+
+
 def test_linear_is_run_to_run_identical():
     x = synth.normal_bf16((6, 4096), 1.0, seed=1, device="cuda")
     q, d = binding.quasar_quantize(synth.normal_bf16((4096, 4096), 0.02, seed=2, device="cuda"))
