@@ -317,14 +317,19 @@ __global__ void __launch_bounds__(256) umma_reduce_kernel(UmmaArgs a) {
 // ---- the weight-only form (int8 weights, 16-bit activations) on the same tensor cores -------------------
 // kind::f16 takes both operands as fp16.  The activations are turned into fp16 once per call by a
 // small pre-pass (exact: a bf16 value times a power of two that puts the row's maximum in [2^14, 2^15) is
-// an fp16 value unless it lies 2^-39 below that maximum), the weights per stage by four converter warps:
-// a stage's 128 rows x 64 contraction bytes land by TMA (64-byte swizzle), thread r turns row r into 64
-// fp16 values - the byte with its sign bit flipped under the high byte 0x64 reads 1024 + (w + 128), one
-// packed subtraction of 1152 leaves w - and stores them as row r of a K-major tile with the 128-byte
-// swizzle the MMA expects.  Per stage: raw weights 8 KB, fp16 weights 16 KB, activations Mpad x 128 B.
-constexpr int kStagesF16 = 3;
+// an fp16 value unless it lies 2^-39 below that maximum).  The weights never exist as a 16-bit tile in shared
+// memory: operand A of the MMA is read from TENSOR memory.  A stage's 128 rows x 64 contraction bytes land by
+// TMA (64-byte swizzle); thread r of the four converter warps turns row r into 64 fp16 values in registers -
+// the byte with its sign bit flipped under the high byte 0x64 reads 1024 + (w + 128), one packed subtraction
+// of 1152 leaves w - and stores them with one tcgen05.st into lane r of the stage's 32 tensor-memory columns
+// (two fp16 per column, contraction index ascending).  Per stage the shared memory holds the raw weights
+// (8 KB) and the activations (Mpad x 128 B) only, which is what lets five stages of two CTAs fit an SM: the
+// kernel's speed is set by the bytes it keeps in flight.
+constexpr int kStagesF16 = 5;
 constexpr int kRawBytes = kTileN * 64;          // 8 KB
-constexpr int kConvBytes = kTileN * 128;        // 16 KB
+constexpr int kAColsPerStage = 32;              // 64 fp16 per row
+constexpr int kAccCols = 96;                    // accumulator columns (Mpad <= 80), then kStagesF16 x 32 columns of A
+constexpr int kTmemColsF16 = 256;
 
 __device__ __forceinline__ void s8x4_to_f16x4(uint32_t w, uint32_t& lo, uint32_t& hi) {
   const uint32_t u = w ^ 0x80808080u;
@@ -337,15 +342,37 @@ __device__ __forceinline__ void s8x4_to_f16x4(uint32_t w, uint32_t& lo, uint32_t
   hi = *reinterpret_cast<const uint32_t*>(&hi2);
 }
 
+// 32 consecutive columns of this thread's tensor-memory lane
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,"
+      "%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};\n" ::"r"(taddr),
+      "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]), "r"(v[9]), "r"(v[10]),
+      "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]), "r"(v[16]), "r"(v[17]), "r"(v[18]), "r"(v[19]), "r"(v[20]),
+      "r"(v[21]), "r"(v[22]), "r"(v[23]), "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]),
+      "r"(v[31])
+      : "memory");
+  asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory");
+}
+
+// D[tmem] (+)= A[tmem] * B[smem descriptor], fp16 x fp16 -> fp32
+__device__ __forceinline__ void umma_ts_f16(uint32_t tmem_d, uint32_t tmem_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}\n" ::"r"(tmem_d),
+      "r"(tmem_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
 __global__ void __launch_bounds__(kThreadsU, 2)
 umma_w8a16_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, UmmaArgs a) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   const int b_bytes = a.Mpad * 128;                               // Mpad rows x 64 fp16
-  const int stage_bytes = kConvBytes + b_bytes + kRawBytes;       // [fp16 weights][activations][raw weights]
+  const int stage_bytes = b_bytes + kRawBytes;                    // [activations][raw weights]
   unsigned char* tiles = smem;
   uint64_t* full = reinterpret_cast<uint64_t*>(smem + kStagesF16 * stage_bytes);   // TMA landed (raw weights + activations)
-  uint64_t* conv = full + kStagesF16;                                              // fp16 weight tile written
+  uint64_t* conv = full + kStagesF16;                                              // fp16 weights stored to tensor memory
   uint64_t* empty = conv + kStagesF16;                                             // MMAs of the stage done
   uint64_t* accum_done = empty + kStagesF16;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(accum_done + 1);
@@ -368,7 +395,8 @@ umma_w8a16_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_consta
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(tmem_slot)), "r"(128u)
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(tmem_slot)),
+                 "r"((uint32_t)kTmemColsF16)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
   }
@@ -385,8 +413,8 @@ umma_w8a16_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_consta
         if (!mbar_wait(empty + s, ph ^ 1u, abort_flag, a.error)) break;
         unsigned char* st = tiles + s * stage_bytes;
         mbar_expect_tx(full + s, (uint32_t)(kRawBytes + b_bytes));
-        tma_load_2d(st + kConvBytes + b_bytes, &map_w, k_begin + kb * 64, n0, full + s);          // 128 rows x 64 int8
-        tma_load_2d(st + kConvBytes, &map_x, (k_begin + kb * 64) * 2, 0, full + s);               // Mpad rows x 64 fp16 (byte coordinate)
+        tma_load_2d(st + b_bytes, &map_w, k_begin + kb * 64, n0, full + s);                       // 128 rows x 64 int8
+        tma_load_2d(st, &map_x, (k_begin + kb * 64) * 2, 0, full + s);                            // Mpad rows x 64 fp16 (byte coordinate)
         if (++s == kStagesF16) { s = 0; ph ^= 1u; }
       }
     }
@@ -399,19 +427,22 @@ umma_w8a16_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_consta
       for (int kb = 0; kb < nkb && ok; ++kb) {
         if (!(ok = mbar_wait(conv + s, ph, abort_flag, a.error))) break;    // (the converters waited for the stage's TMA)
         asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-        const unsigned char* st = tiles + s * stage_bytes;
-        const uint64_t da = umma_desc_sw128(st), db = umma_desc_sw128(st + kConvBytes);
+        const uint64_t db = umma_desc_sw128(tiles + s * stage_bytes);
+        const uint32_t ta = tmem_base + (uint32_t)(kAccCols + s * kAColsPerStage);
 #pragma unroll
-        for (int j = 0; j < 4; ++j)   // one instruction contracts 16 fp16 values: 32 bytes further along the row
-          umma_ss<false>(tmem_base, da + (uint64_t)(j * 2), db + (uint64_t)(j * 2), idesc, (kb > 0 || j > 0) ? 1u : 0u);
+        for (int j = 0; j < 4; ++j)   // one instruction contracts 16 fp16 values: 8 columns of A, 32 bytes further along B's rows
+          umma_ts_f16(tmem_base, ta + (uint32_t)(j * 8), db + (uint64_t)(j * 2), idesc, (kb > 0 || j > 0) ? 1u : 0u);
         umma_commit(empty + s);
         if (++s == kStagesF16) { s = 0; ph ^= 1u; }
       }
       if (ok) umma_commit(accum_done);
     }
   } else {
-    // ---- converters, then the epilogue: warps 2..5, thread r = weight row r of the tile ----
-    const int r = (warp - 2) * 32 + lane;
+    // ---- converters, then the epilogue: warps 2..5; a warp may touch the tensor-memory lanes 32 (warp % 4) .. + 31,
+    //      so thread (q, lane) takes weight row r = 32 q + lane of the tile ----
+    const int q = warp & 3;
+    const int r = q * 32 + lane;
+    const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
     int s = 0;
     uint32_t ph = 0;
     bool ok = true;
@@ -420,27 +451,23 @@ umma_w8a16_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_consta
       if (lane == 0) got = mbar_wait(full + s, ph, abort_flag, a.error) ? 1 : 0;
       got = __shfl_sync(0xffffffffu, got, 0);
       if (!got) { ok = false; break; }
-      unsigned char* st = tiles + s * stage_bytes;
-      const unsigned char* raw = st + kConvBytes + b_bytes + r * 64;          // 64-byte swizzle: piece c sits at c ^ ((r >> 1) & 3)
-      unsigned char* dst = st + (r >> 3) * 1024 + (r & 7) * 128;              // 128-byte swizzle: piece c sits at c ^ (r & 7)
+      const unsigned char* raw = tiles + s * stage_bytes + b_bytes + r * 64;   // 64-byte swizzle: piece c sits at c ^ ((r >> 1) & 3)
+      uint32_t v[32];
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
         const uint4 w = *reinterpret_cast<const uint4*>(raw + ((c ^ ((r >> 1) & 3)) << 4));
-        uint4 o0, o1;
-        s8x4_to_f16x4(w.x, o0.x, o0.y);
-        s8x4_to_f16x4(w.y, o0.z, o0.w);
-        s8x4_to_f16x4(w.z, o1.x, o1.y);
-        s8x4_to_f16x4(w.w, o1.z, o1.w);
-        *reinterpret_cast<uint4*>(dst + (((2 * c) ^ (r & 7)) << 4)) = o0;
-        *reinterpret_cast<uint4*>(dst + (((2 * c + 1) ^ (r & 7)) << 4)) = o1;
+        s8x4_to_f16x4(w.x, v[8 * c + 0], v[8 * c + 1]);
+        s8x4_to_f16x4(w.y, v[8 * c + 2], v[8 * c + 3]);
+        s8x4_to_f16x4(w.z, v[8 * c + 4], v[8 * c + 5]);
+        s8x4_to_f16x4(w.w, v[8 * c + 6], v[8 * c + 7]);
       }
-      asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");   // the tensor core reads what these threads wrote
+      tmem_st32(tmem_base + lane_addr + (uint32_t)(kAccCols + s * kAColsPerStage), v);
+      asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
       __syncwarp();
       if (lane == 0) mbar_arrive(conv + s);
       if (++s == kStagesF16) { s = 0; ph ^= 1u; }
     }
-    const int q = warp & 3;
-    const int n = n0 + q * 32 + lane;
+    const int n = n0 + r;
     int got = ok ? 1 : 0;
     if (ok && lane == 0) got = mbar_wait(accum_done, 0, abort_flag, a.error) ? 1 : 0;
     got = __shfl_sync(0xffffffffu, got, 0);
@@ -448,7 +475,7 @@ umma_w8a16_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_consta
       asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
       for (int c0 = 0; c0 < a.Mpad; c0 += 16) {
         uint32_t v[16];
-        tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
+        tmem_ld16(tmem_base + lane_addr + (uint32_t)c0, v);
         if (n < a.N) {
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
@@ -465,7 +492,8 @@ umma_w8a16_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_consta
   __threadfence();
   __syncthreads();
   if (warp == 1) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem_base), "r"(128u) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem_base), "r"((uint32_t)kTmemColsF16)
+                 : "memory");
   }
 }
 
@@ -822,7 +850,7 @@ int launch_umma_w8a16(const __nv_bfloat16* x, const int8_t* w, const float* dw, 
   a.error = error_word;
   a.M = (int)M; a.Mpad = mpad; a.N = (int)N; a.K = (int)K; a.k_per_split = p.k_per_split; a.nsplit = p.nsplit;
   a.y_is_f32 = y_is_f32 ? 1 : 0;
-  const size_t smem = (size_t)kStagesF16 * (kConvBytes + mpad * 128 + kRawBytes) + 256 + 1024;
+  const size_t smem = (size_t)kStagesF16 * (mpad * 128 + kRawBytes) + 256 + 1024;
   static bool configured = false;
   if (!configured) {
     QUASAR_CUDA_CHECK(cudaFuncSetAttribute(umma_w8a16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 112 * 1024));
