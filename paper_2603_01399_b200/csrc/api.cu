@@ -68,7 +68,7 @@ size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
 
 // Layout of the verify workspace; every offset is a multiple of 256 bytes.
 struct Workspace {
-  size_t x, h, qkv, attn, gu, act, attn16, act16, logits, top1, anc, depth, valid, lin, att, cand, ss_part, amax, attn_count, barrier, total;
+  size_t x, h, qkv, attn, gu, act, attn16, act16, h16, inv3, keys, logits, top1, anc, depth, valid, lin, att, cand, ss_part, amax, attn_count, barrier, total;
   size_t lin_bytes, att_bytes;
 };
 
@@ -88,6 +88,9 @@ Workspace layout(const quasar_config& c, int B, int T_max, int s_max) {
   w.act = take(M * (size_t)c.ffn * 2);
   w.attn16 = take(M * (size_t)c.n_q_heads * c.head_dim * 2);
   w.act16 = take(M * (size_t)c.ffn * 2);
+  w.h16 = take(M * (size_t)c.hidden * 2);
+  w.inv3 = take(3 * align_up(M * 4));
+  w.keys = take(M * 8);
   w.logits = take(M * (size_t)c.vocab * 4);
   w.top1 = take(M * 4);
   w.anc = take(M * 8);
@@ -300,6 +303,69 @@ int verify_impl(quasar_model* m, const quasar_kv* kv, const int32_t* tokens, con
   TRY(launch_embed(tokens, reinterpret_cast<const __nv_bfloat16*>(m->w.embed), M, H, c.vocab, x, stream));
   TRY(tr.put(x, (size_t)M * H * 2));
 
+  // Blocks of 9..80 rows with int8 weights and 16-bit activations: every linear layer is the tcgen05 kernel, which
+  // wants its operand as fp16 rows times a power of two.  The kernel that produces an operand writes that form too, and
+  // the kernel after a residual linear layer adds up its k-ranges, so a layer is 12 launches instead of 17.
+  bool fused = !a8 && wd == QUASAR_W_INT8 && M > 8 && M <= 80;
+  {
+    const int64_t shapes[5][2] = {{qkv_w, H}, {H, (int64_t)Hq * D}, {2 * (int64_t)F, H}, {H, F}, {c.vocab, H}};
+    for (auto& sh : shapes) fused = fused && umma_w8a16_usable(M, sh[0], sh[1]);
+  }
+  if (fused) {
+    void* h16 = wsp + ws.h16;
+    void* attn16 = wsp + ws.attn16;
+    void* act16 = wsp + ws.act16;
+    float* inv_h = reinterpret_cast<float*>(wsp + ws.inv3);
+    float* inv_a = reinterpret_cast<float*>(wsp + ws.inv3 + align_up((size_t)M * 4));
+    float* inv_f = reinterpret_cast<float*>(wsp + ws.inv3 + 2 * align_up((size_t)M * 4));
+    float* partial = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(lin) + 65536);
+    auto norm_of = [&](int l) {
+      return reinterpret_cast<const __nv_bfloat16*>(l < c.n_layers ? m->layers[l].attn_norm : m->w.final_norm);
+    };
+    TRY(launch_rmsnorm_f16(x, norm_of(0), M, H, c.rms_eps, h, h16, inv_h, stream));
+    for (int l = 0; l < c.n_layers; ++l) {
+      const quasar_layer_weights& L = m->layers[l];
+      __nv_bfloat16* kc = reinterpret_cast<__nv_bfloat16*>(kv->k) + (size_t)l * layer_stride;
+      __nv_bfloat16* vc = reinterpret_cast<__nv_bfloat16*>(kv->v) + (size_t)l * layer_stride;
+      int ns = 1, mpad = 16;
+      TRY(tr.put(h, (size_t)M * H * 2));
+      TRY(launch_umma_w8a16_prepared(h16, inv_h, reinterpret_cast<const int8_t*>(L.qkv_w), L.qkv_delta, M, qkv_w, H, qkv, false,
+                                     nullptr, partial, true, status, stream));
+      TRY(tr.put(qkv, (size_t)M * qkv_w * 2));
+      TRY(launch_rope_append(qkv, reinterpret_cast<const __nv_bfloat16*>(c.qk_norm ? L.q_norm : nullptr),
+                             reinterpret_cast<const __nv_bfloat16*>(c.qk_norm ? L.k_norm : nullptr), m->rope_table,
+                             kv->seq_len, block_len, bi, B, T_max, Hq, Hkv, D, c.rms_eps, kc, vc, kv->s_max, stream));
+      TRY(tr.put(qkv, (size_t)M * qkv_w * 2));
+      TRY(launch_attention(qkv, kc, vc, kv->seq_len, block_len, bi, B, T_max, Hq, Hkv, D, kv->s_max, attn, att,
+                           ws.att_bytes, stream));
+      TRY(tr.put(attn, (size_t)M * Hq * D * 2));
+      TRY(launch_f16_rows(attn, M, (int64_t)Hq * D, attn16, inv_a, stream));
+      TRY(launch_umma_w8a16_prepared(attn16, inv_a, reinterpret_cast<const int8_t*>(L.o_w), L.o_delta, M, H, (int64_t)Hq * D, x,
+                                     false, x, partial, false, status, stream));
+      umma_w8a16_plan(M, H, (int64_t)Hq * D, &ns, &mpad);
+      TRY(launch_reduce_residual_rmsnorm_f16(partial, ns, mpad, inv_a, L.o_delta, x,
+                                             reinterpret_cast<const __nv_bfloat16*>(L.mlp_norm), M, H, c.rms_eps, h, h16, inv_h,
+                                             stream));
+      TRY(tr.put(x, (size_t)M * H * 2));
+      TRY(launch_umma_w8a16_prepared(h16, inv_h, reinterpret_cast<const int8_t*>(L.gateup_w), L.gateup_delta, M, 2 * (int64_t)F, H,
+                                     gu, false, nullptr, partial, true, status, stream));
+      TRY(launch_swiglu_f16(gu, M, F, act, act16, inv_f, stream));
+      TRY(tr.put(act, (size_t)M * F * 2));
+      TRY(launch_umma_w8a16_prepared(act16, inv_f, reinterpret_cast<const int8_t*>(L.down_w), L.down_delta, M, H, F, x, false, x,
+                                     partial, false, status, stream));
+      umma_w8a16_plan(M, H, F, &ns, &mpad);
+      TRY(launch_reduce_residual_rmsnorm_f16(partial, ns, mpad, inv_f, L.down_delta, x, norm_of(l + 1), M, H, c.rms_eps, h, h16,
+                                             inv_h, stream));
+      TRY(tr.put(x, (size_t)M * H * 2));
+    }
+    TRY(tr.put(h, (size_t)M * H * 2));
+    TRY(launch_umma_w8a16_prepared(h16, inv_h, reinterpret_cast<const int8_t*>(m->w.lm_w), m->w.lm_delta, M, c.vocab, H, logits,
+                                   true, nullptr, partial, true, status, stream));
+    TRY(launch_argmax(logits, M, c.vocab, top1, reinterpret_cast<unsigned long long*>(wsp + ws.keys), stream));
+    TRY(launch_accept(tokens, parents, block_len, top1, bi, B, T_max, accept_len, bonus, accept_path, stream));
+    return QUASAR_OK;
+  }
+
   for (int l = 0; l < c.n_layers; ++l) {
     const quasar_layer_weights& L = m->layers[l];
     __nv_bfloat16* kc = reinterpret_cast<__nv_bfloat16*>(kv->k) + (size_t)l * layer_stride;
@@ -327,7 +393,7 @@ int verify_impl(quasar_model* m, const quasar_kv* kv, const int32_t* tokens, con
   TRY(launch_rmsnorm(x, reinterpret_cast<const __nv_bfloat16*>(m->w.final_norm), M, H, c.rms_eps, h, stream));
   TRY(tr.put(h, (size_t)M * H * 2));
   TRY(linear(h, m->w.lm_w, m->w.lm_delta, m->w.lm_smooth, c.vocab, H, logits, true, nullptr));
-  TRY(launch_argmax(logits, M, c.vocab, top1, stream));
+  TRY(launch_argmax(logits, M, c.vocab, top1, reinterpret_cast<unsigned long long*>(wsp + ws.keys), stream));
   TRY(launch_accept(tokens, parents, block_len, top1, bi, B, T_max, accept_len, bonus, accept_path, stream));
   return QUASAR_OK;
 }

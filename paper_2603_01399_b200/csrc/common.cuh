@@ -33,6 +33,21 @@ void count_launch(int n = 1);
 
 static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+#ifdef __CUDACC__
+// The fp16 form of an activation row for the tcgen05 weight-only GEMM: the row times the power of two that puts
+// its largest magnitude in [2^14, 2^15), and the inverse of that power (exact both ways).
+__device__ __forceinline__ void f16_row_scale(float amax, float& scale, float& inv) {
+  scale = 1.f;
+  inv = 1.f;
+  if (amax > 0.f && amax < 3.0e38f) {
+    int e;
+    (void)frexpf(amax, &e);            // amax = f * 2^e, f in [0.5, 1)
+    scale = ldexpf(1.f, 15 - e);
+    inv = ldexpf(1.f, e - 15);
+  }
+}
+#endif
+
 constexpr int kMaxRowsPerGemm = 72;  // rows one skinny-GEMM launch handles (9 MMA column tiles)
 
 // ---- launchers (each only enqueues work on `stream`) -------------------------------------------
@@ -72,6 +87,14 @@ bool umma_w8a16_usable(int64_t M, int64_t N, int64_t K);
 size_t umma_w8a16_scratch_bytes(int64_t M, int64_t N, int64_t K);
 int launch_umma_w8a16(const __nv_bfloat16* x, const int8_t* w, const float* dw, int64_t M, int64_t N, int64_t K, void* y,
                       bool y_is_f32, const __nv_bfloat16* residual, void* scratch, int32_t* error_word, cudaStream_t stream);
+// the same in pieces, for a pass that lets the producer of the activations write their fp16 form and the consumer of
+// the result add up the k-ranges (api.cu)
+void umma_w8a16_plan(int64_t M, int64_t N, int64_t K, int* nsplit, int* mpad);
+size_t umma_w8a16_partial_bytes(int64_t M, int64_t N, int64_t K);
+int launch_f16_rows(const __nv_bfloat16* x, int64_t M, int64_t K, void* x16, float* inv_scale, cudaStream_t stream);
+int launch_umma_w8a16_prepared(const void* x16, const float* inv, const int8_t* w, const float* dw, int64_t M, int64_t N,
+                               int64_t K, void* y, bool y_is_f32, const __nv_bfloat16* residual, void* partial, bool finalize,
+                               int32_t* error_word, cudaStream_t stream);
 
 // the weight-only linear layer for at most 8 rows as an exact integer contraction on tcgen05 (umma_gemm.cu)
 bool umma_rows8_usable(int64_t M, int64_t N, int64_t K);
@@ -126,7 +149,19 @@ int launch_attention(const __nv_bfloat16* qkv, const __nv_bfloat16* k_cache_laye
 
 int launch_swiglu(const __nv_bfloat16* gu, int M, int F, __nv_bfloat16* act, cudaStream_t stream);
 
-int launch_argmax(const float* logits, int M, int V, int32_t* top1, cudaStream_t stream);
+// Fused forms for the pass whose linear layers take a prepared fp16 operand (umma_gemm.cu): each also writes the
+// fp16 form of its output rows (x16 [M][width] + inv [M]).
+int launch_rmsnorm_f16(const __nv_bfloat16* x, const __nv_bfloat16* g, int M, int H, float eps, __nv_bfloat16* y, void* y16,
+                       float* inv, cudaStream_t stream);
+int launch_swiglu_f16(const __nv_bfloat16* gu, int M, int F, __nv_bfloat16* act, void* act16, float* inv, cudaStream_t stream);
+// x += bf16(dw * dx * sum of the k-range partial sums) (the epilogue of a residual linear layer), then y = RMSNorm(x) * g
+// with its fp16 form: one kernel in place of the split-K reduction, the norm and the operand pre-pass
+int launch_reduce_residual_rmsnorm_f16(const float* partial, int nsplit, int mpad, const float* dx, const float* dw,
+                                       __nv_bfloat16* x, const __nv_bfloat16* g, int M, int H, float eps, __nv_bfloat16* y,
+                                       void* y16, float* inv, cudaStream_t stream);
+
+// keys: M x 8 bytes of scratch
+int launch_argmax(const float* logits, int M, int V, int32_t* top1, unsigned long long* keys, cudaStream_t stream);
 
 int launch_accept(const int32_t* tokens, const int32_t* parents, const int32_t* block_len, const int32_t* top1,
                   BlockInfo bi, int B, int T_max, int32_t* accept_len, int32_t* bonus, int32_t* accept_path,

@@ -5,6 +5,8 @@
 // bf16 storage.
 #include <math.h>
 
+#include <cuda_fp16.h>
+
 #include "common.cuh"
 
 namespace quasar {
@@ -93,6 +95,95 @@ rmsnorm_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restr
   }
 }
 
+// One thread block per activation row would leave half the SMs idle and every thread with a long chain of
+// dependent round trips to L2, so these row kernels run 1024 threads per row.
+constexpr int kRowThreads = 1024;
+
+// block-wide maximum of non-negative values
+__device__ __forceinline__ float block_max_rows(float v, float* s_buf) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) s_buf[threadIdx.x >> 5] = v;
+  __syncthreads();
+  float r = s_buf[0];
+#pragma unroll
+  for (int i = 1; i < kRowThreads / 32; ++i) r = fmaxf(r, s_buf[i]);
+  return r;
+}
+
+// fp16 form of the row a thread block has just written as bf16 (every thread re-reads the pairs it wrote itself)
+__device__ __forceinline__ void write_f16_row(const __nv_bfloat16* y_row, int width, float amax, __half* y16_row, float* inv_out) {
+  float scale, inv;
+  f16_row_scale(amax, scale, inv);
+  if (threadIdx.x == 0) *inv_out = inv;
+  const __nv_bfloat162* yr = reinterpret_cast<const __nv_bfloat162*>(y_row);
+  __half2* hr = reinterpret_cast<__half2*>(y16_row);
+  for (int i = threadIdx.x; i < width / 2; i += blockDim.x) {
+    const float2 f = __bfloat1622float2(yr[i]);
+    hr[i] = __floats2half2_rn(f.x * scale, f.y * scale);
+  }
+}
+
+// ---- RMSNorm that also leaves the fp16 form of its output; optionally preceded by the epilogue of a residual linear
+//      layer whose k-range partial sums it adds up (REDUCE) ---------------------------------------------------------
+template <bool REDUCE>
+__global__ void __launch_bounds__(kRowThreads)
+rmsnorm_f16_kernel(const float* __restrict__ partial, int nsplit, int mpad, const float* __restrict__ dx,
+                   const float* __restrict__ dw, __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ g, int H,
+                   float eps, __nv_bfloat16* __restrict__ y, __half* __restrict__ y16, float* __restrict__ inv) {
+  const int m = blockIdx.x;
+  __nv_bfloat162* xr = reinterpret_cast<__nv_bfloat162*>(x + (size_t)m * H);
+  const __nv_bfloat162* gr = reinterpret_cast<const __nv_bfloat162*>(g);
+  __nv_bfloat162* yr = reinterpret_cast<__nv_bfloat162*>(y + (size_t)m * H);
+  __shared__ float s_part[kRowThreads / 32];
+  float ss = 0.f;
+  if (REDUCE) {
+    const float dxm = dx[m];
+    const size_t split_stride = (size_t)mpad * H;
+    const float* p0 = partial + (size_t)m * H;
+    for (int i = threadIdx.x; i < H / 2; i += blockDim.x) {
+      float2 acc = make_float2(0.f, 0.f);
+      for (int s = 0; s < nsplit; ++s) {   // k-ranges in ascending order
+        const float2 v = __ldcg(reinterpret_cast<const float2*>(p0 + (size_t)s * split_stride) + i);
+        acc.x += v.x;
+        acc.y += v.y;
+      }
+      const float2 d = *reinterpret_cast<const float2*>(dw + 2 * i);
+      const float2 r = __bfloat1622float2(xr[i]);
+      const float v0 = __bfloat162float(__float2bfloat16_rn((acc.x * dxm) * d.x)) + r.x;
+      const float v1 = __bfloat162float(__float2bfloat16_rn((acc.y * dxm) * d.y)) + r.y;
+      const __nv_bfloat162 o = __floats2bfloat162_rn(v0, v1);
+      xr[i] = o;
+      const float2 f = __bfloat1622float2(o);
+      ss += f.x * f.x + f.y * f.y;
+    }
+  } else {
+    for (int i = threadIdx.x; i < H / 2; i += blockDim.x) {
+      const float2 f = __bfloat1622float2(xr[i]);
+      ss += f.x * f.x + f.y * f.y;
+    }
+  }
+  ss = warp_sum(ss);
+  if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = ss;
+  __syncthreads();
+  float tot = 0.f;
+#pragma unroll
+  for (int i = 0; i < kRowThreads / 32; ++i) tot += s_part[i];
+  const float r = 1.0f / sqrtf(tot / (float)H + eps);
+  float amax = 0.f;
+  for (int i = threadIdx.x; i < H / 2; i += blockDim.x) {
+    const float2 f = __bfloat1622float2(xr[i]);
+    const float2 gg = __bfloat1622float2(gr[i]);
+    const __nv_bfloat162 o = __floats2bfloat162_rn(f.x * r * gg.x, f.y * r * gg.y);
+    yr[i] = o;
+    const float2 of = __bfloat1622float2(o);
+    amax = fmaxf(amax, fmaxf(fabsf(of.x), fabsf(of.y)));
+  }
+  amax = block_max_rows(amax, s_part);
+  write_f16_row(y + (size_t)m * H, H, amax, y16 + (size_t)m * H, inv + m);
+}
+
 // ---- RoPE table: cos/sin(pos * theta^(-2i/D)) evaluated in fp64, stored as fp32 -------------
 __global__ void rope_table_kernel(float2* table, int max_pos, int D, double theta) {
   const int half = D / 2;
@@ -174,38 +265,83 @@ __global__ void swiglu_kernel(const __nv_bfloat16* __restrict__ gu, int F, __nv_
   reinterpret_cast<__nv_bfloat162*>(act + (size_t)m * F)[f2] = __floats2bfloat162_rn(a0, a1);
 }
 
-// ---- arg-max over the vocabulary, lowest index on ties ---------------------------------------
-__global__ void __launch_bounds__(1024) argmax_kernel(const float* __restrict__ logits, int V, int32_t* top1) {
+// the same, one thread block per row, leaving the fp16 form of the row as well
+__global__ void __launch_bounds__(kRowThreads)
+swiglu_f16_kernel(const __nv_bfloat16* __restrict__ gu, int F, __nv_bfloat16* __restrict__ act, __half* __restrict__ act16,
+                  float* __restrict__ inv) {
   const int m = blockIdx.x;
+  const __nv_bfloat162* gr = reinterpret_cast<const __nv_bfloat162*>(gu + (size_t)m * 2 * F);
+  const __nv_bfloat162* ur = reinterpret_cast<const __nv_bfloat162*>(gu + (size_t)m * 2 * F + F);
+  __nv_bfloat162* ar = reinterpret_cast<__nv_bfloat162*>(act + (size_t)m * F);
+  __shared__ float s_part[kRowThreads / 32];
+  float amax = 0.f;
+  for (int i = threadIdx.x; i < F / 2; i += blockDim.x) {
+    const float2 gt = __bfloat1622float2(gr[i]);
+    const float2 up = __bfloat1622float2(ur[i]);
+    const float a0 = gt.x / (1.0f + expf(-gt.x)) * up.x;
+    const float a1 = gt.y / (1.0f + expf(-gt.y)) * up.y;
+    const __nv_bfloat162 o = __floats2bfloat162_rn(a0, a1);
+    ar[i] = o;
+    const float2 of = __bfloat1622float2(o);
+    amax = fmaxf(amax, fmaxf(fabsf(of.x), fabsf(of.y)));
+  }
+  amax = block_max_rows(amax, s_part);
+  write_f16_row(act + (size_t)m * F, F, amax, act16 + (size_t)m * F, inv + m);
+}
+
+// ---- arg-max over the vocabulary, lowest index on ties ---------------------------------------
+// A row is cut into segments, one thread block each; a block's best (value, index) goes into the row's 64-bit key
+// by atomicMax: the value's bits made order-preserving in the high word, the complemented index in the low word,
+// so the largest key is the largest value and, among equals, the lowest index.  NaNs never enter; a row without
+// any number keeps key 0 and decodes to index 0.
+constexpr int kArgmaxSeg = 8192;
+
+__device__ __forceinline__ unsigned long long argmax_key(float x, int idx) {
+  x += 0.0f;                                            // -0 -> +0: they compare equal
+  uint32_t u = __float_as_uint(x);
+  u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+  return ((unsigned long long)u << 32) | (unsigned long long)(0xffffffffu - (uint32_t)idx);
+}
+
+__global__ void __launch_bounds__(256) argmax_segment_kernel(const float* __restrict__ logits, int V, unsigned long long* keys) {
+  const int m = blockIdx.y;
   const float* row = logits + (size_t)m * V;
-  float best = -INFINITY;
-  int bi = 0x7fffffff;
-  for (int v = threadIdx.x; v < V; v += blockDim.x) {
-    const float x = row[v];
-    if (x > best || (x == best && v < bi)) { best = x; bi = v; }
+  const int v0 = blockIdx.x * kArgmaxSeg;
+  const int v1 = min(V, v0 + kArgmaxSeg);
+  unsigned long long best = 0ull;
+  if ((V & 3) == 0) {
+    for (int v = v0 + threadIdx.x * 4; v < v1; v += 256 * 4) {
+      const float4 f = *reinterpret_cast<const float4*>(row + v);
+      const float e[4] = {f.x, f.y, f.z, f.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        if (e[j] == e[j]) {
+          const unsigned long long k = argmax_key(e[j], v + j);
+          best = k > best ? k : best;
+        }
+    }
+  } else {
+    for (int v = v0 + threadIdx.x; v < v1; v += 256) {
+      const float x = row[v];
+      if (x == x) {
+        const unsigned long long k = argmax_key(x, v);
+        best = k > best ? k : best;
+      }
+    }
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
-    const float ob = __shfl_xor_sync(0xffffffffu, best, o);
-    const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-    if (ob > best || (ob == best && oi < bi)) { best = ob; bi = oi; }
+    const unsigned long long ob = __shfl_xor_sync(0xffffffffu, best, o);
+    best = ob > best ? ob : best;
   }
-  __shared__ float s_b[32];
-  __shared__ int s_i[32];
-  if ((threadIdx.x & 31) == 0) { s_b[threadIdx.x >> 5] = best; s_i[threadIdx.x >> 5] = bi; }
-  __syncthreads();
-  if (threadIdx.x < 32) {
-    const int nw = blockDim.x >> 5;
-    best = threadIdx.x < nw ? s_b[threadIdx.x] : -INFINITY;
-    bi = threadIdx.x < nw ? s_i[threadIdx.x] : 0x7fffffff;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      const float ob = __shfl_xor_sync(0xffffffffu, best, o);
-      const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-      if (ob > best || (ob == best && oi < bi)) { best = ob; bi = oi; }
-    }
-    if (threadIdx.x == 0) top1[m] = bi == 0x7fffffff ? 0 : bi;
-  }
+  if ((threadIdx.x & 31) == 0 && best != 0ull) atomicMax(keys + m, best);
+}
+
+__global__ void argmax_decode_kernel(const unsigned long long* __restrict__ keys, int M, int32_t* top1) {
+  const int m = blockIdx.x * blockDim.x + threadIdx.x;
+  if (m >= M) return;
+  const unsigned long long k = keys[m];
+  top1[m] = k == 0ull ? 0 : (int32_t)(0xffffffffu - (uint32_t)(k & 0xffffffffull));
 }
 
 // ---- greedy acceptance: one thread per sequence ----------------------------------------------
@@ -305,6 +441,29 @@ int launch_rmsnorm(const __nv_bfloat16* x, const __nv_bfloat16* g, int M, int H,
   return QUASAR_OK;
 }
 
+int launch_rmsnorm_f16(const __nv_bfloat16* x, const __nv_bfloat16* g, int M, int H, float eps, __nv_bfloat16* y, void* y16,
+                       float* inv, cudaStream_t stream) {
+  rmsnorm_f16_kernel<false><<<M, kRowThreads, 0, stream>>>(nullptr, 0, 0, nullptr, nullptr, const_cast<__nv_bfloat16*>(x), g, H, eps, y,
+                                                    reinterpret_cast<__half*>(y16), inv);
+  QUASAR_LAUNCH_CHECK();
+  return QUASAR_OK;
+}
+
+int launch_reduce_residual_rmsnorm_f16(const float* partial, int nsplit, int mpad, const float* dx, const float* dw,
+                                       __nv_bfloat16* x, const __nv_bfloat16* g, int M, int H, float eps, __nv_bfloat16* y,
+                                       void* y16, float* inv, cudaStream_t stream) {
+  rmsnorm_f16_kernel<true><<<M, kRowThreads, 0, stream>>>(partial, nsplit, mpad, dx, dw, x, g, H, eps, y, reinterpret_cast<__half*>(y16),
+                                                   inv);
+  QUASAR_LAUNCH_CHECK();
+  return QUASAR_OK;
+}
+
+int launch_swiglu_f16(const __nv_bfloat16* gu, int M, int F, __nv_bfloat16* act, void* act16, float* inv, cudaStream_t stream) {
+  swiglu_f16_kernel<<<M, kRowThreads, 0, stream>>>(gu, F, act, reinterpret_cast<__half*>(act16), inv);
+  QUASAR_LAUNCH_CHECK();
+  return QUASAR_OK;
+}
+
 int launch_rope_table(float2* table, int max_pos, int D, float theta, cudaStream_t stream) {
   const int total = max_pos * (D / 2);
   rope_table_kernel<<<(total + 255) / 256, 256, 0, stream>>>(table, max_pos, D, (double)theta);
@@ -339,8 +498,11 @@ int launch_swiglu(const __nv_bfloat16* gu, int M, int F, __nv_bfloat16* act, cud
   return QUASAR_OK;
 }
 
-int launch_argmax(const float* logits, int M, int V, int32_t* top1, cudaStream_t stream) {
-  argmax_kernel<<<M, 1024, 0, stream>>>(logits, V, top1);
+int launch_argmax(const float* logits, int M, int V, int32_t* top1, unsigned long long* keys, cudaStream_t stream) {
+  QUASAR_CUDA_CHECK(cudaMemsetAsync(keys, 0, (size_t)M * sizeof(unsigned long long), stream));
+  argmax_segment_kernel<<<dim3((V + kArgmaxSeg - 1) / kArgmaxSeg, M), 256, 0, stream>>>(logits, V, keys);
+  QUASAR_LAUNCH_CHECK();
+  argmax_decode_kernel<<<(M + 127) / 128, 128, 0, stream>>>(keys, M, top1);
   QUASAR_LAUNCH_CHECK();
   return QUASAR_OK;
 }

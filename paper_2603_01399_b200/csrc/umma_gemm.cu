@@ -49,6 +49,7 @@ struct UmmaArgs {
   int* counters;
   int32_t* error;            // device status word (or nullptr): QUASAR_ERR_TIMEOUT when a wait ran out
   int M, Mpad, N, K, k_per_split, nsplit, y_is_f32;
+  int direct;                // 1: one k-range and the kernel itself applies the epilogue; 0: 32-bit partial sums go to `partial`
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -254,7 +255,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
           for (int j = 0; j < 16; ++j) {
             const int m = c0 + j;
             if (m >= a.M) continue;
-            if (a.nsplit == 1) store_output<true>(a, v[j], m, n);
+            if (a.direct) store_output<true>(a, v[j], m, n);
             else __stcg(reinterpret_cast<uint32_t*>(a.partial) + ((size_t)blockIdx.y * a.Mpad + m) * a.N + n, v[j]);
           }
         }
@@ -481,7 +482,7 @@ umma_w8a16_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_consta
           for (int j = 0; j < 16; ++j) {
             const int m = c0 + j;
             if (m >= a.M) continue;
-            if (a.nsplit == 1) store_output<false>(a, v[j], m, n);
+            if (a.direct) store_output<false>(a, v[j], m, n);
             else __stcg(reinterpret_cast<uint32_t*>(a.partial) + ((size_t)blockIdx.y * a.Mpad + m) * a.N + n, v[j]);
           }
         }
@@ -513,13 +514,8 @@ __global__ void __launch_bounds__(256) f16_rows_kernel(const __nv_bfloat16* __re
   amax = s_max[0];
 #pragma unroll
   for (int i = 1; i < 8; ++i) amax = fmaxf(amax, s_max[i]);
-  float scale = 1.f, inv = 1.f;
-  if (amax > 0.f && amax < 3.0e38f) {
-    int e;
-    (void)frexpf(amax, &e);            // amax = f * 2^e, f in [0.5, 1)
-    scale = ldexpf(1.f, 15 - e);       // scaled maximum in [2^14, 2^15)
-    inv = ldexpf(1.f, e - 15);
-  }
+  float scale, inv;
+  f16_row_scale(amax, scale, inv);
   if (threadIdx.x == 0) inv_scale[m] = inv;
   for (int64_t k = threadIdx.x; k < K; k += 256) x16[m * K + k] = __float2half_rn(__bfloat162float(row[k]) * scale);
 }
@@ -702,7 +698,7 @@ umma_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
           const uint32_t* v = m < 4 ? v0 + 4 * m : v1 + 4 * (m - 4);
           const long long total = ((long long)(int)v[2] << 16) + ((long long)(int)v[1] << 8) + (long long)(int)v[0];
           const uint32_t bits = __float_as_uint((float)total);
-          if (a.nsplit == 1) store_output<false>(a, bits, m, n);
+          if (a.direct) store_output<false>(a, bits, m, n);
           else __stcg(reinterpret_cast<uint32_t*>(a.partial) + ((size_t)split * a.Mpad + m) * a.N + n, bits);
         }
       }
@@ -800,6 +796,7 @@ int launch_umma_w8a8(const int8_t* xq, const float* dx, const int8_t* w, const f
   a.error = error_word;
   a.M = (int)M; a.Mpad = mpad; a.N = (int)N; a.K = (int)K; a.k_per_split = p.k_per_split; a.nsplit = p.nsplit;
   a.y_is_f32 = y_is_f32 ? 1 : 0;
+  a.direct = p.nsplit == 1 ? 1 : 0;
   const size_t smem = (size_t)kStagesI8 * (kTileN * kTileKBytes + mpad * kTileKBytes) + 256 + 1024;
   static bool configured = false;
   if (!configured) {
@@ -822,22 +819,36 @@ bool umma_w8a16_usable(int64_t M, int64_t N, int64_t K) {
   return M > 8 && M <= kMaxMpad && K % 16 == 0 && N >= 1;
 }
 
-// bytes of scratch: fp16 copy of the activation rows, their inverse scales, partial sums of the k-ranges
-size_t umma_w8a16_scratch_bytes(int64_t M, int64_t N, int64_t K) {
-  const SplitU p = plan_split_u(N, K);
-  const size_t mpad = (size_t)((M + 15) / 16) * 16;
-  const size_t partial = p.nsplit > 1 ? (size_t)p.nsplit * mpad * (size_t)N * 4 : 0;
-  return ((size_t)M * K * 2 + 255) / 256 * 256 + ((size_t)M * 4 + 255) / 256 * 256 + partial;
+void umma_w8a16_plan(int64_t M, int64_t N, int64_t K, int* nsplit, int* mpad) {
+  *nsplit = plan_split_u(N, K).nsplit;
+  *mpad = (int)((M + 15) / 16) * 16;
 }
 
-int launch_umma_w8a16(const __nv_bfloat16* x, const int8_t* w, const float* dw, int64_t M, int64_t N, int64_t K, void* y,
-                      bool y_is_f32, const __nv_bfloat16* residual, void* scratch, int32_t* error_word, cudaStream_t stream) {
-  unsigned char* sc = reinterpret_cast<unsigned char*>(scratch);
-  __half* x16 = reinterpret_cast<__half*>(sc);
-  float* inv = reinterpret_cast<float*>(sc + ((size_t)M * K * 2 + 255) / 256 * 256);
-  void* partial = sc + ((size_t)M * K * 2 + 255) / 256 * 256 + ((size_t)M * 4 + 255) / 256 * 256;
-  f16_rows_kernel<<<(unsigned)M, 256, 0, stream>>>(x, K, x16, inv);
+// bytes of the partial sums (also when one k-range is asked to leave its sums for a fused consumer, unless the
+// matrix is as wide as an LM head, which always finishes itself)
+size_t umma_w8a16_partial_bytes(int64_t M, int64_t N, int64_t K) {
+  const SplitU p = plan_split_u(N, K);
+  const size_t mpad = (size_t)((M + 15) / 16) * 16;
+  return (p.nsplit > 1 || N <= 32768) ? (size_t)p.nsplit * mpad * (size_t)N * 4 : 0;
+}
+
+// bytes of scratch: fp16 copy of the activation rows, their inverse scales, partial sums of the k-ranges
+size_t umma_w8a16_scratch_bytes(int64_t M, int64_t N, int64_t K) {
+  return ((size_t)M * K * 2 + 255) / 256 * 256 + ((size_t)M * 4 + 255) / 256 * 256 + umma_w8a16_partial_bytes(M, N, K);
+}
+
+int launch_f16_rows(const __nv_bfloat16* x, int64_t M, int64_t K, void* x16, float* inv_scale, cudaStream_t stream) {
+  f16_rows_kernel<<<(unsigned)M, 256, 0, stream>>>(x, K, reinterpret_cast<__half*>(x16), inv_scale);
   QUASAR_LAUNCH_CHECK();
+  return QUASAR_OK;
+}
+
+// x16 / inv: the activation rows as fp16 times a power of two and the inverse of that power (f16_rows_kernel or a
+// producer that writes the same thing).  finalize = false leaves the partial sums of every k-range in `partial`
+// ([nsplit][mpad][N] fp32, see umma_w8a16_plan) for a consumer that adds them up itself.
+int launch_umma_w8a16_prepared(const void* x16, const float* inv, const int8_t* w, const float* dw, int64_t M, int64_t N,
+                               int64_t K, void* y, bool y_is_f32, const __nv_bfloat16* residual, void* partial, bool finalize,
+                               int32_t* error_word, cudaStream_t stream) {
   CUtensorMap map_w, map_x;
   const int mpad = (int)((M + 15) / 16) * 16;
   int rc = make_map(&map_w, w, (uint64_t)N, (uint64_t)K, kTileN, 64);
@@ -850,6 +861,7 @@ int launch_umma_w8a16(const __nv_bfloat16* x, const int8_t* w, const float* dw, 
   a.error = error_word;
   a.M = (int)M; a.Mpad = mpad; a.N = (int)N; a.K = (int)K; a.k_per_split = p.k_per_split; a.nsplit = p.nsplit;
   a.y_is_f32 = y_is_f32 ? 1 : 0;
+  a.direct = (finalize && p.nsplit == 1) ? 1 : 0;
   const size_t smem = (size_t)kStagesF16 * (mpad * 128 + kRawBytes) + 256 + 1024;
   static bool configured = false;
   if (!configured) {
@@ -858,7 +870,7 @@ int launch_umma_w8a16(const __nv_bfloat16* x, const int8_t* w, const float* dw, 
   }
   umma_w8a16_kernel<<<dim3(p.nblocks, p.nsplit), kThreadsU, smem, stream>>>(map_w, map_x, a);
   QUASAR_LAUNCH_CHECK();
-  if (p.nsplit > 1) {
+  if (finalize && p.nsplit > 1) {
     const int64_t items = M * ((N + 3) / 4);
     umma_reduce_kernel<false><<<(unsigned)((items + 255) / 256), 256, 0, stream>>>(a);
     QUASAR_LAUNCH_CHECK();
@@ -866,6 +878,15 @@ int launch_umma_w8a16(const __nv_bfloat16* x, const int8_t* w, const float* dw, 
   return QUASAR_OK;
 }
 
+int launch_umma_w8a16(const __nv_bfloat16* x, const int8_t* w, const float* dw, int64_t M, int64_t N, int64_t K, void* y,
+                      bool y_is_f32, const __nv_bfloat16* residual, void* scratch, int32_t* error_word, cudaStream_t stream) {
+  unsigned char* sc = reinterpret_cast<unsigned char*>(scratch);
+  float* inv = reinterpret_cast<float*>(sc + ((size_t)M * K * 2 + 255) / 256 * 256);
+  void* partial = sc + ((size_t)M * K * 2 + 255) / 256 * 256 + ((size_t)M * 4 + 255) / 256 * 256;
+  int rc = launch_f16_rows(x, M, K, sc, inv, stream);
+  if (rc != QUASAR_OK) return rc;
+  return launch_umma_w8a16_prepared(sc, inv, w, dw, M, N, K, y, y_is_f32, residual, partial, true, error_word, stream);
+}
 
 // ---- weight-only form, at most 8 rows ----
 namespace {
@@ -918,6 +939,7 @@ int launch_umma_rows8(const __nv_bfloat16* x, const int8_t* w, const float* dw, 
   a.error = error_word;
   a.M = (int)M; a.Mpad = (int)M; a.N = (int)N; a.K = (int)K; a.k_per_split = p.k_per_split; a.nsplit = p.nsplit;
   a.y_is_f32 = y_is_f32 ? 1 : 0;
+  a.direct = p.nsplit == 1 ? 1 : 0;
   const size_t smem = (size_t)kStagesS * kTileN * kTileKBytes + (size_t)p.nb * p.k_per_split + 256 + 1024;
   static bool configured = false;
   if (!configured) {
