@@ -23,8 +23,8 @@ namespace quasar {
 
 namespace {
 
-constexpr int kKeyTile = 64;   // keys staged in shared memory at a time
-constexpr int kMaxWarps = 4;   // per CTA; three CTAs share an SM (168 registers per thread)
+constexpr int kKeyTile = 32;   // keys staged in shared memory at a time
+constexpr int kMaxWarps = 3;   // per CTA; four CTAs share an SM (168 registers per thread, 35 KB of tiles)
 constexpr float kLog2e = 1.4426950408889634f;
 
 struct AttnArgs {
@@ -79,7 +79,7 @@ __device__ __forceinline__ void split_bf16(float a, float b, uint32_t& hi, uint3
 }
 
 template <int D>
-__global__ void __launch_bounds__(kMaxWarps * 32, 3) verify_attention_kernel(AttnArgs a) {
+__global__ void __launch_bounds__(kMaxWarps * 32, 4) verify_attention_kernel(AttnArgs a) {
   constexpr int kStride = D + 8;  // padded row of the staged K / V tiles (bf16 elements)
   constexpr int kDSteps = D / 16;
   // two K tiles and two V tiles: the next tile of the chunk lands (cp.async) while the current one is multiplied
