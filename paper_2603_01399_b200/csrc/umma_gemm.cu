@@ -10,10 +10,12 @@
 //   * W8A8 (kind::i8, s8 x s8 -> s32): tiles of 128 rows x 128 contraction bytes are brought in by
 //     TMA (cp.async.bulk.tensor, 128-byte swizzle) exactly as the MMA reads them - no instruction
 //     touches a weight byte.  Accumulators are exact integers.
-//   * W8A16 (kind::f16, bf16 x bf16 -> f32): the same int8 tiles land in a raw ring; four warps
-//     turn each into a bf16 tile in the MMA's swizzled layout (int8 -> bf16 is exact), which is
-//     what the weight-only form costs on this path: 2 more bytes of shared-memory traffic per
-//     weight and one conversion instruction per two weights.
+//   * W8A16 (kind::f16, fp16 x fp16 -> f32): the same int8 tiles land in a raw ring; four warps turn each
+//     row into fp16 in registers (int8 -> fp16 is exact) and store it into tensor memory, from where the MMA
+//     reads operand A - which is what the weight-only form costs on this path: one conversion instruction
+//     per two weights and two bytes of tensor-memory stores per weight.
+//   * at most 8 rows on a very large matrix: a persistent stream kernel in which the 16-bit activations ride
+//     the integer MMAs as three int8 digits (further down).
 // Roles: warp 0 issues the TMA loads, warp 1 the MMAs (one elected thread), warps 2-5 convert
 // (W8A16) and run the epilogue (tcgen05.ld, one tensor-memory lane = one output channel per
 // thread).  k-ranges of one channel block are added up in a fixed order by a second, fully parallel kernel.

@@ -82,19 +82,7 @@ def _check_against_oracle(shape, r, buf, block_len, margin=5e-2):
             assert np.array_equal(buf.accept_path[b].cpu().numpy(), r.accept_path[b])
 
 
-def test_config1_chain_block_with_trace(world):
-    """Tiny decoder, 64-token prefix, chain draft of 4 = the bf16 model's greedy continuation with
-    replacement probability 0.3; every intermediate tensor is compared, then logits and acceptance."""
-    shape, om, gm, okv, root = world
-    ob = oracle_model(shape, seed=0, int8=False)
-    g = oracle_greedy_continuation(ob, okv, root, 4)
-    draft = synth.corrupt_draft(torch.tensor(g), 0.3, shape.vocab, seed=2).tolist()
-    tokens = np.array([[root] + draft], np.int32)
-    bl = np.array([5], np.int32)
-    okv2 = _copy(okv)
-    r = oracle.verify(om, okv2, tokens, None, bl, want_trace=True)
-    kv, buf, tr = _run_gpu(shape, gm, okv, tokens, None, bl, trace=True)
-    assert int(buf.status[0]) == 0
+def _compare_trace(shape, r, tr, rows):
     Hq, D = shape.n_q_heads, shape.head_dim
 
     # Tolerances, in bf16 half-ulps of the magnitudes involved.  This comparison runs the whole pass on both
@@ -121,13 +109,29 @@ def test_config1_chain_block_with_trace(world):
         early = 2.5 if l == 0 else 6.0          # nothing upstream has flipped yet in the first layer
         cmp(f"l{l}.h1", tr[f"l{l}.h1"][0], r.trace[f"l{l}.h1.b0"], ulps=early)
         cmp(f"l{l}.qkv", tr[f"l{l}.qkv"][0], r.trace[f"l{l}.qkv.b0"], ulps=early)
-        cmp(f"l{l}.q", tr[f"l{l}.qkv_rope"][0][:, : Hq * D], r.trace[f"l{l}.q.b0"].reshape(5, Hq * D), ulps=early)
+        cmp(f"l{l}.q", tr[f"l{l}.qkv_rope"][0][:, : Hq * D], r.trace[f"l{l}.q.b0"].reshape(rows, Hq * D), ulps=early)
         cmp(f"l{l}.attn", tr[f"l{l}.attn"][0], r.trace[f"l{l}.attn.b0"])
         x_in = r.trace["embed.b0"] if l == 0 else r.trace[f"l{l - 1}.x_mlp.b0"]
         cmp(f"l{l}.x_attn", tr[f"l{l}.x_attn"][0], r.trace[f"l{l}.x_attn.b0"], prev=x_in)
         cmp(f"l{l}.act", tr[f"l{l}.act"][0], r.trace[f"l{l}.act.b0"], ulps=10.0)   # two flipped factors + rounding
         cmp(f"l{l}.x_mlp", tr[f"l{l}.x_mlp"][0], r.trace[f"l{l}.x_mlp.b0"], prev=r.trace[f"l{l}.x_attn.b0"])
     cmp("hf", tr["hf"][0], r.trace["hf.b0"])
+
+
+def test_config1_chain_block_with_trace(world):
+    """Tiny decoder, 64-token prefix, chain draft of 4 = the bf16 model's greedy continuation with
+    replacement probability 0.3; every intermediate tensor is compared, then logits and acceptance."""
+    shape, om, gm, okv, root = world
+    ob = oracle_model(shape, seed=0, int8=False)
+    g = oracle_greedy_continuation(ob, okv, root, 4)
+    draft = synth.corrupt_draft(torch.tensor(g), 0.3, shape.vocab, seed=2).tolist()
+    tokens = np.array([[root] + draft], np.int32)
+    bl = np.array([5], np.int32)
+    okv2 = _copy(okv)
+    r = oracle.verify(om, okv2, tokens, None, bl, want_trace=True)
+    kv, buf, tr = _run_gpu(shape, gm, okv, tokens, None, bl, trace=True)
+    assert int(buf.status[0]) == 0
+    _compare_trace(shape, r, tr, 5)
     # K written at slots 63..67: the first layer's rows within one rounding, the second layer's with the
     # inherited flips
     P = int(okv.seq_len[0])
@@ -138,6 +142,23 @@ def test_config1_chain_block_with_trace(world):
     assert torch.equal(kv.seq_len.cpu(), torch.from_numpy(okv.seq_len))          # verify does not commit
     _check_against_oracle(shape, r, buf, bl)
     assert 0 <= int(buf.accept_len[0]) <= 4
+
+def test_every_tensor_of_a_twelve_row_block(world):
+    """A chain of 11 drafts (12 block rows) is beyond the persistent kernel: the pass runs as one kernel per step,
+    with int8 weights in its fused form (tcgen05 linear layers fed by producers that write the fp16 operand, the
+    k-ranges of the residual layers added up by the following norm kernel).  Every intermediate tensor is
+    compared with the oracle, at the tolerances of the 5-row test."""
+    shape, om, gm, okv, root = world
+    g = oracle_greedy_continuation(om, okv, root, 11)
+    draft = synth.corrupt_draft(torch.tensor(g), 0.3, shape.vocab, seed=5).tolist()
+    tokens = np.array([[root] + draft], np.int32)
+    bl = np.array([12], np.int32)
+    r = oracle.verify(om, _copy(okv), tokens, None, bl, want_trace=True)
+    kv, buf, tr = _run_gpu(shape, gm, okv, tokens, None, bl, trace=True)
+    assert int(buf.status[0]) == 0
+    _compare_trace(shape, r, tr, 12)
+    _check_against_oracle(shape, r, buf, bl)
+    assert 0 <= int(buf.accept_len[0]) <= 11
 
 
 def test_own_greedy_draft_fully_accepted_and_idempotent(world):
