@@ -301,20 +301,40 @@ __global__ void __launch_bounds__(128) attention_merge_kernel(AttnArgs a) {
   const int Lk = a.seq_len[b] + a.block_len[b];
   const int nch = (Lk + a.chunk - 1) / a.chunk;
   const size_t slot0 = ((size_t)b * a.Hkv + hk) * a.nchunk * a.Rpad;
+  // the row's maximum over the chunks: the lanes take the chunks in turn
   float mx = -INFINITY;
-  for (int c = 0; c < nch; ++c) mx = fmaxf(mx, a.ml_part[(slot0 + (size_t)c * a.Rpad + r) * 2]);
+  for (int c = lane; c < nch; c += 32) mx = fmaxf(mx, a.ml_part[(slot0 + (size_t)c * a.Rpad + r) * 2]);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
   float acc[kPer];
 #pragma unroll
   for (int e = 0; e < kPer; ++e) acc[e] = 0.f;
   float den = 0.f;
-  for (int c = 0; c < nch; ++c) {
-    const size_t s = slot0 + (size_t)c * a.Rpad + r;
-    const float mc = a.ml_part[s * 2];
-    if (mc == -INFINITY) continue;
-    const float w = exp2f(mc - mx);
-    den += w * a.ml_part[s * 2 + 1];
+  // chunks are added in chunk order, eight at a time so that their loads are in flight together
+  for (int c0 = 0; c0 < nch; c0 += 8) {
+    float2 ml[8];
+    float ov[8][kPer];
 #pragma unroll
-    for (int e = 0; e < kPer; ++e) acc[e] += w * a.o_part[s * D + lane * kPer + e];
+    for (int j = 0; j < 8; ++j) {
+      const bool in = c0 + j < nch;
+      const size_t s = slot0 + (size_t)(in ? c0 + j : c0) * a.Rpad + r;
+      ml[j] = in ? *reinterpret_cast<const float2*>(a.ml_part + s * 2) : make_float2(-INFINITY, 0.f);
+      if constexpr (kPer == 4) {
+        const float4 v = *reinterpret_cast<const float4*>(a.o_part + s * D + lane * kPer);
+        ov[j][0] = v.x; ov[j][1] = v.y; ov[j][2] = v.z; ov[j][3] = v.w;
+      } else {
+        const float2 v = *reinterpret_cast<const float2*>(a.o_part + s * D + lane * kPer);
+        ov[j][0] = v.x; ov[j][1] = v.y;
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      if (ml[j].x == -INFINITY) continue;
+      const float w = exp2f(ml[j].x - mx);
+      den += w * ml[j].y;
+#pragma unroll
+      for (int e = 0; e < kPer; ++e) acc[e] += w * ov[j][e];
+    }
   }
   const float inv = 1.0f / den;
 #pragma unroll
