@@ -306,7 +306,7 @@ int verify_impl(quasar_model* m, const quasar_kv* kv, const int32_t* tokens, con
   // Blocks of 9..80 rows with int8 weights and 16-bit activations: every linear layer is the tcgen05 kernel, which
   // wants its operand as fp16 rows times a power of two.  The kernel that produces an operand writes that form too, and
   // the kernel after a residual linear layer adds up its k-ranges, so a layer is 12 launches instead of 17.
-  bool fused = !a8 && wd == QUASAR_W_INT8 && M > 8 && M <= 80;
+  bool fused = !a8 && wd == QUASAR_W_INT8 && M > 8 && M <= 80 && H <= 8192 && F <= 24576;   // (rows the fused row kernels hold in registers)
   {
     const int64_t shapes[5][2] = {{qkv_w, H}, {H, (int64_t)Hq * D}, {2 * (int64_t)F, H}, {H, F}, {c.vocab, H}};
     for (auto& sh : shapes) fused = fused && umma_w8a16_usable(M, sh[0], sh[1]);

@@ -112,21 +112,10 @@ __device__ __forceinline__ float block_max_rows(float v, float* s_buf) {
   return r;
 }
 
-// fp16 form of the row a thread block has just written as bf16 (every thread re-reads the pairs it wrote itself)
-__device__ __forceinline__ void write_f16_row(const __nv_bfloat16* y_row, int width, float amax, __half* y16_row, float* inv_out) {
-  float scale, inv;
-  f16_row_scale(amax, scale, inv);
-  if (threadIdx.x == 0) *inv_out = inv;
-  const __nv_bfloat162* yr = reinterpret_cast<const __nv_bfloat162*>(y_row);
-  __half2* hr = reinterpret_cast<__half2*>(y16_row);
-  for (int i = threadIdx.x; i < width / 2; i += blockDim.x) {
-    const float2 f = __bfloat1622float2(yr[i]);
-    hr[i] = __floats2half2_rn(f.x * scale, f.y * scale);
-  }
-}
+// A row stays in registers between its passes: thread t holds the pairs t, t + 1024, ... (at most kNormPairs of them,
+// i.e. rows of up to 8192 elements; the launcher refuses longer ones).
+constexpr int kNormPairs = 4;
 
-// ---- RMSNorm that also leaves the fp16 form of its output; optionally preceded by the epilogue of a residual linear
-//      layer whose k-range partial sums it adds up (REDUCE) ---------------------------------------------------------
 template <bool REDUCE>
 __global__ void __launch_bounds__(kRowThreads)
 rmsnorm_f16_kernel(const float* __restrict__ partial, int nsplit, int mpad, const float* __restrict__ dx,
@@ -136,32 +125,39 @@ rmsnorm_f16_kernel(const float* __restrict__ partial, int nsplit, int mpad, cons
   __nv_bfloat162* xr = reinterpret_cast<__nv_bfloat162*>(x + (size_t)m * H);
   const __nv_bfloat162* gr = reinterpret_cast<const __nv_bfloat162*>(g);
   __nv_bfloat162* yr = reinterpret_cast<__nv_bfloat162*>(y + (size_t)m * H);
+  __half2* hr = reinterpret_cast<__half2*>(y16 + (size_t)m * H);
   __shared__ float s_part[kRowThreads / 32];
+  const int np = H / 2;
+  float2 xv[kNormPairs], gv[kNormPairs];
   float ss = 0.f;
-  if (REDUCE) {
-    const float dxm = dx[m];
-    const size_t split_stride = (size_t)mpad * H;
-    const float* p0 = partial + (size_t)m * H;
-    for (int i = threadIdx.x; i < H / 2; i += blockDim.x) {
-      float2 acc = make_float2(0.f, 0.f);
-      for (int s = 0; s < nsplit; ++s) {   // k-ranges in ascending order
-        const float2 v = __ldcg(reinterpret_cast<const float2*>(p0 + (size_t)s * split_stride) + i);
-        acc.x += v.x;
-        acc.y += v.y;
+#pragma unroll
+  for (int j = 0; j < kNormPairs; ++j) {
+    const int i = threadIdx.x + j * kRowThreads;
+    xv[j] = make_float2(0.f, 0.f);
+    gv[j] = make_float2(0.f, 0.f);
+    if (i < np) {
+      gv[j] = __bfloat1622float2(gr[i]);
+      if (REDUCE) {
+        const float dxm = dx[m];
+        const size_t split_stride = (size_t)mpad * H;
+        const float* p0 = partial + (size_t)m * H;
+        float2 acc = make_float2(0.f, 0.f);
+        for (int sp = 0; sp < nsplit; ++sp) {   // k-ranges in ascending order
+          const float2 v = __ldcg(reinterpret_cast<const float2*>(p0 + (size_t)sp * split_stride) + i);
+          acc.x += v.x;
+          acc.y += v.y;
+        }
+        const float2 d = *reinterpret_cast<const float2*>(dw + 2 * i);
+        const float2 r = __bfloat1622float2(xr[i]);
+        const float v0 = __bfloat162float(__float2bfloat16_rn((acc.x * dxm) * d.x)) + r.x;
+        const float v1 = __bfloat162float(__float2bfloat16_rn((acc.y * dxm) * d.y)) + r.y;
+        const __nv_bfloat162 o = __floats2bfloat162_rn(v0, v1);
+        xr[i] = o;
+        xv[j] = __bfloat1622float2(o);
+      } else {
+        xv[j] = __bfloat1622float2(xr[i]);
       }
-      const float2 d = *reinterpret_cast<const float2*>(dw + 2 * i);
-      const float2 r = __bfloat1622float2(xr[i]);
-      const float v0 = __bfloat162float(__float2bfloat16_rn((acc.x * dxm) * d.x)) + r.x;
-      const float v1 = __bfloat162float(__float2bfloat16_rn((acc.y * dxm) * d.y)) + r.y;
-      const __nv_bfloat162 o = __floats2bfloat162_rn(v0, v1);
-      xr[i] = o;
-      const float2 f = __bfloat1622float2(o);
-      ss += f.x * f.x + f.y * f.y;
-    }
-  } else {
-    for (int i = threadIdx.x; i < H / 2; i += blockDim.x) {
-      const float2 f = __bfloat1622float2(xr[i]);
-      ss += f.x * f.x + f.y * f.y;
+      ss += xv[j].x * xv[j].x + xv[j].y * xv[j].y;
     }
   }
   ss = warp_sum(ss);
@@ -172,16 +168,25 @@ rmsnorm_f16_kernel(const float* __restrict__ partial, int nsplit, int mpad, cons
   for (int i = 0; i < kRowThreads / 32; ++i) tot += s_part[i];
   const float r = 1.0f / sqrtf(tot / (float)H + eps);
   float amax = 0.f;
-  for (int i = threadIdx.x; i < H / 2; i += blockDim.x) {
-    const float2 f = __bfloat1622float2(xr[i]);
-    const float2 gg = __bfloat1622float2(gr[i]);
-    const __nv_bfloat162 o = __floats2bfloat162_rn(f.x * r * gg.x, f.y * r * gg.y);
-    yr[i] = o;
-    const float2 of = __bfloat1622float2(o);
-    amax = fmaxf(amax, fmaxf(fabsf(of.x), fabsf(of.y)));
+#pragma unroll
+  for (int j = 0; j < kNormPairs; ++j) {
+    const int i = threadIdx.x + j * kRowThreads;
+    if (i < np) {
+      const __nv_bfloat162 o = __floats2bfloat162_rn(xv[j].x * r * gv[j].x, xv[j].y * r * gv[j].y);
+      yr[i] = o;
+      xv[j] = __bfloat1622float2(o);
+      amax = fmaxf(amax, fmaxf(fabsf(xv[j].x), fabsf(xv[j].y)));
+    }
   }
   amax = block_max_rows(amax, s_part);
-  write_f16_row(y + (size_t)m * H, H, amax, y16 + (size_t)m * H, inv + m);
+  float scale, inv_s;
+  f16_row_scale(amax, scale, inv_s);
+  if (threadIdx.x == 0) inv[m] = inv_s;
+#pragma unroll
+  for (int j = 0; j < kNormPairs; ++j) {
+    const int i = threadIdx.x + j * kRowThreads;
+    if (i < np) hr[i] = __floats2half2_rn(xv[j].x * scale, xv[j].y * scale);
+  }
 }
 
 // ---- RoPE table: cos/sin(pos * theta^(-2i/D)) evaluated in fp64, stored as fp32 -------------
@@ -265,7 +270,10 @@ __global__ void swiglu_kernel(const __nv_bfloat16* __restrict__ gu, int F, __nv_
   reinterpret_cast<__nv_bfloat162*>(act + (size_t)m * F)[f2] = __floats2bfloat162_rn(a0, a1);
 }
 
-// the same, one thread block per row, leaving the fp16 form of the row as well
+// the same, one thread block per row, leaving the fp16 form of the row as well (the row stays in registers between
+// the two passes: at most kActPairs pairs per thread, i.e. rows of up to 24576 elements)
+constexpr int kActPairs = 12;
+
 __global__ void __launch_bounds__(kRowThreads)
 swiglu_f16_kernel(const __nv_bfloat16* __restrict__ gu, int F, __nv_bfloat16* __restrict__ act, __half* __restrict__ act16,
                   float* __restrict__ inv) {
@@ -273,20 +281,37 @@ swiglu_f16_kernel(const __nv_bfloat16* __restrict__ gu, int F, __nv_bfloat16* __
   const __nv_bfloat162* gr = reinterpret_cast<const __nv_bfloat162*>(gu + (size_t)m * 2 * F);
   const __nv_bfloat162* ur = reinterpret_cast<const __nv_bfloat162*>(gu + (size_t)m * 2 * F + F);
   __nv_bfloat162* ar = reinterpret_cast<__nv_bfloat162*>(act + (size_t)m * F);
+  __half2* hr = reinterpret_cast<__half2*>(act16 + (size_t)m * F);
   __shared__ float s_part[kRowThreads / 32];
+  const int np = F / 2;
+  __nv_bfloat162 av[kActPairs];
   float amax = 0.f;
-  for (int i = threadIdx.x; i < F / 2; i += blockDim.x) {
-    const float2 gt = __bfloat1622float2(gr[i]);
-    const float2 up = __bfloat1622float2(ur[i]);
-    const float a0 = gt.x / (1.0f + expf(-gt.x)) * up.x;
-    const float a1 = gt.y / (1.0f + expf(-gt.y)) * up.y;
-    const __nv_bfloat162 o = __floats2bfloat162_rn(a0, a1);
-    ar[i] = o;
-    const float2 of = __bfloat1622float2(o);
-    amax = fmaxf(amax, fmaxf(fabsf(of.x), fabsf(of.y)));
+#pragma unroll
+  for (int j = 0; j < kActPairs; ++j) {
+    const int i = threadIdx.x + j * kRowThreads;
+    if (i < np) {
+      const float2 gt = __bfloat1622float2(gr[i]);
+      const float2 up = __bfloat1622float2(ur[i]);
+      const float a0 = gt.x / (1.0f + expf(-gt.x)) * up.x;
+      const float a1 = gt.y / (1.0f + expf(-gt.y)) * up.y;
+      av[j] = __floats2bfloat162_rn(a0, a1);
+      ar[i] = av[j];
+      const float2 of = __bfloat1622float2(av[j]);
+      amax = fmaxf(amax, fmaxf(fabsf(of.x), fabsf(of.y)));
+    }
   }
   amax = block_max_rows(amax, s_part);
-  write_f16_row(act + (size_t)m * F, F, amax, act16 + (size_t)m * F, inv + m);
+  float scale, inv_s;
+  f16_row_scale(amax, scale, inv_s);
+  if (threadIdx.x == 0) inv[m] = inv_s;
+#pragma unroll
+  for (int j = 0; j < kActPairs; ++j) {
+    const int i = threadIdx.x + j * kRowThreads;
+    if (i < np) {
+      const float2 of = __bfloat1622float2(av[j]);
+      hr[i] = __floats2half2_rn(of.x * scale, of.y * scale);
+    }
+  }
 }
 
 // ---- arg-max over the vocabulary, lowest index on ties ---------------------------------------
@@ -443,6 +468,7 @@ int launch_rmsnorm(const __nv_bfloat16* x, const __nv_bfloat16* g, int M, int H,
 
 int launch_rmsnorm_f16(const __nv_bfloat16* x, const __nv_bfloat16* g, int M, int H, float eps, __nv_bfloat16* y, void* y16,
                        float* inv, cudaStream_t stream) {
+  if (H > 2 * kNormPairs * kRowThreads) { set_error("rmsnorm_f16: rows of %d elements (at most %d)", H, 2 * kNormPairs * kRowThreads); return QUASAR_ERR_SHAPE; }
   rmsnorm_f16_kernel<false><<<M, kRowThreads, 0, stream>>>(nullptr, 0, 0, nullptr, nullptr, const_cast<__nv_bfloat16*>(x), g, H, eps, y,
                                                     reinterpret_cast<__half*>(y16), inv);
   QUASAR_LAUNCH_CHECK();
@@ -452,6 +478,7 @@ int launch_rmsnorm_f16(const __nv_bfloat16* x, const __nv_bfloat16* g, int M, in
 int launch_reduce_residual_rmsnorm_f16(const float* partial, int nsplit, int mpad, const float* dx, const float* dw,
                                        __nv_bfloat16* x, const __nv_bfloat16* g, int M, int H, float eps, __nv_bfloat16* y,
                                        void* y16, float* inv, cudaStream_t stream) {
+  if (H > 2 * kNormPairs * kRowThreads) { set_error("rmsnorm_f16: rows of %d elements (at most %d)", H, 2 * kNormPairs * kRowThreads); return QUASAR_ERR_SHAPE; }
   rmsnorm_f16_kernel<true><<<M, kRowThreads, 0, stream>>>(partial, nsplit, mpad, dx, dw, x, g, H, eps, y, reinterpret_cast<__half*>(y16),
                                                    inv);
   QUASAR_LAUNCH_CHECK();
@@ -459,6 +486,7 @@ int launch_reduce_residual_rmsnorm_f16(const float* partial, int nsplit, int mpa
 }
 
 int launch_swiglu_f16(const __nv_bfloat16* gu, int M, int F, __nv_bfloat16* act, void* act16, float* inv, cudaStream_t stream) {
+  if (F > 2 * kActPairs * kRowThreads) { set_error("swiglu_f16: rows of %d elements (at most %d)", F, 2 * kActPairs * kRowThreads); return QUASAR_ERR_SHAPE; }
   swiglu_f16_kernel<<<M, kRowThreads, 0, stream>>>(gu, F, act, reinterpret_cast<__half*>(act16), inv);
   QUASAR_LAUNCH_CHECK();
   return QUASAR_OK;
