@@ -686,7 +686,7 @@ def run_reference(args):
         "unit": "accepted tok/s", "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": step_s * 1e3, "ms_per_pass_extrapolated": full * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-        "data": "synthetic", "config": {"workload": WORKLOAD},
+        "data": "synthetic", "config": {"workload": WORKLOAD, "replicas": 1, "batch": BATCH, "prefix": PREFIX, "gamma": GAMMA},
         "cpu_baseline": {"value": val, "unit": "accepted tok/s", "kind": "oracle", "cores": sample.threads,
                          "sample": "each step: 1 of 36 decoder layers + LM head at full widths, scaled to 36 layers; "
                                    "counts the bonus token only (1 token per pass)"},
