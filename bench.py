@@ -404,7 +404,7 @@ def time_tree14b(binding, reps, hbm_peak):
 def time_w8a8(binding, shape, kv, tokens_host, reps, hbm_peak):
     """The paper's W8A8 verifier (Section 3.2-3.3) on the headline workload: smoothing factors from synthetic
     calibration maxima, int8 activations per token, integer tensor-core GEMMs."""
-    model = binding.Model.from_master(shape, master_getter(shape, 0, "cuda"), PREFIX + 16, int8=True, act_int8=True,
+    model = binding.Model.from_master(shape, master_getter(shape, 0, "cuda"), 4096 + 16, int8=True, act_int8=True,
                                       get_act_absmax=lambda kind, layer: synth.activation_absmax(shape, kind, layer, 0, "cuda"))
     buf = binding.VerifyBuffers(model, BATCH, GAMMA + 1, want_logits=False)
     buf.tokens.copy_(tokens_host)
@@ -420,6 +420,10 @@ def time_w8a8(binding, shape, kv, tokens_host, reps, hbm_peak):
            "roofline": {"bound": "hbm", "achieved": gbs, "peak": hbm_peak, "unit": "GB/s", "frac": gbs / hbm_peak},
            "launch": model.launch_kind(BATCH, GAMMA + 1), "device_status": int(buf.status[0])}
     plan.close()
+    # the batch-of-eight workload with the same W8A8 model (72 block rows: tcgen05 kind::i8 linear layers)
+    b8 = time_batch8(binding, model, shape, max(3, reps // 2), hbm_peak)
+    b8["workload"] = b8["workload"].replace("int8 weights", "int8 weights and int8 activations (W8A8, smoothed)")
+    out["batch8_ragged"] = b8
     model.close()
     del model, buf
     torch.cuda.empty_cache()

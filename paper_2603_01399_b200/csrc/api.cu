@@ -366,13 +366,23 @@ int verify_impl(quasar_model* m, const quasar_kv* kv, const int32_t* tokens, con
     return QUASAR_OK;
   }
 
+  // W8A8: the norm and SwiGLU kernels smooth and quantise their output rows themselves (Eq. 9), straight into the place
+  // where the linear layer that follows keeps its quantised operand; that layer is then called without an input.
+  const bool a8_fuse = a8 && M <= kMaxRowsPerGemm && H <= 8192 && F <= 24576;
+  auto norm = [&](const __nv_bfloat16* in, const void* gain, const float* smooth) -> int {
+    if (!a8_fuse) return launch_rmsnorm(in, reinterpret_cast<const __nv_bfloat16*>(gain), M, H, c.rms_eps, h, stream);
+    int8_t* xq = nullptr;
+    float* dxp = nullptr;
+    linear_w8a8_operand_slots(lin, M, H, &xq, &dxp);
+    return launch_rmsnorm_q8(in, reinterpret_cast<const __nv_bfloat16*>(gain), smooth, M, H, c.rms_eps, h, xq, dxp, stream);
+  };
   for (int l = 0; l < c.n_layers; ++l) {
     const quasar_layer_weights& L = m->layers[l];
     __nv_bfloat16* kc = reinterpret_cast<__nv_bfloat16*>(kv->k) + (size_t)l * layer_stride;
     __nv_bfloat16* vc = reinterpret_cast<__nv_bfloat16*>(kv->v) + (size_t)l * layer_stride;
-    TRY(launch_rmsnorm(x, reinterpret_cast<const __nv_bfloat16*>(L.attn_norm), M, H, c.rms_eps, h, stream));
+    TRY(norm(x, L.attn_norm, L.qkv_smooth));
     TRY(tr.put(h, (size_t)M * H * 2));
-    TRY(linear(h, L.qkv_w, L.qkv_delta, L.qkv_smooth, qkv_w, H, qkv, false, nullptr));
+    TRY(linear(a8_fuse ? nullptr : h, L.qkv_w, L.qkv_delta, L.qkv_smooth, qkv_w, H, qkv, false, nullptr));
     TRY(tr.put(qkv, (size_t)M * qkv_w * 2));
     TRY(launch_rope_append(qkv, reinterpret_cast<const __nv_bfloat16*>(c.qk_norm ? L.q_norm : nullptr),
                            reinterpret_cast<const __nv_bfloat16*>(c.qk_norm ? L.k_norm : nullptr), m->rope_table,
@@ -383,16 +393,23 @@ int verify_impl(quasar_model* m, const quasar_kv* kv, const int32_t* tokens, con
     TRY(tr.put(attn, (size_t)M * Hq * D * 2));
     TRY(linear(attn, L.o_w, L.o_delta, L.o_smooth, H, Hq * D, x, false, x));
     TRY(tr.put(x, (size_t)M * H * 2));
-    TRY(launch_rmsnorm(x, reinterpret_cast<const __nv_bfloat16*>(L.mlp_norm), M, H, c.rms_eps, h, stream));
-    TRY(linear(h, L.gateup_w, L.gateup_delta, L.gateup_smooth, 2 * F, H, gu, false, nullptr));
-    TRY(launch_swiglu(gu, M, F, act, stream));
+    TRY(norm(x, L.mlp_norm, L.gateup_smooth));
+    TRY(linear(a8_fuse ? nullptr : h, L.gateup_w, L.gateup_delta, L.gateup_smooth, 2 * F, H, gu, false, nullptr));
+    if (a8_fuse) {
+      int8_t* xq = nullptr;
+      float* dxp = nullptr;
+      linear_w8a8_operand_slots(lin, M, F, &xq, &dxp);
+      TRY(launch_swiglu_q8(gu, L.down_smooth, M, F, act, xq, dxp, stream));
+    } else {
+      TRY(launch_swiglu(gu, M, F, act, stream));
+    }
     TRY(tr.put(act, (size_t)M * F * 2));
-    TRY(linear(act, L.down_w, L.down_delta, L.down_smooth, H, F, x, false, x));
+    TRY(linear(a8_fuse ? nullptr : act, L.down_w, L.down_delta, L.down_smooth, H, F, x, false, x));
     TRY(tr.put(x, (size_t)M * H * 2));
   }
-  TRY(launch_rmsnorm(x, reinterpret_cast<const __nv_bfloat16*>(m->w.final_norm), M, H, c.rms_eps, h, stream));
+  TRY(norm(x, m->w.final_norm, m->w.lm_smooth));
   TRY(tr.put(h, (size_t)M * H * 2));
-  TRY(linear(h, m->w.lm_w, m->w.lm_delta, m->w.lm_smooth, c.vocab, H, logits, true, nullptr));
+  TRY(linear(a8_fuse ? nullptr : h, m->w.lm_w, m->w.lm_delta, m->w.lm_smooth, c.vocab, H, logits, true, nullptr));
   TRY(launch_argmax(logits, M, c.vocab, top1, reinterpret_cast<unsigned long long*>(wsp + ws.keys), stream));
   TRY(launch_accept(tokens, parents, block_len, top1, bi, B, T_max, accept_len, bonus, accept_path, stream));
   return QUASAR_OK;

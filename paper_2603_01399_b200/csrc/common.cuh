@@ -72,6 +72,7 @@ int launch_smoothing_factors(const float* act_absmax, const __nv_bfloat16* w, in
 int launch_quantize_smoothed(const __nv_bfloat16* v, const float* s, int mode, int64_t rows, int64_t K, int8_t* q,
                              float* delta, cudaStream_t stream);
 size_t linear_w8a8_workspace_bytes(int64_t M, int64_t N, int64_t K);
+void linear_w8a8_operand_slots(void* workspace, int64_t M, int64_t K, int8_t** xq, float** dx);
 int launch_linear_w8a8(const __nv_bfloat16* x, const float* smooth, const int8_t* w, const float* delta_w, int64_t M,
                        int64_t N, int64_t K, void* y, bool y_is_f32, const __nv_bfloat16* residual, int32_t* acc_out,
                        void* workspace, size_t workspace_bytes, int32_t* status, cudaStream_t stream);
@@ -153,6 +154,11 @@ int launch_swiglu(const __nv_bfloat16* gu, int M, int F, __nv_bfloat16* act, cud
 // fp16 form of its output rows (x16 [M][width] + inv [M]).
 int launch_rmsnorm_f16(const __nv_bfloat16* x, const __nv_bfloat16* g, int M, int H, float eps, __nv_bfloat16* y, void* y16,
                        float* inv, cudaStream_t stream);
+// The same for the W8A8 pass: the producer smooths and quantises its output rows per token (Eq. 9) into xq / dx.
+int launch_rmsnorm_q8(const __nv_bfloat16* x, const __nv_bfloat16* g, const float* smooth, int M, int H, float eps,
+                      __nv_bfloat16* y, int8_t* xq, float* dx, cudaStream_t stream);
+int launch_swiglu_q8(const __nv_bfloat16* gu, const float* smooth, int M, int F, __nv_bfloat16* act, int8_t* xq, float* dx,
+                     cudaStream_t stream);
 int launch_swiglu_f16(const __nv_bfloat16* gu, int M, int F, __nv_bfloat16* act, void* act16, float* inv, cudaStream_t stream);
 // x += bf16(dw * dx * sum of the k-range partial sums) (the epilogue of a residual linear layer), then y = RMSNorm(x) * g
 // with its fp16 form: one kernel in place of the split-K reduction, the norm and the operand pre-pass

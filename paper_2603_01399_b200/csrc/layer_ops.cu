@@ -189,6 +189,71 @@ rmsnorm_f16_kernel(const float* __restrict__ partial, int nsplit, int mpad, cons
   }
 }
 
+// Eq. 9 for a row held in registers as pairs: the per-token step from the maximum of the smoothed values, then the codes.
+// v: the thread's smoothed values (pair j = elements 2 (thread + j * kRowThreads), +1); np pairs in the row.
+template <int PAIRS>
+__device__ __forceinline__ void quantize_row_pairs(const float2 (&v)[PAIRS], int np, float* s_part, int8_t* xq_row, float* dx_out) {
+  float amax = 0.f;
+#pragma unroll
+  for (int j = 0; j < PAIRS; ++j)
+    if ((int)threadIdx.x + j * kRowThreads < np) amax = fmaxf(amax, fmaxf(fabsf(v[j].x), fabsf(v[j].y)));
+  amax = block_max_rows(amax, s_part);
+  const float d = (amax == 0.f) ? 1.0f : __fdiv_rn(amax, 127.0f);
+  if (threadIdx.x == 0) *dx_out = d;
+#pragma unroll
+  for (int j = 0; j < PAIRS; ++j) {
+    const int i = (int)threadIdx.x + j * kRowThreads;
+    if (i < np) {
+      const int q0 = max(-127, min(127, __float2int_rn(__fdiv_rn(v[j].x, d))));
+      const int q1 = max(-127, min(127, __float2int_rn(__fdiv_rn(v[j].y, d))));
+      reinterpret_cast<char2*>(xq_row)[i] = make_char2((signed char)q0, (signed char)q1);
+    }
+  }
+}
+
+// RMSNorm whose output row is also smoothed and quantised per token for the W8A8 linear layer that follows.
+__global__ void __launch_bounds__(kRowThreads)
+rmsnorm_q8_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ g, const float* __restrict__ smooth, int H,
+                  float eps, __nv_bfloat16* __restrict__ y, int8_t* __restrict__ xq, float* __restrict__ dx) {
+  const int m = blockIdx.x;
+  const __nv_bfloat162* xr = reinterpret_cast<const __nv_bfloat162*>(x + (size_t)m * H);
+  const __nv_bfloat162* gr = reinterpret_cast<const __nv_bfloat162*>(g);
+  __nv_bfloat162* yr = reinterpret_cast<__nv_bfloat162*>(y + (size_t)m * H);
+  __shared__ float s_part[kRowThreads / 32];
+  const int np = H / 2;
+  float2 xv[kNormPairs];
+  float ss = 0.f;
+#pragma unroll
+  for (int j = 0; j < kNormPairs; ++j) {
+    const int i = threadIdx.x + j * kRowThreads;
+    xv[j] = make_float2(0.f, 0.f);
+    if (i < np) {
+      xv[j] = __bfloat1622float2(xr[i]);
+      ss += xv[j].x * xv[j].x + xv[j].y * xv[j].y;
+    }
+  }
+  ss = warp_sum(ss);
+  if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = ss;
+  __syncthreads();
+  float tot = 0.f;
+#pragma unroll
+  for (int i = 0; i < kRowThreads / 32; ++i) tot += s_part[i];
+  const float r = 1.0f / sqrtf(tot / (float)H + eps);
+#pragma unroll
+  for (int j = 0; j < kNormPairs; ++j) {
+    const int i = threadIdx.x + j * kRowThreads;
+    if (i < np) {
+      const float2 gg = __bfloat1622float2(gr[i]);
+      const __nv_bfloat162 o = __floats2bfloat162_rn(xv[j].x * r * gg.x, xv[j].y * r * gg.y);
+      yr[i] = o;
+      const float2 h = __bfloat1622float2(o);
+      const float2 sv = smooth != nullptr ? *reinterpret_cast<const float2*>(smooth + 2 * i) : make_float2(1.f, 1.f);
+      xv[j] = make_float2(__fmul_rn(h.x, sv.x), __fmul_rn(h.y, sv.y));
+    }
+  }
+  quantize_row_pairs<kNormPairs>(xv, np, s_part, xq + (size_t)m * H, dx + m);
+}
+
 // ---- RoPE table: cos/sin(pos * theta^(-2i/D)) evaluated in fp64, stored as fp32 -------------
 __global__ void rope_table_kernel(float2* table, int max_pos, int D, double theta) {
   const int half = D / 2;
@@ -312,6 +377,34 @@ swiglu_f16_kernel(const __nv_bfloat16* __restrict__ gu, int F, __nv_bfloat16* __
       hr[i] = __floats2half2_rn(of.x * scale, of.y * scale);
     }
   }
+}
+
+// SwiGLU whose output row is also smoothed and quantised per token for the W8A8 down projection.
+__global__ void __launch_bounds__(kRowThreads)
+swiglu_q8_kernel(const __nv_bfloat16* __restrict__ gu, const float* __restrict__ smooth, int F, __nv_bfloat16* __restrict__ act,
+                 int8_t* __restrict__ xq, float* __restrict__ dx) {
+  const int m = blockIdx.x;
+  const __nv_bfloat162* gr = reinterpret_cast<const __nv_bfloat162*>(gu + (size_t)m * 2 * F);
+  const __nv_bfloat162* ur = reinterpret_cast<const __nv_bfloat162*>(gu + (size_t)m * 2 * F + F);
+  __nv_bfloat162* ar = reinterpret_cast<__nv_bfloat162*>(act + (size_t)m * F);
+  __shared__ float s_part[kRowThreads / 32];
+  const int np = F / 2;
+  float2 v[kActPairs];
+#pragma unroll
+  for (int j = 0; j < kActPairs; ++j) {
+    const int i = threadIdx.x + j * kRowThreads;
+    v[j] = make_float2(0.f, 0.f);
+    if (i < np) {
+      const float2 gt = __bfloat1622float2(gr[i]);
+      const float2 up = __bfloat1622float2(ur[i]);
+      const __nv_bfloat162 o = __floats2bfloat162_rn(gt.x / (1.0f + expf(-gt.x)) * up.x, gt.y / (1.0f + expf(-gt.y)) * up.y);
+      ar[i] = o;
+      const float2 h = __bfloat1622float2(o);
+      const float2 sv = smooth != nullptr ? *reinterpret_cast<const float2*>(smooth + 2 * i) : make_float2(1.f, 1.f);
+      v[j] = make_float2(__fmul_rn(h.x, sv.x), __fmul_rn(h.y, sv.y));
+    }
+  }
+  quantize_row_pairs<kActPairs>(v, np, s_part, xq + (size_t)m * F, dx + m);
 }
 
 // ---- arg-max over the vocabulary, lowest index on ties ---------------------------------------
@@ -481,6 +574,22 @@ int launch_reduce_residual_rmsnorm_f16(const float* partial, int nsplit, int mpa
   if (H > 2 * kNormPairs * kRowThreads) { set_error("rmsnorm_f16: rows of %d elements (at most %d)", H, 2 * kNormPairs * kRowThreads); return QUASAR_ERR_SHAPE; }
   rmsnorm_f16_kernel<true><<<M, kRowThreads, 0, stream>>>(partial, nsplit, mpad, dx, dw, x, g, H, eps, y, reinterpret_cast<__half*>(y16),
                                                    inv);
+  QUASAR_LAUNCH_CHECK();
+  return QUASAR_OK;
+}
+
+int launch_rmsnorm_q8(const __nv_bfloat16* x, const __nv_bfloat16* g, const float* smooth, int M, int H, float eps,
+                      __nv_bfloat16* y, int8_t* xq, float* dx, cudaStream_t stream) {
+  if (H > 2 * kNormPairs * kRowThreads) { set_error("rmsnorm_q8: rows of %d elements (at most %d)", H, 2 * kNormPairs * kRowThreads); return QUASAR_ERR_SHAPE; }
+  rmsnorm_q8_kernel<<<M, kRowThreads, 0, stream>>>(x, g, smooth, H, eps, y, xq, dx);
+  QUASAR_LAUNCH_CHECK();
+  return QUASAR_OK;
+}
+
+int launch_swiglu_q8(const __nv_bfloat16* gu, const float* smooth, int M, int F, __nv_bfloat16* act, int8_t* xq, float* dx,
+                     cudaStream_t stream) {
+  if (F > 2 * kActPairs * kRowThreads) { set_error("swiglu_q8: rows of %d elements (at most %d)", F, 2 * kActPairs * kRowThreads); return QUASAR_ERR_SHAPE; }
+  swiglu_q8_kernel<<<M, kRowThreads, 0, stream>>>(gu, smooth, F, act, xq, dx);
   QUASAR_LAUNCH_CHECK();
   return QUASAR_OK;
 }

@@ -323,6 +323,14 @@ size_t linear_w8a8_workspace_bytes(int64_t M, int64_t N, int64_t K) {
   return kCounterBytes + align256((size_t)M * K) + align256((size_t)M * sizeof(float)) + partial;
 }
 
+// where launch_linear_w8a8 keeps the quantised activation rows and their step sizes inside its workspace: a kernel that
+// produces the operand may write them there itself and pass x == nullptr
+void linear_w8a8_operand_slots(void* workspace, int64_t M, int64_t K, int8_t** xq, float** dx) {
+  unsigned char* ws = reinterpret_cast<unsigned char*>(workspace);
+  *xq = reinterpret_cast<int8_t*>(ws + kCounterBytes);
+  *dx = reinterpret_cast<float*>(ws + kCounterBytes + align256((size_t)M * K));
+}
+
 int launch_linear_w8a8(const __nv_bfloat16* x, const float* smooth, const int8_t* w, const float* delta_w, int64_t M,
                        int64_t N, int64_t K, void* y, bool y_is_f32, const __nv_bfloat16* residual, int32_t* acc_out,
                        void* workspace, size_t workspace_bytes, int32_t* status, cudaStream_t stream) {
@@ -340,8 +348,10 @@ int launch_linear_w8a8(const __nv_bfloat16* x, const float* smooth, const int8_t
   float* dx = reinterpret_cast<float*>(ws + kCounterBytes + align256((size_t)M * K));
   int32_t* partial = reinterpret_cast<int32_t*>(ws + kCounterBytes + align256((size_t)M * K) + align256((size_t)M * sizeof(float)));
   // Eq. 9: fused smoothing + per-token quantisation of the activations
-  const int rc0 = launch_quantize_smoothed(x, smooth, kMultiply, M, K, xq, dx, stream);
-  if (rc0 != QUASAR_OK) return rc0;
+  if (x != nullptr) {   // (nullptr: the producer of the activations has already written xq and dx)
+    const int rc0 = launch_quantize_smoothed(x, smooth, kMultiply, M, K, xq, dx, stream);
+    if (rc0 != QUASAR_OK) return rc0;
+  }
   const SplitPlan p = plan_split(N, K);
   const size_t ybytes = y_is_f32 ? 4 : 2;
   if (M > 8 && umma_w8a8_usable(M < 80 ? M : 80, N, K)) {
