@@ -295,7 +295,9 @@ int launch_w(const GemmArgs& a, const SplitPlan& p, cudaStream_t stream) {
 
 }  // namespace
 
-size_t linear_workspace_bytes(int64_t M, int64_t N, int64_t K) {
+// the least a call needs: without the scratch of the stream kernel that blocks of at most 8 rows take on very large
+// matrices WHEN the workspace has room for it (they fall back to the warp-level kernel otherwise)
+static size_t linear_workspace_bytes_min(int64_t M, int64_t N, int64_t K) {
   const SplitPlan p = plan_split(N, K);
   const int64_t rows = M < kMaxRowsPerGemm ? M : kMaxRowsPerGemm;
   const size_t mpad = (size_t)((rows + 7) / 8) * 8;
@@ -308,11 +310,20 @@ size_t linear_workspace_bytes(int64_t M, int64_t N, int64_t K) {
     const size_t su = umma_w8a16_scratch_bytes(rows_u, N, K);
     partial = su > partial ? su : partial;
   }
-  if (M <= 8 && N * K >= kRows8UmmaMinBytes && umma_rows8_usable(M, N, K)) {
-    const size_t su = umma_rows8_scratch_bytes(M, N, K);
-    partial = su > partial ? su : partial;
-  }
   return counters + partial;
+}
+
+static bool rows8_stream_eligible(int64_t M, int64_t N, int64_t K) {
+  return M <= 8 && N * K >= kRows8UmmaMinBytes && umma_rows8_usable(M, N, K);
+}
+
+size_t linear_workspace_bytes(int64_t M, int64_t N, int64_t K) {
+  size_t need = linear_workspace_bytes_min(M, N, K);
+  if (rows8_stream_eligible(M, N, K)) {
+    const size_t su = kCounterBytes + umma_rows8_scratch_bytes(M, N, K);
+    need = su > need ? su : need;
+  }
+  return need;
 }
 
 int launch_linear(const __nv_bfloat16* x, const void* w, const float* delta, int weight_dtype, int64_t M, int64_t N,
@@ -323,7 +334,7 @@ int launch_linear(const __nv_bfloat16* x, const void* w, const float* delta, int
               (long long)M, (long long)N, (long long)K, (long long)kMaxChannels);
     return QUASAR_ERR_SHAPE;
   }
-  if (workspace_bytes < linear_workspace_bytes(M, N, K)) {
+  if (workspace_bytes < linear_workspace_bytes_min(M, N, K)) {
     set_error("linear: workspace of %zu bytes, need %zu", workspace_bytes, linear_workspace_bytes(M, N, K));
     return QUASAR_ERR_CAPACITY;
   }
@@ -345,7 +356,7 @@ int launch_linear(const __nv_bfloat16* x, const void* w, const float* delta, int
   // A matrix of LM-head size with at most 8 rows is a long pure stream: the persistent tcgen05 kernel that feeds
   // the int8 tiles straight into integer MMAs (activations as base-256 digits, umma_gemm.cu) sustains a higher
   // rate than the warp-level kernel there; below that size its two extra launches cost more than it gains.
-  if (weight_dtype == QUASAR_W_INT8 && M <= 8 && N * K >= kRows8UmmaMinBytes && umma_rows8_usable(M, N, K))
+  if (weight_dtype == QUASAR_W_INT8 && rows8_stream_eligible(M, N, K) && workspace_bytes >= kCounterBytes + umma_rows8_scratch_bytes(M, N, K))
     return launch_umma_rows8(x, reinterpret_cast<const int8_t*>(w), delta, M, N, K, y, y_is_f32, residual,
                              reinterpret_cast<unsigned char*>(workspace) + counters, status, stream);
   for (int64_t m0 = 0; m0 < M; m0 += kMaxRowsPerGemm) {
@@ -385,7 +396,7 @@ int launch_linear_static(const __nv_bfloat16* x, const void* w, const float* del
               (long long)M, (long long)N, (long long)K, (long long)kMaxChannels);
     return QUASAR_ERR_SHAPE;
   }
-  const size_t need = linear_workspace_bytes(M, N, K);
+  const size_t need = linear_workspace_bytes_min(M, N, K);
   if (need > kStaticScratchBytes) {
     set_error("linear_static: M=%lld N=%lld K=%lld needs %zu bytes of scratch, the built-in array holds %zu; "
               "use quasar_linear with a workspace",

@@ -75,3 +75,16 @@ def test_refuses_shapes_beyond_the_built_in_scratch():
     with pytest.raises(binding.QuasarError) as e:
         binding.quasar_linear_static(x, w, d, out)
     assert e.value.code == -3 and "scratch" in str(e.value)
+
+
+def test_a_very_large_matrix_with_few_rows_still_fits_the_built_in_scratch():
+    """With a workspace, blocks of at most 8 rows on matrices of LM-head size take a kernel that needs several MB of
+    scratch; without one the call must fall back to the kernel that needs none for this shape, not refuse it."""
+    m, n, k = 6, 33000, 4112
+    x = synth.normal_bf16((m, k), 1.0, seed=3, device="cuda")
+    q, d = binding.quasar_quantize(synth.normal_bf16((n, k), 0.02, seed=4, device="cuda"))
+    out = torch.zeros((m, n), dtype=torch.float32, device="cuda")
+    binding.quasar_linear_static(x, q, d, out)
+    want = binding.quasar_linear(x, q, d, out_f32=True)      # (the stream kernel: sums exact integers, so not bit-equal)
+    torch.cuda.synchronize()
+    assert torch.all((out - want).abs() <= 1e-5 * want.abs() + 3e-4)      # fp32 accumulation of 4112 terms of size ~0.02
