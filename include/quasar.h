@@ -87,6 +87,13 @@ int quasar_quantize(const void* w_bf16, int64_t N, int64_t K, int8_t* q_out, flo
  * workspace: at least quasar_linear_workspace_bytes(M, N, K) bytes; its first
  * use must find its first 64 KiB zero-filled, and every call leaves it reusable by the next call of
  * any shape (the split-K arrival counters live in those 64 KiB and reset themselves).
+ * Accumulation is fp32, or better: int8 weights with more than 8 rows run on the tcgen05 tensor
+ * cores (fp16 operands - exact for bf16 rows scaled by a power of two - fp32 sums in tensor
+ * memory); int8 weights with at most 8 rows on a matrix of at least 128 MiB run as an exact
+ * integer contraction (the activation row as 21-bit fixed point against a power of two above its
+ * largest magnitude).  Which kernel runs depends only on the shape and on whether the workspace
+ * has the size quasar_linear_workspace_bytes reports (a smaller one that still fits the fp32
+ * kernel is accepted); the kernels agree to fp32 accumulation accuracy, not bit for bit.
  * ---------------------------------------------------------------------- */
 int quasar_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, size_t* bytes_out /* host */);
 int quasar_linear(const void* x, const void* w, const float* delta, int32_t weight_dtype, int64_t M, int64_t N,
