@@ -761,7 +761,7 @@ SplitU plan_split_u(int64_t N, int64_t K) {
   SplitU p;
   p.nblocks = (int)((N + kTileN - 1) / kTileN);
   const int kbs = (int)((K + kTileKBytes - 1) / kTileKBytes);
-  int want = 148 / p.nblocks;                          // about one wave of CTAs; no split once the channel blocks fill the SMs
+  int want = 296 / p.nblocks;                          // about two CTAs per SM (what its shared memory holds); no split once the channel blocks fill them
   want = want < 1 ? 1 : (want > kbs ? kbs : want);
   want = want > 32 ? 32 : want;
   const int per = (kbs + want - 1) / want;
