@@ -103,6 +103,21 @@ __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* m
       : "memory");
 }
 
+// The same for a tile that is read once (weights): evict-first in L2, so that the stream does not push out the activation
+// rows and partial sums that are read again.
+__device__ __forceinline__ uint64_t l2_evict_first_policy() {
+  uint64_t policy;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;\n" : "=l"(policy));
+  return policy;
+}
+__device__ __forceinline__ void tma_load_2d_stream(void* smem_dst, const CUtensorMap* map, int x, int y, uint64_t* bar, uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;\n" ::"r"(
+          smem_u32(smem_dst)),
+      "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y), "l"(policy)
+      : "memory");
+}
+
 // K-major operand tile with 128-byte swizzle: rows of 128 bytes, groups of 8 rows 1024 bytes apart.
 __device__ __forceinline__ uint64_t umma_desc_sw128(const void* smem_tile) {
   uint64_t d = 0;
@@ -210,13 +225,14 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
 
   if (warp == 0) {
     if (lane == 0) {   // ---- TMA producer ----
+      const uint64_t wpolicy = l2_evict_first_policy();
       int s = 0;
       uint32_t ph = 0;
       for (int kb = 0; kb < nkb; ++kb) {
         if (!mbar_wait(empty + s, ph ^ 1u, abort_flag, a.error)) break;
         unsigned char* at = tiles + s * stage_bytes;
         mbar_expect_tx(full + s, (uint32_t)stage_bytes);
-        tma_load_2d(at, &map_w, k_begin + kb * kTileKBytes, n0, full + s);
+        tma_load_2d_stream(at, &map_w, k_begin + kb * kTileKBytes, n0, full + s, wpolicy);
         tma_load_2d(at + kTileN * kTileKBytes, &map_x, k_begin + kb * kTileKBytes, 0, full + s);
         if (++s == kStagesI8) { s = 0; ph ^= 1u; }
       }
@@ -410,13 +426,14 @@ umma_w8a16_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_consta
 
   if (warp == 0) {
     if (lane == 0) {   // ---- TMA producer ----
+      const uint64_t wpolicy = l2_evict_first_policy();
       int s = 0;
       uint32_t ph = 0;
       for (int kb = 0; kb < nkb; ++kb) {
         if (!mbar_wait(empty + s, ph ^ 1u, abort_flag, a.error)) break;
         unsigned char* st = tiles + s * stage_bytes;
         mbar_expect_tx(full + s, (uint32_t)(kRawBytes + b_bytes));
-        tma_load_2d(st + b_bytes, &map_w, k_begin + kb * 64, n0, full + s);                       // 128 rows x 64 int8
+        tma_load_2d_stream(st + b_bytes, &map_w, k_begin + kb * 64, n0, full + s, wpolicy);                       // 128 rows x 64 int8
         tma_load_2d(st, &map_x, (k_begin + kb * 64) * 2, 0, full + s);                            // Mpad rows x 64 fp16 (byte coordinate)
         if (++s == kStagesF16) { s = 0; ph ^= 1u; }
       }
@@ -635,6 +652,7 @@ umma_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
 
   if (warp == 0) {
     if (lane == 0) {   // ---- TMA producer: the digit rows once, then the weight tiles of every channel block ----
+      const uint64_t wpolicy = l2_evict_first_policy();
       mbar_expect_tx(b_full, (uint32_t)(nkb * nb * kTileKBytes));
       for (int kb = 0; kb < nkb; ++kb)
         tma_load_2d(b_res + (size_t)kb * nb * kTileKBytes, &map_xd, k_begin + kb * kTileKBytes, 0, b_full);
@@ -645,7 +663,7 @@ umma_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
         for (int kb = 0; kb < nkb; ++kb) {
           if (!(ok = mbar_wait(empty + s, ph ^ 1u, abort_flag, a.error))) break;
           mbar_expect_tx(full + s, (uint32_t)kATile);
-          tma_load_2d(ring + s * kATile, &map_w, k_begin + kb * kTileKBytes, t * kTileN, full + s);
+          tma_load_2d_stream(ring + s * kATile, &map_w, k_begin + kb * kTileKBytes, t * kTileN, full + s, wpolicy);
           if (++s == kStagesS) { s = 0; ph ^= 1u; }
         }
       }
