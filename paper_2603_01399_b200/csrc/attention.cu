@@ -133,6 +133,9 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 4) verify_attention_kernel(Att
   const __nv_bfloat16* kbase = a.kc + ((size_t)b * a.Hkv + hk) * (size_t)a.s_max * D;
   const __nv_bfloat16* vbase = a.vc + ((size_t)b * a.Hkv + hk) * (size_t)a.s_max * D;
 
+  // the cached K / V rows are read once per pass: evict-first in L2
+  uint64_t kv_policy;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;\n" : "=l"(kv_policy));
   auto stage_tile = [&](int buf, int k0) {
     __nv_bfloat16* kd = tiles + buf * 2 * kTileElems;
     __nv_bfloat16* vd = kd + kTileElems;
@@ -141,8 +144,8 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 4) verify_attention_kernel(Att
       if (k0 + key < key_end) {
         const uint32_t ks = (uint32_t)__cvta_generic_to_shared(kd + key * kStride + ch * 8);
         const uint32_t vs = (uint32_t)__cvta_generic_to_shared(vd + key * kStride + ch * 8);
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(ks), "l"(kbase + (size_t)(k0 + key) * D + ch * 8) : "memory");
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(vs), "l"(vbase + (size_t)(k0 + key) * D + ch * 8) : "memory");
+        asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;\n" ::"r"(ks), "l"(kbase + (size_t)(k0 + key) * D + ch * 8), "l"(kv_policy) : "memory");
+        asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;\n" ::"r"(vs), "l"(vbase + (size_t)(k0 + key) * D + ch * 8), "l"(kv_policy) : "memory");
       } else {
         *reinterpret_cast<uint4*>(kd + key * kStride + ch * 8) = make_uint4(0, 0, 0, 0);
         *reinterpret_cast<uint4*>(vd + key * kStride + ch * 8) = make_uint4(0, 0, 0, 0);
